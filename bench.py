@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the weight remap: full-model GB/s moved (read + write) on B200.
+
+A step is one pass of the whole hot path over one model: wb_remap on a bound plan (one
+persistent launch).  Layout description and planning happen once before the timed region,
+as in the paper (plan once in `connect`, execute every update); their wall time is reported
+in `config.plan_build_s`.  Prints one JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg4|cfg5]
+  python bench.py --impl reference ...      # the CPU oracle on a bounded sample, same metric
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from wb_workloads import TENSOR_DTYPE, SLICE_DTYPE, make_workload  # noqa: E402
+
+METRIC = "full-model weight remap GB/s (read+write)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one wb_remap launch, from the ncu capture
+# summarised under profiles/ (None until a capture for that workload exists)
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--scale", default="full")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tile-bytes", type=int, default=0)
+    ap.add_argument("--grid-ctas", type=int, default=0)
+    ap.add_argument("--path", default="remap", choices=["remap", "pack_unpack"])
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for p in self.samples:
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU baseline: the oracle, as it stands, on a bounded sample of the same workload
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(wl, fetch_src, budget_elems=60_000_000):
+    """Run the oracle on the first checkpoint tensors of the workload (in order) up to about
+    `budget_elems` elements.  Only the local tensors those touch are materialised on the host.
+    Returns (seconds, bytes moved, description)."""
+    from oracle import remap_oracle
+
+    picked, total = [], 0
+    for i, c in enumerate(wl.ckpt):
+        if picked and total + c.numel > budget_elems:
+            break
+        picked.append(i)
+        total += c.numel
+        if total >= budget_elems:
+            break
+    pick = np.array(picked)
+
+    def restrict(layout):
+        keep = np.isin(layout.slices["ckpt"], pick)
+        sl = layout.slices[keep].copy()
+        used = np.unique(sl["tensor"])
+        remap = {int(t): k for k, t in enumerate(used)}
+        sl["tensor"] = np.array([remap[int(t)] for t in sl["tensor"]], dtype=np.uint32)
+        return layout.tensors[used].copy(), sl, [int(t) for t in used]
+
+    t_t, t_s, t_used = restrict(wl.trainer)
+    r_t, r_s, _ = restrict(wl.rollout)
+    src = [fetch_src(k) for k in t_used]
+    shapes = [(c.rows, c.cols) for c in wl.ckpt]
+    t0 = time.perf_counter()
+    res = remap_oracle(shapes, t_t, t_s, r_t, r_s, src)
+    dt = time.perf_counter() - t0
+    es = 4 if wl.src_dtype == 0 else 2
+    ed = 4 if wl.dst_dtype == 0 else 2
+    moved = res.n_ids_consumed * es + res.n_written * ed
+    desc = (f"first {len(picked)} checkpoint tensors of {wl.name} in order "
+            f"({res.n_ids_consumed} elements), numpy oracle, single thread")
+    return dt, moved, desc
+
+
+def to_bits_np(t: torch.Tensor) -> np.ndarray:
+    t = t.detach().cpu().contiguous().reshape(-1)
+    if t.dtype == torch.float32:
+        return t.view(torch.int32).numpy().view(np.uint32)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = make_workload(args.workload, args.scale)
+    rng = np.random.default_rng(wl.seed)
+    cache = {}
+
+    def fetch(k):   # seeded synthetic source bits, generated on the host for the sampled tensors only
+        if k not in cache:
+            n = int(wl.trainer.tensors[k]["numel"])
+            v = (rng.standard_normal(n, dtype=np.float32) * 0.02)
+            cache[k] = v.view(np.uint32) if wl.src_dtype == 0 else \
+                to_bits_np(torch.from_numpy(v).to(torch.bfloat16))
+        return cache[k]
+
+    budget = 20_000_000
+    times, moved, desc = [], 0, ""
+    for _ in range(args.warmup):
+        oracle_sample(wl, fetch, budget)
+    for _ in range(args.steps):
+        dt, moved, desc = oracle_sample(wl, fetch, budget)
+        times.append(dt)
+    ms = 1e3 * sum(times) / max(len(times), 1)
+    value = moved / (ms * 1e-3) / 1e9 if times else 0.0
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "u16" if wl.src_dtype == 1 else "f32->bf16",
+           "data": "synthetic", "config": {"workload": wl.name, "note": "each step = bounded sample"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    from paper_2609_25442_b200 import binding as wb
+    from paper_2609_25442_b200.device import RankArenas, bind, require_cuda
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    require_cuda()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- inputs: resident in HBM before the timed region -------------------------------------
+    wl = make_workload(args.workload, args.scale)
+    t0 = time.perf_counter()
+    tl = wb.Layout(wl.trainer.tensors, wl.trainer.slices)
+    rl = wb.Layout(wl.rollout.tensors, wl.rollout.slices)
+    plan = wb.Plan(tl, rl, tile_bytes=args.tile_bytes, grid_ctas=args.grid_ctas)
+    plan_s = time.perf_counter() - t0
+    stats = plan.stats()
+    src = RankArenas(wl.trainer.tensors, dev, fill_byte=0)
+    dst = RankArenas(wl.rollout.tensors, dev, fill_byte=0)
+    wl.load_side("trainer", lambda i: wl.ckpt_values(i, dev), lambda k, t: src.tensors[k].copy_(t))
+    bind(plan, src, dst)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream().cuda_stream
+    bytes_step = stats["src_bytes_read"] + stats["dst_bytes_written"]
+
+    n_rounds = plan.num_rounds()
+    buckets = None
+    if args.path == "pack_unpack":
+        buckets = [torch.empty(max(plan.bucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
+                   for _ in range(2)]
+
+    def step():
+        if args.path == "remap":
+            plan.remap(stream)
+            return 1
+        for r in range(n_rounds):
+            b = buckets[r % 2].data_ptr()
+            plan.pack(r, b, stream)
+            plan.unpack(r, b, stream)
+        return 2 * n_rounds
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    launches = 0
+    evs[0].record()
+    for k in range(args.steps):
+        launches += step()
+        evs[k + 1].record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = evs[0].elapsed_time(evs[-1])
+    per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * bytes_step / (ms_per_step * 1e-3) / 1e9
+
+    # ---- roofline of the dominant (only) kernel --------------------------------------------------
+    peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        pass
+    launch_ms = float(np.mean(per_step)) / (1 if args.path == "remap" else 1)
+    achieved = bytes_step / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+                "peak_source": peak_src, "kernel": "wb_exec_kernel", "best_ms": float(min(per_step)),
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # ---- end to end through the host-buffer entry point -------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        try:
+            host_src = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in src.tensors]
+            host_dst = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in dst.tensors]
+            pinned = True
+        except RuntimeError:
+            host_src = [torch.empty(t.shape, dtype=t.dtype) for t in src.tensors]
+            host_dst = [torch.empty(t.shape, dtype=t.dtype) for t in dst.tensors]
+            pinned = False
+        for h, t in zip(host_src, src.tensors):
+            h.copy_(t)
+        hs = [t.data_ptr() for t in host_src]
+        hd = [t.data_ptr() for t in host_dst]
+        plan.remap_host(hs, hd, stream)
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.e2e_steps):
+            plan.remap_host(hs, hd, stream)
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e_ms /= args.e2e_steps
+        e2e = {"value": world * bytes_step / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": src.total_bytes(), "d2h_bytes_per_step": dst.total_bytes(),
+               "ms_per_step": e_ms, "steps": args.e2e_steps, "pinned": pinned}
+        del host_src, host_dst
+
+    # ---- CPU baseline (rank 0, N = 1 only) -----------------------------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        dt, moved, desc = oracle_sample(wl, lambda k: to_bits_np(src.tensors[k]))
+        cpu = {"value": moved / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
+               "seconds": dt}
+
+    if rank == 0:
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+               "scaling": "weak", "vs_baseline": None,
+               "dtype": {0: "f32", 1: "bf16"}[wl.src_dtype] + "->" + {0: "f32", 1: "bf16"}[wl.dst_dtype],
+               "data": "synthetic",
+               "config": {"workload": wl.name, "path": args.path, "l2": "inputs_larger_than_l2",
+                          "bytes_per_step": bytes_step, "tiles": stats["n_tiles_remap"],
+                          "slabs": stats["n_slabs"], "rounds": stats["n_rounds"],
+                          "grid_ctas": stats["grid_ctas"], "tile_bytes": stats["tile_bytes"],
+                          "plan_build_s": plan_s, "replicas_per_gpu": 1,
+                          "multi_gpu": "independent replicas, no collective"},
+               "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+               "gpu_launches": launches, "pct_of_8TBs_nominal": 100.0 * value / world / 8000.0}
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

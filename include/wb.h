@@ -1,0 +1,244 @@
+/*
+ * wb.h -- C ABI of the B200 weight-remap library.
+ *
+ * The library moves every model parameter element from a trainer's sharded layout into a
+ * rollout (inference) engine's layout, casting on the way, without reading any source
+ * element twice.  It follows the weight-transfer method of the WeightBridge paper:
+ *
+ *   - Section 3.1: each side's layout is a *source map*, a list of slice-copy operations
+ *     (optionally transposed) that say which checkpoint elements a worker's local tensors
+ *     hold.  Two local elements correspond iff the same checkpoint element supplies both.
+ *   - Section 3.2: a planner turns the correspondence into a non-redundant plan
+ *     (replicas on the trainer side each send a distinct slice; replicas on the rollout
+ *     side are fed from one copy), splits the model into roughly equal rounds that fit a
+ *     transfer-buffer budget, and an executor runs the plan every iteration with one
+ *     batched packing kernel (trainer side) and one batched assembly kernel (rollout side)
+ *     per round.
+ *
+ * Here all virtual trainer and rollout ranks are regions of ONE GPU's memory, so the wire
+ * between packing and assembly is a device buffer ("bucket"), and a fused path
+ * (wb_remap) goes from trainer tensors to rollout tensors directly.
+ *
+ * Conventions
+ *   - Every function returns a wb_status and never throws or aborts.  On error the
+ *     out-parameters are left untouched and nothing is launched.
+ *   - "host" / "device" is stated for every pointer.  The caller owns all weight memory,
+ *     all buckets and the CUDA stream; layouts and plans are opaque, owned by the library
+ *     and released with their _free function.
+ *   - A plan is immutable after wb_plan_bind and is reused for every model version
+ *     (Section 3: the plan is computed once, in `connect`, and executed per update).
+ *   - wb_pack / wb_unpack / wb_remap are asynchronous on the given stream, allocate
+ *     nothing and copy nothing between host and device.
+ *   - Local-tensor elements that no slice describes (e.g. FSDP padding) are never read on
+ *     the source side and never written on the destination side.
+ *   - Replicated source elements are assumed bit-identical.
+ */
+#ifndef WB_H_
+#define WB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  WB_OK = 0,
+  WB_ERR_INVALID_ARG = 1,      /* NULL pointer, bad index, unsupported strides              */
+  WB_ERR_DTYPE = 2,            /* unknown dtype, or mixed dtypes on one side                 */
+  WB_ERR_SHAPE_MISMATCH = 3,   /* one checkpoint tensor described with two different shapes  */
+  WB_ERR_OUT_OF_RANGE = 4,     /* a slice leaves its checkpoint tensor or its local tensor   */
+  WB_ERR_DST_OVERLAP = 5,      /* a destination element is described by two slices           */
+  WB_ERR_UNCOVERED = 6,        /* a destination element needs a checkpoint id no source holds*/
+  WB_ERR_BUCKET_TOO_SMALL = 7, /* the bucket budget cannot hold a single payload chunk       */
+  WB_ERR_OOM = 8,              /* host or device allocation failed                           */
+  WB_ERR_CUDA = 9,             /* a CUDA runtime call failed                                 */
+  WB_ERR_NOT_BOUND = 10,       /* execution requested before wb_plan_bind                    */
+  WB_ERR_INTERNAL = 11         /* a plan invariant does not hold (wb_plan_verify)            */
+} wb_status;
+
+typedef enum { WB_F32 = 0, WB_BF16 = 1 } wb_dtype;
+
+/* One local tensor of a virtual rank (a flat array of `numel` elements). */
+typedef struct {
+  uint32_t rank;   /* virtual rank that owns it (used for per-rank accounting and buckets) */
+  uint32_t dtype;  /* wb_dtype */
+  uint64_t numel;
+} wb_tensor_desc;
+
+/* One slice-copy operation of a source map (Section 3.1).  The rectangle
+ * [r0, r0+nr) x [c0, c0+nc) of checkpoint tensor `ckpt_tensor` -- viewed as a row-major
+ * ckpt_rows x ckpt_cols matrix; vectors are [1, n]; N-D tensors collapse leading dims --
+ * lives in local tensor `tensor` (an index into the layout's tensor table); checkpoint
+ * element (r0+i, c0+j) is local element local_off + i*stride_r + j*stride_c.
+ * Supported stride shapes: rows contiguous (stride_c == 1, stride_r >= nc) or, for a
+ * transposed copy, columns contiguous (stride_r == 1, stride_c >= nr); a stride whose
+ * extent is 1 is ignored.  Zero-area slices are ignored. */
+typedef struct {
+  uint32_t tensor;
+  uint32_t reserved;      /* must be 0 */
+  uint64_t local_off;
+  int64_t  stride_r;
+  int64_t  stride_c;
+  uint64_t ckpt_tensor;
+  uint64_t ckpt_rows;
+  uint64_t ckpt_cols;
+  uint64_t r0, c0, nr, nc;
+} wb_slice;
+
+typedef struct wb_layout wb_layout;
+typedef struct wb_plan wb_plan;
+
+/* Planner options; zero-initialise for defaults. */
+typedef struct {
+  uint64_t bucket_budget_bytes; /* bytes of transfer buffer one round may use; 0 = 4 GiB
+                                   (the paper's default RDMA budget, Appendix D)           */
+  uint32_t tile_bytes;          /* target bytes moved (read + written) per tile; 0 = auto   */
+  uint32_t grid_ctas;           /* thread blocks per launch; 0 = auto (multiple of 148 SMs) */
+  uint32_t flags;               /* WB_PLAN_* bits                                           */
+  uint32_t reserved;
+} wb_plan_opts;
+
+#define WB_PLAN_NO_REPLICA_SPLIT 1u /* read replicated source regions from the lowest rank
+                                       only instead of a distinct slice per replica        */
+
+typedef struct {
+  uint64_t n_ckpt_tensors;      /* checkpoint tensors the destination consumes              */
+  uint64_t n_slabs;             /* one-to-one (or one-to-k fan-out) copy rectangles          */
+  uint64_t n_fanout_slabs;      /* slabs with more than one destination                      */
+  uint64_t n_rounds;
+  uint64_t n_tiles_remap;
+  uint64_t n_tiles_pack;        /* summed over rounds                                        */
+  uint64_t n_tiles_unpack;
+  uint64_t src_elems_read;      /* distinct checkpoint elements read == source elements read */
+  uint64_t dst_elems_written;
+  uint64_t src_bytes_read;
+  uint64_t dst_bytes_written;
+  uint64_t replica_elems_skipped; /* source elements never read because a replica supplies them */
+  uint64_t bucket_bytes_total;  /* payload + alignment padding, summed over rounds           */
+  uint64_t bucket_bytes_max;    /* largest round                                             */
+  uint64_t table_bytes;         /* device bytes of all tile tables                           */
+  uint64_t remap_cta_bytes_max; /* bytes moved by the most loaded thread block (remap)       */
+  uint64_t remap_cta_bytes_mean;
+  uint32_t grid_ctas;
+  uint32_t tile_bytes;
+  double   build_seconds;       /* wall time of wb_plan_build                                */
+} wb_plan_stats_t;
+
+/* One payload of a round's bucket: the checkpoint rectangle it carries, row-major in the
+ * destination dtype, starting `bucket_off` bytes into the bucket (16-byte aligned). */
+typedef struct {
+  uint32_t sender;        /* virtual trainer rank the bytes come from                       */
+  uint32_t receiver;      /* virtual rollout rank the payload is addressed to               */
+  uint64_t ckpt_tensor;
+  uint64_t r0, c0, nr, nc;
+  uint64_t bucket_off;
+  uint32_t dtype;         /* wb_dtype of the payload (== destination dtype)                 */
+  uint32_t n_dst;         /* rollout tensors this payload is written to by wb_unpack        */
+} wb_bucket_entry;
+
+/* Host view of one tile of a tile table (for verification on the host).  A tile copies
+ * dst[dst_off + i*dst_sr + j*dst_sc] = cast(src[src_off + i*src_sr + j*src_sc]) for
+ * i < nr, j < nc; a tensor index of -1 means the bucket, with offsets in elements of the
+ * bucket dtype.  A fan-out tile appears once per destination; entries after the first
+ * carry WB_TILE_FANOUT_CONT and re-use the first entry's source read. */
+typedef struct {
+  int32_t  src_tensor, dst_tensor;
+  uint64_t src_off, dst_off;
+  uint32_t nr, nc;
+  uint32_t src_sr, src_sc, dst_sr, dst_sc;
+  uint32_t kind;          /* kernel path hint: 0 rows, 1 transpose, 2 element-wise          */
+  uint32_t flags;
+  uint32_t cta;           /* thread block the tile is assigned to                           */
+  uint32_t reserved;
+} wb_tile_view;
+
+#define WB_TILE_FANOUT_CONT 1u
+
+enum { WB_TABLE_REMAP = 0, WB_TABLE_PACK = 1, WB_TABLE_UNPACK = 2 };
+
+/* ---- layouts (host only) --------------------------------------------------------------
+ * wb_layout_describe: ingest one side's source map (Section 3.1, "sequence of slice-copy
+ * operations ... each optionally involving transpose").  `tensors` and `slices` are host
+ * arrays, copied.  Checks indices, dtypes, stride shapes, that every slice stays inside its
+ * checkpoint tensor and its local tensor, and that a checkpoint tensor has one shape.
+ * Errors: INVALID_ARG, DTYPE, SHAPE_MISMATCH, OUT_OF_RANGE, OOM. */
+wb_status wb_layout_describe(const wb_tensor_desc* tensors, size_t n_tensors,
+                             const wb_slice* slices, size_t n_slices, wb_layout** out);
+void wb_layout_free(wb_layout* layout);
+
+/* ---- planning (host only, no CUDA call) -------------------------------------------------
+ * wb_plan_build: Section 3.2.  Intersects the two source maps per checkpoint tensor
+ * (element correspondence), de-duplicates replicas on both sides so that every consumed
+ * checkpoint element is read exactly once (trainer replicas each supply a distinct slice;
+ * rollout replicas are written by fan-out from one read), cuts the resulting slabs into
+ * load-balanced tiles assigned to thread blocks, and partitions the model into rounds whose
+ * buckets fit `bucket_budget_bytes`.  `trainer` is the source side, `rollout` the
+ * destination side; swap them for the inverse transfer.  `opts` may be NULL.
+ * Errors: INVALID_ARG, DTYPE, SHAPE_MISMATCH, DST_OVERLAP, UNCOVERED, BUCKET_TOO_SMALL, OOM. */
+wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* rollout,
+                        const wb_plan_opts* opts, wb_plan** out);
+void wb_plan_free(wb_plan* plan);
+
+/* wb_plan_verify: re-derives, by interval arithmetic over the slabs only, that destination
+ * spans are pairwise disjoint and cover every described destination element, that source
+ * spans of different slabs are disjoint in checkpoint coordinates (each id read once), and
+ * that every tile of every table stays inside its tensors / bucket.  INTERNAL on failure. */
+wb_status wb_plan_verify(const wb_plan* plan);
+wb_status wb_plan_stats(const wb_plan* plan, wb_plan_stats_t* out /* host */);
+/* Bytes a virtual rank sends (side 0: trainer egress, source dtype) or receives
+ * (side 1: rollout ingress through buckets, destination dtype).  Section 3.2: trainers
+ * collectively transmit exactly one copy of the model. */
+wb_status wb_plan_rank_bytes(const wb_plan* plan, int side, uint32_t rank, uint64_t* out);
+
+size_t wb_plan_num_rounds(const wb_plan* plan);
+size_t wb_plan_bucket_bytes(const wb_plan* plan, size_t round);   /* 0 if round is invalid */
+/* Directory of a round's bucket.  Writes up to `cap` entries to `out` (host, may be NULL)
+ * and the total count to *n. */
+wb_status wb_plan_bucket_entries(const wb_plan* plan, size_t round, wb_bucket_entry* out,
+                                 size_t cap, size_t* n);
+/* Host view of a tile table (`which` = WB_TABLE_*; `round` ignored for WB_TABLE_REMAP). */
+wb_status wb_plan_tiles(const wb_plan* plan, int which, size_t round, wb_tile_view* out,
+                        size_t cap, size_t* n);
+
+/* ---- binding (device memory; synchronous; allocates the plan's device tables) ------------
+ * src_base[i] / dst_base[i]: DEVICE address of trainer / rollout local tensor i, aligned to
+ * its element size (16-byte alignment lets the kernels use their widest path).  Host
+ * arrays of device pointers, copied.  May be called again to re-bind.  The bound regions
+ * must not alias each other.  Errors: INVALID_ARG, OOM, CUDA. */
+wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, size_t n_src,
+                       void* const* dst_base, size_t n_dst);
+
+/* ---- execution (device; asynchronous on `cuda_stream`, a cudaStream_t or NULL) -----------
+ * wb_remap: the fused path, trainer tensors -> rollout tensors in one persistent launch:
+ * dst[x] = cast(src[y]) for every corresponding pair (Section 3.1), fp32 -> bf16 by
+ * round-to-nearest-even, same dtype = bit copy.
+ * wb_pack: Section 3.2 packing kernel: this round's source slabs -> checkpoint-format
+ * payloads in `bucket` (device, >= wb_plan_bucket_bytes(round), 16-byte aligned), cast
+ * applied here so the bucket carries destination-dtype bytes.
+ * wb_unpack: Section 3.2 assembly kernel: payloads of `bucket` -> rollout tensors (fused
+ * qkv / gate_up concatenation, head regrouping, expert stacking, transposition, fan-out).
+ * Errors: INVALID_ARG, NOT_BOUND, CUDA. */
+wb_status wb_remap(const wb_plan* plan, void* cuda_stream);
+wb_status wb_pack(const wb_plan* plan, size_t round, void* bucket, void* cuda_stream);
+wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bucket, void* cuda_stream);
+
+/* wb_remap_host: the same transfer for callers whose weights are in HOST memory:
+ * copies every trainer tensor host -> its bound device region, runs wb_remap, copies every
+ * rollout tensor back, all on `cuda_stream`, and returns without synchronising.
+ * host_src[i] / host_dst[i]: HOST addresses (page-locked for real asynchrony) of the
+ * tensors in table order.  Errors: INVALID_ARG, NOT_BOUND, CUDA. */
+wb_status wb_remap_host(const wb_plan* plan, const void* const* host_src, size_t n_src,
+                        void* const* host_dst, size_t n_dst, void* cuda_stream);
+
+/* Number of kernels wb_remap / wb_pack / wb_unpack launch per call (always 1). */
+int wb_launches_per_call(void);
+
+const char* wb_status_str(wb_status s);
+const char* wb_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WB_H_ */

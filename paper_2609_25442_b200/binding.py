@@ -1,0 +1,244 @@
+"""Thin ctypes binding of the C ABI in include/wb.h.
+
+Argument marshalling only: every step of the remap runs inside libwb.so.  Function and
+type names mirror the header.  There is no fallback: if the library cannot be built or
+loaded, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+WB_OK = 0
+WB_F32, WB_BF16 = 0, 1
+WB_TABLE_REMAP, WB_TABLE_PACK, WB_TABLE_UNPACK = 0, 1, 2
+WB_TILE_FANOUT_CONT = 1
+WB_PLAN_NO_REPLICA_SPLIT = 1
+
+STATUS_NAMES = {
+    0: "WB_OK", 1: "WB_ERR_INVALID_ARG", 2: "WB_ERR_DTYPE", 3: "WB_ERR_SHAPE_MISMATCH",
+    4: "WB_ERR_OUT_OF_RANGE", 5: "WB_ERR_DST_OVERLAP", 6: "WB_ERR_UNCOVERED",
+    7: "WB_ERR_BUCKET_TOO_SMALL", 8: "WB_ERR_OOM", 9: "WB_ERR_CUDA", 10: "WB_ERR_NOT_BOUND",
+    11: "WB_ERR_INTERNAL",
+}
+
+
+class WbError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        self.name = STATUS_NAMES.get(status, str(status))
+        msg = _lib.wb_status_str(status).decode() if _lib is not None else ""
+        super().__init__(f"{where}: {self.name} ({msg})")
+
+
+class wb_tensor_desc(C.Structure):
+    _fields_ = [("rank", C.c_uint32), ("dtype", C.c_uint32), ("numel", C.c_uint64)]
+
+
+class wb_slice(C.Structure):
+    _fields_ = [("tensor", C.c_uint32), ("reserved", C.c_uint32), ("local_off", C.c_uint64),
+                ("stride_r", C.c_int64), ("stride_c", C.c_int64),
+                ("ckpt_tensor", C.c_uint64), ("ckpt_rows", C.c_uint64), ("ckpt_cols", C.c_uint64),
+                ("r0", C.c_uint64), ("c0", C.c_uint64), ("nr", C.c_uint64), ("nc", C.c_uint64)]
+
+
+class wb_plan_opts(C.Structure):
+    _fields_ = [("bucket_budget_bytes", C.c_uint64), ("tile_bytes", C.c_uint32),
+                ("grid_ctas", C.c_uint32), ("flags", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class wb_plan_stats_t(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in (
+        "n_ckpt_tensors", "n_slabs", "n_fanout_slabs", "n_rounds", "n_tiles_remap", "n_tiles_pack",
+        "n_tiles_unpack", "src_elems_read", "dst_elems_written", "src_bytes_read",
+        "dst_bytes_written", "replica_elems_skipped", "bucket_bytes_total", "bucket_bytes_max",
+        "table_bytes", "remap_cta_bytes_max", "remap_cta_bytes_mean")] + \
+        [("grid_ctas", C.c_uint32), ("tile_bytes", C.c_uint32), ("build_seconds", C.c_double)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+BUCKET_ENTRY_DTYPE = np.dtype([
+    ("sender", "<u4"), ("receiver", "<u4"), ("ckpt_tensor", "<u8"), ("r0", "<u8"), ("c0", "<u8"),
+    ("nr", "<u8"), ("nc", "<u8"), ("bucket_off", "<u8"), ("dtype", "<u4"), ("n_dst", "<u4")])
+TILE_VIEW_DTYPE = np.dtype([
+    ("src_tensor", "<i4"), ("dst_tensor", "<i4"), ("src_off", "<u8"), ("dst_off", "<u8"),
+    ("nr", "<u4"), ("nc", "<u4"), ("src_sr", "<u4"), ("src_sc", "<u4"), ("dst_sr", "<u4"),
+    ("dst_sc", "<u4"), ("kind", "<u4"), ("flags", "<u4"), ("cta", "<u4"), ("reserved", "<u4")])
+assert BUCKET_ENTRY_DTYPE.itemsize == 64 and TILE_VIEW_DTYPE.itemsize == 64
+
+EXPORTS = [
+    "wb_layout_describe", "wb_layout_free", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
+    "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
+    "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
+    "wb_remap_host", "wb_launches_per_call", "wb_status_str", "wb_version",
+]
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load() -> C.CDLL:
+    """Build (if stale) and load libwb.so; raises if that is impossible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    lib = C.CDLL(path)
+    vp, sz = C.c_void_p, C.c_size_t
+    lib.wb_layout_describe.argtypes = [vp, sz, vp, sz, C.POINTER(vp)]
+    lib.wb_layout_free.argtypes = [vp]
+    lib.wb_layout_free.restype = None
+    lib.wb_plan_build.argtypes = [vp, vp, C.POINTER(wb_plan_opts), C.POINTER(vp)]
+    lib.wb_plan_free.argtypes = [vp]
+    lib.wb_plan_free.restype = None
+    lib.wb_plan_verify.argtypes = [vp]
+    lib.wb_plan_stats.argtypes = [vp, C.POINTER(wb_plan_stats_t)]
+    lib.wb_plan_rank_bytes.argtypes = [vp, C.c_int, C.c_uint32, C.POINTER(C.c_uint64)]
+    lib.wb_plan_num_rounds.argtypes = [vp]
+    lib.wb_plan_num_rounds.restype = sz
+    lib.wb_plan_bucket_bytes.argtypes = [vp, sz]
+    lib.wb_plan_bucket_bytes.restype = sz
+    lib.wb_plan_bucket_entries.argtypes = [vp, sz, vp, sz, C.POINTER(sz)]
+    lib.wb_plan_tiles.argtypes = [vp, C.c_int, sz, vp, sz, C.POINTER(sz)]
+    lib.wb_plan_bind.argtypes = [vp, vp, sz, vp, sz]
+    lib.wb_remap.argtypes = [vp, vp]
+    lib.wb_pack.argtypes = [vp, sz, vp, vp]
+    lib.wb_unpack.argtypes = [vp, sz, vp, vp]
+    lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
+    lib.wb_launches_per_call.restype = C.c_int
+    lib.wb_status_str.argtypes = [C.c_int]
+    lib.wb_status_str.restype = C.c_char_p
+    lib.wb_version.restype = C.c_char_p
+    _lib = lib
+    return lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != WB_OK:
+        raise WbError(status, where)
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    arr = (C.c_void_p * max(len(ptrs), 1))()
+    for i, p in enumerate(ptrs):
+        arr[i] = p
+    return arr
+
+
+class Layout:
+    """Owns a wb_layout*."""
+
+    def __init__(self, tensors: np.ndarray, slices: np.ndarray):
+        lib = load()
+        tensors = np.ascontiguousarray(tensors)
+        slices = np.ascontiguousarray(slices)
+        assert tensors.dtype.itemsize == C.sizeof(wb_tensor_desc)
+        assert slices.dtype.itemsize == C.sizeof(wb_slice)
+        self.n_tensors = len(tensors)
+        self.handle = C.c_void_p()
+        _check(lib.wb_layout_describe(tensors.ctypes.data, len(tensors), slices.ctypes.data,
+                                      len(slices), C.byref(self.handle)), "wb_layout_describe")
+
+    def __del__(self):
+        if _lib is not None and getattr(self, "handle", None):
+            _lib.wb_layout_free(self.handle)
+            self.handle = None
+
+
+def wb_layout_describe(tensors: np.ndarray, slices: np.ndarray) -> Layout:
+    return Layout(tensors, slices)
+
+
+class Plan:
+    """Owns a wb_plan*."""
+
+    def __init__(self, trainer: Layout, rollout: Layout, bucket_budget_bytes: int = 0,
+                 tile_bytes: int = 0, grid_ctas: int = 0, flags: int = 0):
+        lib = load()
+        opts = wb_plan_opts(bucket_budget_bytes, tile_bytes, grid_ctas, flags, 0)
+        self.handle = C.c_void_p()
+        self.n_src, self.n_dst = trainer.n_tensors, rollout.n_tensors
+        _check(lib.wb_plan_build(trainer.handle, rollout.handle, C.byref(opts), C.byref(self.handle)),
+               "wb_plan_build")
+
+    def __del__(self):
+        if _lib is not None and getattr(self, "handle", None):
+            _lib.wb_plan_free(self.handle)
+            self.handle = None
+
+    # ---- host queries ---------------------------------------------------------------------
+    def verify(self) -> None:
+        _check(_lib.wb_plan_verify(self.handle), "wb_plan_verify")
+
+    def stats(self) -> dict:
+        st = wb_plan_stats_t()
+        _check(_lib.wb_plan_stats(self.handle, C.byref(st)), "wb_plan_stats")
+        return st.as_dict()
+
+    def rank_bytes(self, side: int, rank: int) -> int:
+        out = C.c_uint64()
+        _check(_lib.wb_plan_rank_bytes(self.handle, side, rank, C.byref(out)), "wb_plan_rank_bytes")
+        return out.value
+
+    def num_rounds(self) -> int:
+        return _lib.wb_plan_num_rounds(self.handle)
+
+    def bucket_bytes(self, rnd: int) -> int:
+        return _lib.wb_plan_bucket_bytes(self.handle, rnd)
+
+    def bucket_entries(self, rnd: int) -> np.ndarray:
+        n = C.c_size_t()
+        _check(_lib.wb_plan_bucket_entries(self.handle, rnd, None, 0, C.byref(n)), "wb_plan_bucket_entries")
+        out = np.zeros(n.value, BUCKET_ENTRY_DTYPE)
+        _check(_lib.wb_plan_bucket_entries(self.handle, rnd, out.ctypes.data, n.value, C.byref(n)),
+               "wb_plan_bucket_entries")
+        return out
+
+    def tiles(self, which: int, rnd: int = 0) -> np.ndarray:
+        n = C.c_size_t()
+        _check(_lib.wb_plan_tiles(self.handle, which, rnd, None, 0, C.byref(n)), "wb_plan_tiles")
+        out = np.zeros(n.value, TILE_VIEW_DTYPE)
+        _check(_lib.wb_plan_tiles(self.handle, which, rnd, out.ctypes.data, n.value, C.byref(n)),
+               "wb_plan_tiles")
+        return out
+
+    # ---- device ------------------------------------------------------------------------------
+    def bind(self, src_ptrs: Sequence[int], dst_ptrs: Sequence[int]) -> None:
+        a, b = _ptr_array(src_ptrs), _ptr_array(dst_ptrs)
+        _check(_lib.wb_plan_bind(self.handle, a, len(src_ptrs), b, len(dst_ptrs)), "wb_plan_bind")
+
+    def remap(self, stream: int = 0) -> None:
+        _check(_lib.wb_remap(self.handle, stream), "wb_remap")
+
+    def pack(self, rnd: int, bucket_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_pack(self.handle, rnd, bucket_ptr, stream), "wb_pack")
+
+    def unpack(self, rnd: int, bucket_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_unpack(self.handle, rnd, bucket_ptr, stream), "wb_unpack")
+
+    def remap_host(self, host_src_ptrs: Sequence[int], host_dst_ptrs: Sequence[int], stream: int = 0) -> None:
+        a, b = _ptr_array(host_src_ptrs), _ptr_array(host_dst_ptrs)
+        _check(_lib.wb_remap_host(self.handle, a, len(host_src_ptrs), b, len(host_dst_ptrs), stream),
+               "wb_remap_host")
+
+
+def wb_plan_build(trainer: Layout, rollout: Layout, **opts) -> Plan:
+    return Plan(trainer, rollout, **opts)
+
+
+def wb_launches_per_call() -> int:
+    return load().wb_launches_per_call()
+
+
+def wb_version() -> str:
+    return load().wb_version().decode()

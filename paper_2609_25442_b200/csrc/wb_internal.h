@@ -1,0 +1,166 @@
+// Internal data structures shared by the host planner and the CUDA executor.
+#pragma once
+
+#include <cstdint>
+#include <cstddef>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "wb.h"
+
+namespace wbi {
+
+struct Rect {
+  uint64_t r0, c0, nr, nc;
+  uint64_t area() const { return nr * nc; }
+  uint64_t r1() const { return r0 + nr; }
+  uint64_t c1() const { return c0 + nc; }
+};
+
+inline bool intersect(const Rect& a, const Rect& b, Rect* out) {
+  uint64_t r0 = a.r0 > b.r0 ? a.r0 : b.r0;
+  uint64_t c0 = a.c0 > b.c0 ? a.c0 : b.c0;
+  uint64_t r1 = a.r1() < b.r1() ? a.r1() : b.r1();
+  uint64_t c1 = a.c1() < b.c1() ? a.c1() : b.c1();
+  if (r1 <= r0 || c1 <= c0) return false;
+  if (out) *out = Rect{r0, c0, r1 - r0, c1 - c0};
+  return true;
+}
+
+// A validated slice-copy operation.  Checkpoint element (r0+i, c0+j) is local element
+// off + i*pitch + j (rows contiguous) or off + j*pitch + i (transposed: columns contiguous).
+struct NSlice {
+  uint32_t tensor;
+  uint32_t ckpt_index;   // index into wb_layout::ckpts
+  uint64_t off;
+  uint64_t pitch;
+  bool transposed;
+  Rect rect;
+  uint64_t elem(uint64_t r, uint64_t c) const {
+    uint64_t i = r - rect.r0, j = c - rect.c0;
+    return transposed ? off + j * pitch + i : off + i * pitch + j;
+  }
+  uint64_t sr() const { return transposed ? 1 : pitch; }
+  uint64_t sc() const { return transposed ? pitch : 1; }
+};
+
+struct CkptInfo {
+  uint64_t id, rows, cols;
+  uint32_t first, count;   // range in wb_layout::by_ckpt
+};
+
+}  // namespace wbi
+
+struct wb_layout {
+  std::vector<wb_tensor_desc> tensors;
+  std::vector<wbi::NSlice> slices;
+  std::vector<wbi::CkptInfo> ckpts;        // sorted by id
+  std::vector<uint32_t> by_ckpt;           // slice indices grouped by checkpoint tensor
+  uint32_t dtype = 0;                      // uniform element type of the side
+  uint32_t n_ranks = 0;
+};
+
+namespace wbi {
+
+enum : uint32_t { KIND_ROWS = 0, KIND_TRANS = 1, KIND_ELEM = 2 };
+
+// Resident thread blocks per SM the executor kernel is compiled for; the planner's default
+// grid is kNumSMs * kCtasPerSM so that one launch is exactly one wave on a B200.
+constexpr uint32_t kNumSMs = 148;
+constexpr uint32_t kCtasPerSM = 3;
+
+// Host form of a tile: tensor indices and element offsets (resolved to addresses at bind).
+struct HTile {
+  int32_t src_tensor, dst_tensor;     // -1 = bucket
+  uint64_t src_off, dst_off;          // elements
+  uint32_t nr, nc;
+  uint32_t ssr, ssc, dsr, dsc;        // element strides over (i, j)
+  uint32_t kind;
+  uint32_t n_extra, extra;            // fan-out destinations beyond the first
+  uint32_t cta;
+  uint64_t bytes;                     // bytes moved (read + all writes)
+};
+
+struct HDst {
+  int32_t tensor;
+  uint64_t off;
+  uint32_t sr, sc;
+};
+
+// Device form.  `src` / `dst` are absolute device addresses for bound tensors, or byte
+// offsets into the bucket for the side of a pack / unpack table that is the bucket (the
+// kernel adds the bucket base to every tile of such a table).
+struct alignas(16) DTile {
+  uint64_t src;
+  uint64_t dst;
+  uint32_t nr, nc;
+  uint32_t ssr, ssc;
+  uint32_t dsr, dsc;
+  uint32_t kind_extra;   // kind | n_extra << 8
+  uint32_t extra;
+};
+static_assert(sizeof(DTile) == 48, "tile descriptor is three 16-byte words");
+
+struct alignas(16) DDst {
+  uint64_t dst;
+  uint32_t sr, sc;
+};
+static_assert(sizeof(DDst) == 16, "");
+
+struct TileTable {
+  std::vector<HTile> tiles;           // ordered by thread block, then checkpoint order
+  std::vector<HDst> extras;
+  std::vector<uint32_t> cta_begin;    // grid + 1 offsets into tiles
+  uint64_t bytes_max_cta = 0, bytes_total = 0;
+  // device copies (owned by the plan; allocated at bind)
+  DTile* d_tiles = nullptr;
+  DDst* d_extras = nullptr;
+  uint32_t* d_cta_begin = nullptr;
+};
+
+struct Slab {
+  uint32_t ckpt_index;      // into the destination layout's ckpts
+  Rect rect;
+  uint32_t src_slice;       // into source layout slices
+  uint32_t dst_begin, dst_count;   // into wb_plan::slab_dsts (destination slice indices)
+  uint32_t sender, receiver;       // virtual ranks
+};
+
+struct Payload {
+  uint32_t slab;
+  Rect rect;
+  uint64_t bucket_off;      // bytes
+};
+
+struct Round {
+  std::vector<Payload> payloads;
+  uint64_t bucket_bytes = 0;
+  TileTable pack, unpack;
+};
+
+}  // namespace wbi
+
+struct wb_plan {
+  wb_layout src, dst;                   // private copies
+  wb_plan_opts opts{};
+  std::vector<wbi::Slab> slabs;
+  std::vector<uint32_t> slab_dsts;
+  std::vector<wbi::Round> rounds;
+  wbi::TileTable remap;
+  std::vector<uint64_t> egress, ingress;
+  wb_plan_stats_t stats{};
+  uint32_t grid = 0;
+  // binding
+  bool bound = false;
+  int device = -1;
+  std::vector<const void*> src_base;
+  std::vector<void*> dst_base;
+  void* d_arena = nullptr;              // one device allocation holding every table
+  size_t arena_bytes = 0;
+};
+
+namespace wbi {
+// implemented in wb_exec.cu
+void release_device_tables(wb_plan* plan);
+}

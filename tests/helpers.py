@@ -92,6 +92,9 @@ def fuzz_case(seed: int, src_dtype=WB_F32, dst_dtype=WB_BF16, n_ckpt=None, max_d
                 for r in rects:
                     if rng.uniform() < 0.25:
                         extra.append(r)
+                if rng.uniform() < 0.5:      # a replica that straddles partition boundaries
+                    a0, b0 = rng.randint(0, rows - 1), rng.randint(0, cols - 1)
+                    extra.append((a0, b0, rng.randint(1, rows - a0), rng.randint(1, cols - b0)))
             for (r0, c0, nr, nc) in rects + extra:
                 loc = rng.randint(0, n_local - 1)
                 transposed = rng.uniform() < 0.3

@@ -1,0 +1,230 @@
+"""Parity of the CUDA path against the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import CANARY, DeviceCase, prefill_bits
+from helpers import ckpt_shapes, from_bits, fuzz_case, random_bits, scatter_checkpoint, to_bits
+from oracle import checkpoint_view, remap_oracle
+from oracle.cast import cast_bits, f32_to_bf16_bits
+from paper_2609_25442_b200 import binding as wb
+from paper_2609_25442_b200.device import RankArenas, bind
+from wb_workloads import WB_BF16, WB_F32, Layout, make_workload
+
+pytestmark = pytest.mark.gpu
+BITS = {WB_F32: np.uint32, WB_BF16: np.uint16}
+
+CASES = [("cfg1", "full"), ("cfg1b", "full"), ("cfg1c", "full"), ("cfg2", "small"), ("cfg3", "small"),
+         ("cfg4", "small"), ("cfg5", "small"), ("cfg2", "medium"), ("cfg3", "medium"),
+         ("cfg4", "medium"), ("cfg5", "medium")]
+
+
+@pytest.fixture(scope="module")
+def device():
+    assert torch.cuda.is_available()
+    return torch.device("cuda:0")
+
+
+def oracle_for(case: DeviceCase):
+    wl = case.wl
+    return remap_oracle(ckpt_shapes(wl), case.trainer.tensors, case.trainer.slices,
+                        case.rollout.tensors, case.rollout.slices, case.src_bits(),
+                        prefill_bits(case.rollout, BITS[int(case.rollout.tensors[0]["dtype"])]))
+
+
+def assert_dst_equals(case, want):
+    got = case.dst_bits()
+    for k in range(len(got)):
+        if not np.array_equal(got[k], want.dst[k]):
+            bad = np.nonzero(got[k] != want.dst[k])[0]
+            raise AssertionError(f"{case.rollout.names[k]}: {bad.size} of {got[k].size} elements differ, "
+                                 f"first at {bad[:5]}")
+    assert case.gaps_intact()
+
+
+@pytest.mark.parametrize("name,scale", CASES)
+def test_remap_matches_oracle(device, name, scale):
+    case = DeviceCase(make_workload(name, scale), device)
+    want = oracle_for(case)
+    case.plan.remap()
+    torch.cuda.synchronize()
+    assert_dst_equals(case, want)
+    # a second call on the same plan gives the same result (the plan is reused every update)
+    case.reset_dst()
+    case.plan.remap()
+    torch.cuda.synchronize()
+    assert_dst_equals(case, want)
+
+
+@pytest.mark.parametrize("name,scale,budget", [
+    ("cfg1", "full", 0), ("cfg1b", "full", 1 << 20), ("cfg3", "small", 1 << 20), ("cfg4", "small", 1 << 19),
+    ("cfg5", "small", 1 << 18), ("cfg2", "medium", 16 << 20), ("cfg3", "medium", 32 << 20),
+    ("cfg5", "medium", 16 << 20)])
+def test_pack_unpack_matches_oracle(device, name, scale, budget):
+    wl = make_workload(name, scale)
+    case = DeviceCase(wl, device, bucket_budget_bytes=budget)
+    want = oracle_for(case)
+    src_bits = case.src_bits()
+    shapes = ckpt_shapes(wl)
+    n_rounds = case.plan.num_rounds()
+    if budget:
+        assert n_rounds > 1
+    views = {}
+    for r in range(n_rounds):
+        nb = case.plan.bucket_bytes(r)
+        bucket = torch.full((nb + 64,), 0x5A, dtype=torch.uint8, device=device)
+        case.plan.pack(r, bucket.data_ptr())
+        torch.cuda.synchronize()
+        assert bool((bucket[nb:] == 0x5A).all())
+        raw = bucket[:nb].cpu().numpy().view(BITS[wl.dst_dtype])
+        covered = np.zeros(raw.size, bool)
+        for e in case.plan.bucket_entries(r):
+            t = int(e["ckpt_tensor"])
+            if t not in views:
+                views[t] = checkpoint_view(t, shapes[t], case.trainer.slices, src_bits)[0]
+            r0, c0, nr, nc = (int(e[k]) for k in ("r0", "c0", "nr", "nc"))
+            rect = cast_bits(views[t][r0:r0 + nr, c0:c0 + nc].reshape(-1), wl.src_dtype, wl.dst_dtype)
+            off = int(e["bucket_off"]) // raw.itemsize
+            assert np.array_equal(raw[off:off + nr * nc], rect), (r, t)
+            covered[off:off + nr * nc] = True
+        pad = 0x5A5A if raw.itemsize == 2 else 0x5A5A5A5A
+        assert (raw[~covered] == pad).all()          # alignment padding is never written
+        case.plan.unpack(r, bucket.data_ptr())
+        torch.cuda.synchronize()
+    assert_dst_equals(case, want)
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_fuzz_layouts(device, seed):
+    src_dt, dst_dt = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][seed % 4]
+    shapes, tl, rl = fuzz_case(9000 + seed, src_dt, dst_dt, max_dim=[40, 150, 300][seed % 3])
+    rng = np.random.default_rng(seed)
+    ck = [random_bits(rng, r * c, src_dt) for (r, c) in shapes]
+    src_host = scatter_checkpoint(tl, ck)
+    src = RankArenas(tl.tensors, device, fill_byte=0)
+    dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+    for t, h in zip(src.tensors, src_host):
+        t.copy_(from_bits(h))
+    plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices),
+                   tile_bytes=[4096, 65536][seed % 2], bucket_budget_bytes=[0, 8192][seed % 2])
+    bind(plan, src, dst)
+    want = remap_oracle(shapes, tl.tensors, tl.slices, rl.tensors, rl.slices, src_host,
+                        prefill_bits(rl, BITS[dst_dt]))
+    plan.remap()
+    torch.cuda.synchronize()
+    for k, t in enumerate(dst.tensors):
+        assert np.array_equal(to_bits(t), want.dst[k]), k
+    for a in dst.arenas.values():
+        a.fill_(CANARY)
+    for r in range(plan.num_rounds()):
+        bucket = torch.empty(plan.bucket_bytes(r) + 16, dtype=torch.uint8, device=device)
+        plan.pack(r, bucket.data_ptr())
+        plan.unpack(r, bucket.data_ptr())
+    torch.cuda.synchronize()
+    for k, t in enumerate(dst.tensors):
+        assert np.array_equal(to_bits(t), want.dst[k]), k
+
+
+def _one_tensor_plan(n, src_dt, dst_dt, device, src_off=0, dst_off=0):
+    tl, rl = Layout("t"), Layout("r")
+    tl.add_tensor("T", 0, src_dt, n + src_off)
+    rl.add_tensor("R", 0, dst_dt, n + dst_off)
+    tl.add_slice(0, src_off, n, 1, 0, 1, n, 0, 0, 1, n)
+    rl.add_slice(0, dst_off, n, 1, 0, 1, n, 0, 0, 1, n)
+    tl.freeze(); rl.freeze()
+    src = RankArenas(tl.tensors, device)
+    dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+    plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices))
+    bind(plan, src, dst)
+    return plan, src, dst
+
+
+def test_cast_all_fp32_patterns(device):
+    """Every one of the 2^32 fp32 bit patterns through the kernel's fp32 -> bf16 path, NaNs
+    included, against the oracle's integer rounding."""
+    n = 1 << 26
+    plan, src, dst = _one_tensor_plan(n, WB_F32, WB_BF16, device)
+    ar = torch.arange(n, dtype=torch.int64, device=device)
+    for chunk in range(64):
+        src.tensors[0].view(torch.int32).copy_((ar + chunk * n).to(torch.int32))   # wraps to the pattern
+        plan.remap()
+        torch.cuda.synchronize()
+        got = to_bits(dst.tensors[0])
+        pats = (np.arange(n, dtype=np.uint64) + chunk * n).astype(np.uint32)
+        want = f32_to_bf16_bits(pats)
+        assert np.array_equal(got, want), chunk
+
+
+def test_same_dtype_is_a_bit_copy(device):
+    n = 1 << 16
+    plan, src, dst = _one_tensor_plan(n, WB_BF16, WB_BF16, device, src_off=3, dst_off=5)
+    src.tensors[0].view(torch.int16)[3:].copy_(torch.arange(n, device=device).to(torch.int16))
+    plan.remap()
+    torch.cuda.synchronize()
+    assert np.array_equal(to_bits(dst.tensors[0])[5:], np.arange(n, dtype=np.uint16))
+    assert (to_bits(dst.tensors[0])[:5] == 0xCDCD).all()
+    # fp32: NaN payloads, signalling NaNs and subnormals survive
+    n = 1 << 24
+    plan, src, dst = _one_tensor_plan(n, WB_F32, WB_F32, device, src_off=1, dst_off=2)
+    g = torch.Generator(device=device); g.manual_seed(1)
+    pats = torch.randint(-(1 << 31), (1 << 31) - 1, (n,), dtype=torch.int64, device=device, generator=g).to(torch.int32)
+    src.tensors[0].view(torch.int32)[1:].copy_(pats)
+    plan.remap()
+    torch.cuda.synchronize()
+    assert torch.equal(dst.tensors[0].view(torch.int32)[2:], pats)
+
+
+def test_widening_bf16_to_fp32(device):
+    n = 1 << 16
+    plan, src, dst = _one_tensor_plan(n, WB_BF16, WB_F32, device, src_off=1)
+    src.tensors[0].view(torch.int16)[1:].copy_(torch.arange(n, device=device).to(torch.int16))
+    plan.remap()
+    torch.cuda.synchronize()
+    want = cast_bits(np.arange(n, dtype=np.uint16), WB_BF16, WB_F32)
+    assert np.array_equal(to_bits(dst.tensors[0]), want)
+
+
+@pytest.mark.parametrize("src_off,dst_off", [(0, 0), (1, 0), (0, 1), (3, 7), (5, 2), (4, 4)])
+@pytest.mark.parametrize("dts", [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32)])
+def test_unaligned_runs(device, src_off, dst_off, dts):
+    """Runs that start off a 16-byte boundary on either side, of every length around the
+    vector width, must not touch a neighbouring element."""
+    for n in list(range(1, 40)) + [255, 256, 257, 4099, 70001]:
+        plan, src, dst = _one_tensor_plan(n, dts[0], dts[1], device, src_off, dst_off)
+        rng = np.random.default_rng(n)
+        bits = random_bits(rng, n + src_off, dts[0])
+        src.tensors[0].copy_(from_bits(bits))
+        plan.remap()
+        torch.cuda.synchronize()
+        got = to_bits(dst.tensors[0])
+        want = cast_bits(bits[src_off:], dts[0], dts[1])
+        assert np.array_equal(got[dst_off:], want), n
+        assert (got[:dst_off] == (0xCDCD if dts[1] == WB_BF16 else 0xCDCDCDCD)).all()
+
+
+def test_inverse_remap_restores_the_trainer(device):
+    wl = make_workload("cfg1b")
+    tl, rl = wl.trainer.swapped_dtype(WB_BF16), wl.rollout.swapped_dtype(WB_BF16)
+    fwd = DeviceCase(wl, device, trainer=tl, rollout=rl)
+    fwd.plan.remap()
+    inv_plan = wb.Plan(wb.Layout(rl.tensors, rl.slices), wb.Layout(tl.tensors, tl.slices))
+    back = RankArenas(tl.tensors, device, fill_byte=0)      # trainer padding was loaded as zeros
+    bind(inv_plan, fwd.dst, back)
+    inv_plan.remap()
+    torch.cuda.synchronize()
+    for a, b in zip(fwd.src.tensors, back.tensors):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+def test_remap_from_host_buffers(device):
+    wl = make_workload("cfg3", "small")
+    case = DeviceCase(wl, device)
+    want = oracle_for(case)
+    host_src = [t.cpu().pin_memory() for t in case.src.tensors]
+    host_dst = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in case.dst.tensors]
+    for t in case.src.tensors:
+        t.zero_()
+    case.plan.remap_host([t.data_ptr() for t in host_src], [t.data_ptr() for t in host_dst])
+    torch.cuda.synchronize()
+    for k, t in enumerate(host_dst):
+        assert np.array_equal(to_bits(t), want.dst[k])

@@ -1,0 +1,299 @@
+"""Host logic of the library: C-ABI surface, layout validation, the planner's invariants,
+and the tile tables executed on the host against the oracle.  No GPU needed."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from helpers import ckpt_shapes, fuzz_case, random_bits, scatter_checkpoint, to_bits
+from oracle import checkpoint_view, remap_oracle
+from oracle.cast import cast_bits
+from paper_2609_25442_b200 import binding as wb
+from plan_interp import run_table
+from wb_workloads import SLICE_DTYPE, TENSOR_DTYPE, WB_BF16, WB_F32, Layout, make_workload
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SMALL = [("cfg1", "full"), ("cfg1b", "full"), ("cfg1c", "full"), ("cfg2", "small"),
+         ("cfg3", "small"), ("cfg4", "small"), ("cfg5", "small")]
+BITS = {WB_F32: np.uint32, WB_BF16: np.uint16}
+
+
+def build(tl: Layout, rl: Layout, **opts):
+    a = wb.Layout(tl.tensors, tl.slices)
+    b = wb.Layout(rl.tensors, rl.slices)
+    return wb.Plan(a, b, **opts)
+
+
+# ---- ABI surface -----------------------------------------------------------------------------
+def test_library_exports_every_declared_symbol():
+    lib = wb.load()
+    header = open(os.path.join(ROOT, "include", "wb.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(wb_[a-z_]+)\s*\(", header))
+    assert {"wb_layout_describe", "wb_plan_build", "wb_pack", "wb_unpack", "wb_remap"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(wb.EXPORTS)
+
+
+def test_struct_sizes_match_the_generators():
+    assert ctypes.sizeof(wb.wb_slice) == SLICE_DTYPE.itemsize == 88
+    assert ctypes.sizeof(wb.wb_tensor_desc) == TENSOR_DTYPE.itemsize == 16
+    for (name, _), f in zip(wb.wb_slice._fields_, SLICE_DTYPE.names):
+        assert getattr(wb.wb_slice, name).offset == SLICE_DTYPE.fields[f][1]
+    assert wb.wb_launches_per_call() == 1
+    assert "sm_100a" in wb.wb_version()
+
+
+# ---- plans reproduce the oracle when executed on the host -----------------------------------------
+def _check_plan_against_oracle(shapes, tl, rl, src, plan, src_dt, dst_dt):
+    plan.verify()
+    want = remap_oracle(shapes, tl.tensors, tl.slices, rl.tensors, rl.slices, src,
+                        [np.full(int(t["numel"]), 0xBEEF, BITS[dst_dt]) for t in rl.tensors])
+    # fused remap
+    dst = [np.full(int(t["numel"]), 0xBEEF, BITS[dst_dt]) for t in rl.tensors]
+    reads = [np.zeros(int(t["numel"]), np.int32) for t in tl.tensors]
+    writes = [np.zeros(int(t["numel"]), np.int32) for t in rl.tensors]
+    run_table(plan.tiles(wb.WB_TABLE_REMAP), src, dst, None, src_dt, dst_dt, reads, writes)
+    for k in range(len(dst)):
+        assert np.array_equal(dst[k], want.dst[k]), k
+        assert np.array_equal(writes[k] == 1, want.written[k]) and writes[k].max(initial=0) <= 1
+    assert max(int(r.max(initial=0)) for r in reads) <= 1           # no source element read twice
+    assert sum(int(r.sum()) for r in reads) == want.n_ids_consumed   # every consumed id read once
+    # pack -> bucket -> unpack, round by round
+    dst2 = [np.full(int(t["numel"]), 0xBEEF, BITS[dst_dt]) for t in rl.tensors]
+    reads2 = [np.zeros(int(t["numel"]), np.int32) for t in tl.tensors]
+    for r in range(plan.num_rounds()):
+        nb = plan.bucket_bytes(r)
+        assert nb % 16 == 0
+        bucket = np.full(nb // BITS[dst_dt]().itemsize, 0x7A7A, BITS[dst_dt])
+        bw = np.zeros(bucket.size, np.int32)
+        run_table(plan.tiles(wb.WB_TABLE_PACK, r), src, None, bucket, src_dt, dst_dt, reads2,
+                  bucket_writes=bw)
+        assert bw.max(initial=0) <= 1
+        # directory: each payload is its checkpoint rectangle, row-major, destination dtype
+        for e in plan.bucket_entries(r):
+            t = int(e["ckpt_tensor"])
+            view, held = checkpoint_view(t, shapes[t], tl.slices, src)
+            r0, c0, nr, nc = (int(e[k]) for k in ("r0", "c0", "nr", "nc"))
+            rect = cast_bits(view[r0:r0 + nr, c0:c0 + nc].reshape(-1), src_dt, dst_dt)
+            off = int(e["bucket_off"]) // bucket.itemsize
+            assert int(e["bucket_off"]) % 16 == 0
+            assert np.array_equal(bucket[off:off + nr * nc], rect)
+            assert (bw[off:off + nr * nc] == 1).all()
+        run_table(plan.tiles(wb.WB_TABLE_UNPACK, r), None, dst2, bucket, dst_dt, dst_dt)
+    for k in range(len(dst2)):
+        assert np.array_equal(dst2[k], want.dst[k]), k
+    assert max(int(r.max(initial=0)) for r in reads2) <= 1
+    return want
+
+
+@pytest.mark.parametrize("name,scale", SMALL)
+def test_plan_tables_reproduce_oracle(name, scale):
+    wl = make_workload(name, scale)
+    src = [to_bits(t) for t in wl.trainer_weights()]
+    budget = 0 if name != "cfg3" else 1 << 20          # cfg3: force several rounds
+    plan = build(wl.trainer, wl.rollout, bucket_budget_bytes=budget, tile_bytes=16384)
+    want = _check_plan_against_oracle(ckpt_shapes(wl), wl.trainer, wl.rollout, src, plan,
+                                      wl.src_dtype, wl.dst_dtype)
+    st = plan.stats()
+    assert st["src_elems_read"] == wl.ckpt_numel() == want.n_ids_consumed
+    assert st["dst_elems_written"] == want.n_written
+    if name == "cfg3":
+        assert st["n_rounds"] > 4 and st["n_fanout_slabs"] > 0
+        assert st["bucket_bytes_max"] <= 1 << 20
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_fuzz_plans(seed):
+    src_dt, dst_dt = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][seed % 4]
+    shapes, tl, rl = fuzz_case(5000 + seed, src_dt, dst_dt, max_dim=70)
+    rng = np.random.default_rng(seed)
+    ck = [random_bits(rng, r * c, src_dt) for (r, c) in shapes]
+    src = scatter_checkpoint(tl, ck)
+    plan = build(tl, rl, tile_bytes=4096, bucket_budget_bytes=[0, 4096, 16384][seed % 3], grid_ctas=7)
+    _check_plan_against_oracle(shapes, tl, rl, src, plan, src_dt, dst_dt)
+
+
+def test_inverse_plan_is_identity():
+    wl = make_workload("cfg1b")
+    tl, rl = wl.trainer.swapped_dtype(WB_BF16), wl.rollout.swapped_dtype(WB_BF16)
+    rng = np.random.default_rng(0)
+    ck = [rng.integers(0, 1 << 16, c.numel, dtype=np.uint64).astype(np.uint16) for c in wl.ckpt]
+    src = scatter_checkpoint(tl, ck, fill_bits=0x1111)
+    fwd, inv = build(tl, rl), build(rl, tl)
+    mid = [np.zeros(int(t["numel"]), np.uint16) for t in rl.tensors]
+    run_table(fwd.tiles(wb.WB_TABLE_REMAP), src, mid, None, WB_BF16, WB_BF16)
+    back = [np.full(int(t["numel"]), 0x1111, np.uint16) for t in tl.tensors]
+    run_table(inv.tiles(wb.WB_TABLE_REMAP), mid, back, None, WB_BF16, WB_BF16)
+    for a, b in zip(src, back):
+        assert np.array_equal(a, b)
+    # the inverse writes the norms to every trainer replica from one read (fan-out)
+    assert inv.stats()["n_fanout_slabs"] > 0 and inv.stats()["src_elems_read"] == wl.ckpt_numel()
+
+
+# ---- de-duplication -------------------------------------------------------------------------------
+def test_trainer_replicas_each_supply_a_distinct_slice():
+    wl = make_workload("cfg1")          # norms are replicated on both TP ranks
+    plan = build(wl.trainer, wl.rollout)
+    st = plan.stats()
+    assert st["replica_elems_skipped"] == 5 * 256          # 2 layers x 2 norms + final norm
+    egress = [plan.rank_bytes(0, r) for r in range(4)]
+    assert sum(egress) == wl.ckpt_numel() * 4 == st["src_bytes_read"]   # exactly one model copy
+    norm_tensor = wl.rollout.index("r0.final_norm")
+    srcs = {int(t["src_tensor"]) for t in plan.tiles(wb.WB_TABLE_REMAP) if int(t["dst_tensor"]) == norm_tensor}
+    ranks = {int(wl.trainer.tensors[s]["rank"]) // 2 for s in srcs}      # tp = rank // W
+    assert ranks == {0, 1}
+    lazy = build(wl.trainer, wl.rollout, flags=wb.WB_PLAN_NO_REPLICA_SPLIT)
+    srcs = {int(t["src_tensor"]) for t in lazy.tiles(wb.WB_TABLE_REMAP) if int(t["dst_tensor"]) == norm_tensor}
+    assert {int(wl.trainer.tensors[s]["rank"]) // 2 for s in srcs} == {0}
+
+
+def test_rollout_replicas_share_one_read():
+    wl = make_workload("cfg3", "small")
+    plan = build(wl.trainer, wl.rollout)
+    st = plan.stats()
+    H = wl.meta["spec"].H
+    n_norms = 2 * wl.meta["spec"].L + 1
+    assert st["src_elems_read"] == wl.ckpt_numel()
+    assert st["dst_elems_written"] == wl.ckpt_numel() + n_norms * H
+    ingress = [plan.rank_bytes(1, r) for r in range(2)]
+    assert sum(ingress) == wl.ckpt_numel() * 2                # each id enters the rollout side once
+    assert abs(ingress[0] - ingress[1]) <= 2 * H
+
+
+# ---- full-size plans: byte totals, balance, table overhead ------------------------------------------
+@pytest.mark.parametrize("name,src_bytes,dst_bytes", [
+    ("cfg2", 16_060_522_496, 16_060_522_496),
+    ("cfg3", 32_121_044_992, 16_061_054_976),
+    ("cfg4", 61_064_220_672, 61_064_220_672),
+    ("cfg5", None, None)])
+def test_full_size_plans(name, src_bytes, dst_bytes):
+    wl = make_workload(name, "full")
+    plan = build(wl.trainer, wl.rollout)
+    plan.verify()
+    st = plan.stats()
+    r, w = wl.algorithmic_bytes()
+    assert (st["src_bytes_read"], st["dst_bytes_written"]) == (r, w)
+    if src_bytes:
+        assert (r, w) == (src_bytes, dst_bytes)
+    assert st["table_bytes"] < 0.01 * (r + w)                      # descriptors << payload
+    assert st["bucket_bytes_max"] <= 4 << 30
+    assert st["n_rounds"] == plan.num_rounds() >= -(-w // (4 << 30))
+    sizes = [plan.bucket_bytes(k) for k in range(plan.num_rounds())]
+    assert max(sizes) - min(sizes) <= 0.1 * max(sizes)              # roughly equal rounds
+    assert st["remap_cta_bytes_max"] <= 1.06 * st["remap_cta_bytes_mean"]
+    assert sum(plan.rank_bytes(0, k) for k in range(8)) == r
+    assert st["build_seconds"] < 5.0
+
+
+# ---- error paths: nothing is built, a status comes back -----------------------------------------------
+def _tiny():
+    tl, rl = Layout("t"), Layout("r")
+    tl.add_tensor("T", 0, WB_F32, 16)
+    rl.add_tensor("R", 0, WB_BF16, 16)
+    return tl, rl
+
+
+def _expect(status_name, fn):
+    with pytest.raises(wb.WbError) as e:
+        fn()
+    assert e.value.name == status_name, e.value
+
+
+def test_error_slice_leaves_checkpoint_tensor():
+    tl, _ = _tiny()
+    tl.add_slice(0, 0, 4, 1, 0, 4, 4, 2, 0, 3, 4)
+    tl.freeze()
+    _expect("WB_ERR_OUT_OF_RANGE", lambda: wb.Layout(tl.tensors, tl.slices))
+
+
+def test_error_slice_leaves_local_tensor():
+    tl, _ = _tiny()
+    tl.add_slice(0, 4, 4, 1, 0, 4, 4, 0, 0, 4, 4)
+    tl.freeze()
+    _expect("WB_ERR_OUT_OF_RANGE", lambda: wb.Layout(tl.tensors, tl.slices))
+
+
+def test_error_bad_strides_and_indices():
+    tl, _ = _tiny()
+    tl.add_slice(0, 0, 2, 3, 0, 4, 4, 0, 0, 2, 2)
+    tl.freeze()
+    _expect("WB_ERR_INVALID_ARG", lambda: wb.Layout(tl.tensors, tl.slices))
+    tl2, _ = _tiny()
+    tl2.add_slice(5, 0, 4, 1, 0, 4, 4, 0, 0, 4, 4)
+    tl2.freeze()
+    _expect("WB_ERR_INVALID_ARG", lambda: wb.Layout(tl2.tensors, tl2.slices))
+    tl3, _ = _tiny()
+    tl3.add_slice(0, 0, 2, 1, 0, 4, 4, 0, 0, 4, 4)      # rows overlap: pitch 2 < 4 columns
+    tl3.freeze()
+    _expect("WB_ERR_INVALID_ARG", lambda: wb.Layout(tl3.tensors, tl3.slices))
+
+
+def test_error_dtype_and_shape_mismatch():
+    t = np.array([(0, 7, 16)], dtype=TENSOR_DTYPE)
+    _expect("WB_ERR_DTYPE", lambda: wb.Layout(t, np.zeros(0, SLICE_DTYPE)))
+    t = np.array([(0, 0, 16), (0, 1, 16)], dtype=TENSOR_DTYPE)
+    _expect("WB_ERR_DTYPE", lambda: wb.Layout(t, np.zeros(0, SLICE_DTYPE)))
+    tl, _ = _tiny()
+    tl.add_slice(0, 0, 4, 1, 0, 4, 4, 0, 0, 2, 4)
+    tl.add_slice(0, 8, 4, 1, 0, 2, 8, 0, 0, 1, 8)
+    tl.freeze()
+    _expect("WB_ERR_SHAPE_MISMATCH", lambda: wb.Layout(tl.tensors, tl.slices))
+    tl, rl = _tiny()
+    tl.add_slice(0, 0, 4, 1, 0, 4, 4, 0, 0, 4, 4)
+    rl.add_slice(0, 0, 8, 1, 0, 2, 8, 0, 0, 2, 8)
+    tl.freeze(); rl.freeze()
+    _expect("WB_ERR_SHAPE_MISMATCH", lambda: build(tl, rl))
+
+
+def test_error_uncovered_and_overlap():
+    tl, rl = _tiny()
+    tl.add_slice(0, 0, 4, 1, 0, 4, 4, 0, 0, 3, 4)           # row 3 held by nobody
+    rl.add_slice(0, 0, 4, 1, 0, 4, 4, 0, 0, 4, 4)
+    tl.freeze(); rl.freeze()
+    _expect("WB_ERR_UNCOVERED", lambda: build(tl, rl))
+    tl, rl = _tiny()
+    tl.add_slice(0, 0, 4, 1, 0, 4, 4, 0, 0, 4, 4)
+    rl.add_slice(0, 0, 4, 1, 1, 4, 4, 0, 0, 4, 4)           # checkpoint tensor 1 unknown to the trainer
+    tl.freeze(); rl.freeze()
+    _expect("WB_ERR_UNCOVERED", lambda: build(tl, rl))
+    tl, rl = _tiny()
+    tl.add_slice(0, 0, 4, 1, 0, 4, 4, 0, 0, 4, 4)
+    rl.add_slice(0, 0, 4, 1, 0, 4, 4, 0, 0, 2, 4)
+    rl.add_slice(0, 6, 4, 1, 0, 4, 4, 2, 0, 2, 4)           # lands on elements 6.. already described
+    tl.freeze(); rl.freeze()
+    _expect("WB_ERR_DST_OVERLAP", lambda: build(tl, rl))
+
+
+def test_error_bucket_too_small_and_unbound_execution():
+    wl = make_workload("cfg1")
+    _expect("WB_ERR_BUCKET_TOO_SMALL", lambda: build(wl.trainer, wl.rollout, bucket_budget_bytes=64))
+    plan = build(wl.trainer, wl.rollout)
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.remap())
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.pack(99, 16))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.bind([0] * plan.n_src, [0] * plan.n_dst))
+    lib = wb.load()
+    assert lib.wb_remap(None, None) == 1
+    assert lib.wb_plan_build(None, None, None, None) == 1
+    assert lib.wb_plan_num_rounds(None) == 0
+
+
+def test_interleaved_column_blocks_are_not_an_overlap():
+    # two column blocks of one matrix stored interleaved in one local tensor: bounding
+    # intervals overlap, elements do not
+    tl, rl = Layout("t"), Layout("r")
+    tl.add_tensor("T", 0, WB_F32, 32)
+    rl.add_tensor("R", 0, WB_F32, 32)
+    tl.add_slice(0, 0, 8, 1, 0, 4, 8, 0, 0, 4, 8)
+    rl.add_slice(0, 0, 8, 1, 0, 4, 8, 0, 0, 4, 3)
+    rl.add_slice(0, 3, 8, 1, 0, 4, 8, 0, 3, 4, 5)
+    tl.freeze(); rl.freeze()
+    plan = build(tl, rl)
+    plan.verify()
+    src = [np.arange(32, dtype=np.uint32)]
+    dst = [np.zeros(32, np.uint32)]
+    run_table(plan.tiles(wb.WB_TABLE_REMAP), src, dst, None, WB_F32, WB_F32)
+    assert np.array_equal(dst[0], src[0])
