@@ -116,12 +116,12 @@ def oracle_sample(wl, fetch_src, budget_elems=60_000_000):
     from oracle import remap_oracle
 
     picked, total = [], 0
-    for i, c in enumerate(wl.ckpt):
-        if picked and total + c.numel > budget_elems:
-            break
+    for i, c in enumerate(wl.ckpt):      # in order, skipping tensors that would overshoot
+        if total + c.numel > budget_elems:
+            continue
         picked.append(i)
         total += c.numel
-        if total >= budget_elems:
+        if total >= 0.9 * budget_elems:
             break
     pick = np.array(picked)
 
@@ -143,7 +143,7 @@ def oracle_sample(wl, fetch_src, budget_elems=60_000_000):
     es = 4 if wl.src_dtype == 0 else 2
     ed = 4 if wl.dst_dtype == 0 else 2
     moved = res.n_ids_consumed * es + res.n_written * ed
-    desc = (f"first {len(picked)} checkpoint tensors of {wl.name} in order "
+    desc = (f"the first {len(picked)} checkpoint tensors of {wl.name} that fit a {budget_elems}-element budget "
             f"({res.n_ids_consumed} elements), numpy oracle, single thread")
     return dt, moved, desc
 
