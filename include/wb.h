@@ -224,6 +224,11 @@ wb_status wb_remap(const wb_plan* plan, void* cuda_stream);
 wb_status wb_pack(const wb_plan* plan, size_t round, void* bucket, void* cuda_stream);
 wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bucket, void* cuda_stream);
 
+/* wb_plan_check: synchronises with the device and reports whether any launch on this plan
+ * recorded an error (the kernels bound every internal wait; a wait that ran out sets a
+ * sticky error word instead of hanging).  OK, NOT_BOUND, CUDA, or INTERNAL. */
+wb_status wb_plan_check(const wb_plan* plan);
+
 /* wb_remap_host: the same transfer for callers whose weights are in HOST memory:
  * copies every trainer tensor host -> its bound device region, runs wb_remap, copies every
  * rollout tensor back, all on `cuda_stream`, and returns without synchronising.

@@ -77,7 +77,7 @@ EXPORTS = [
     "wb_layout_describe", "wb_layout_free", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
-    "wb_remap_host", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_remap_host", "wb_plan_check", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -115,6 +115,7 @@ def load() -> C.CDLL:
     lib.wb_pack.argtypes = [vp, sz, vp, vp]
     lib.wb_unpack.argtypes = [vp, sz, vp, vp]
     lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
+    lib.wb_plan_check.argtypes = [vp]
     lib.wb_launches_per_call.restype = C.c_int
     lib.wb_status_str.argtypes = [C.c_int]
     lib.wb_status_str.restype = C.c_char_p
@@ -216,6 +217,9 @@ class Plan:
     def bind(self, src_ptrs: Sequence[int], dst_ptrs: Sequence[int]) -> None:
         a, b = _ptr_array(src_ptrs), _ptr_array(dst_ptrs)
         _check(_lib.wb_plan_bind(self.handle, a, len(src_ptrs), b, len(dst_ptrs)), "wb_plan_bind")
+
+    def check(self) -> None:
+        _check(_lib.wb_plan_check(self.handle), "wb_plan_check")
 
     def remap(self, stream: int = 0) -> None:
         _check(_lib.wb_remap(self.handle, stream), "wb_remap")

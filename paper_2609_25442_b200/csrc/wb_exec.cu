@@ -26,8 +26,7 @@ using namespace wbi;
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kMinBlocksPerSM = wbi::kCtasPerSM;
+constexpr int kThreads = 512;   // warp 0: producer; warps 1..15: workers
 
 // ---------------------------------------------------------------------------------------------
 // memory access helpers: streaming (evict-first) loads and stores, the data is touched once
@@ -221,100 +220,294 @@ __device__ __forceinline__ TileRegs load_tile(const DTile* p) {
   return r;
 }
 
-constexpr int kTB = 64;   // transpose block edge
+// ---------------------------------------------------------------------------------------------
+// mbarrier / bulk-copy (TMA) primitives.  Every wait is bounded: after kSpinLimit failed
+// polls the caller records an error code and leaves, so a lost signal cannot hang the GPU.
+// ---------------------------------------------------------------------------------------------
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
 
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t addr, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+      : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Wait for the phase with the given parity to complete; gives up after kWaitLimitNs.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  if (mbar_try(addr, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try(addr, parity)) return true;
+    if ((it & 255u) == 0 && global_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+constexpr int kWorkers = kThreads - 32;       // warps 1.. run the cooperative tile code
+constexpr int kDirectStages = 4;              // bulk ring of the direct (load -> store) path
+constexpr int kDirectBytes = 16384;
+constexpr int kDescSlots = 8;                 // producer -> worker tile queue
+constexpr int kTB = 64;                       // transpose block edge
+constexpr uint32_t kEndOfWork = 0xFFFFFFFFu;
+
+__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
+
+struct TileFields {
+  const char* s;
+  char* d;
+  uint32_t nr, nc, ssr, ssc, dsr, dsc, kind, n_extra, extra;
+};
+__device__ __forceinline__ TileFields decode(const TileRegs& r, uint64_t src_add, uint64_t dst_add) {
+  TileFields f;
+  f.s = reinterpret_cast<const char*>(((uint64_t)r.a.y << 32 | r.a.x) + src_add);
+  f.d = reinterpret_cast<char*>(((uint64_t)r.a.w << 32 | r.a.z) + dst_add);
+  f.nr = r.b.x; f.nc = r.b.y; f.ssr = r.b.z; f.ssc = r.b.w;
+  f.dsr = r.c.x; f.dsc = r.c.y;
+  f.kind = r.c.z & 0xFF; f.n_extra = (r.c.z >> 8) & 0xFF; f.extra = r.c.w;
+  return f;
+}
+
+// A tile the producer thread can move by itself with bulk copies: same element size, rows that
+// are long enough, and source / destination congruent modulo 16 bytes in every row.
 template <int ES, int ED>
-__global__ void __launch_bounds__(kThreads, kMinBlocksPerSM)
-wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta_begin,
-               const DDst* __restrict__ extras, uint64_t src_add, uint64_t dst_add) {
-  using E = Elem<ES, ED>;
-  __shared__ typename E::V smem[kTB][kTB + (ED == 2 ? 2 : 1)];
-  const uint32_t t = threadIdx.x;
-  uint32_t k = cta_begin[blockIdx.x];
-  const uint32_t end = cta_begin[blockIdx.x + 1];
-  if (k >= end) return;
-  TileRegs nxt = load_tile(tiles + k);
-  for (; k < end; ++k) {
-    const TileRegs cur = nxt;
-    if (k + 1 < end) nxt = load_tile(tiles + k + 1);
-    const char* s = reinterpret_cast<const char*>(((uint64_t)cur.a.y << 32 | cur.a.x) + src_add);
-    char* d = reinterpret_cast<char*>(((uint64_t)cur.a.w << 32 | cur.a.z) + dst_add);
-    const uint32_t nr = cur.b.x, nc = cur.b.y, ssr = cur.b.z, ssc = cur.b.w;
-    const uint32_t dsr = cur.c.x, dsc = cur.c.y;
-    const uint32_t kind = cur.c.z & 0xFF, n_extra = (cur.c.z >> 8) & 0xFF, extra = cur.c.w;
+__device__ __forceinline__ bool direct_ok(const TileFields& f) {
+  if (ES != ED || f.kind != KIND_ROWS || f.n_extra != 0) return false;
+  if ((((uintptr_t)f.s ^ (uintptr_t)f.d) & 15u) != 0) return false;
+  if (f.nr > 1 && (((((size_t)f.ssr - (size_t)f.dsr) * ES) & 15u) != 0 || (size_t)f.nc * ES < 1024)) return false;
+  return (size_t)f.nc * ES >= 256;
+}
 
-    if (kind == KIND_ROWS && n_extra == 0) {
-      if (nr == 1) {
-        copy_run<ES, ED>(s, d, nc, t, kThreads);
-      } else {
-        const bool aligned = (((uintptr_t)d & 15u) == 0) && ((((size_t)dsr * ED) & 15u) == 0) &&
-                             (((uintptr_t)s & (Unit<ES, ED>::SRC_ALIGN - 1)) == 0) &&
-                             ((((size_t)ssr * ES) & (Unit<ES, ED>::SRC_ALIGN - 1)) == 0);
-        if (aligned) {
-          copy_rows_aligned<ES, ED>(s, d, nr, nc, ssr, dsr, t, kThreads);
-        } else if (nc >= 128) {
-          const uint32_t lane = t & 31, warp = t >> 5;
-          for (uint32_t row = warp; row < nr; row += kThreads / 32)
-            copy_run<ES, ED>(s + (size_t)row * ssr * ES, d + (size_t)row * dsr * ED, nc, lane, 32);
-        } else {
-          const uint32_t cnt = nr * nc;
-          for (uint32_t e = t; e < cnt; e += kThreads) {
-            const uint32_t i = e / nc, j = e - i * nc;
-            E::store(d + ((size_t)i * dsr + j) * ED, E::load(s + ((size_t)i * ssr + j) * ES));
-          }
-        }
-      }
-    } else if (kind == KIND_TRANS && n_extra == 0) {
-      // dst[j*dsc + i] = src[i*ssr + j]; 64x64 blocks through shared memory
-      for (uint32_t i0 = 0; i0 < nr; i0 += kTB) {
-        for (uint32_t j0 = 0; j0 < nc; j0 += kTB) {
-          const uint32_t bi = min((uint32_t)kTB, nr - i0), bj = min((uint32_t)kTB, nc - j0);
-          // load: threads sweep j fastest (coalesced on the source)
-          for (uint32_t e = t; e < bi * kTB; e += kThreads) {
-            const uint32_t i = e / kTB, j = e % kTB;
-            if (j < bj) smem[i][j] = E::load(s + ((size_t)(i0 + i) * ssr + (j0 + j)) * ES);
-          }
-          __syncthreads();
-          // store: threads sweep i fastest (coalesced on the destination)
-          for (uint32_t e = t; e < bj * kTB; e += kThreads) {
-            const uint32_t j = e / kTB, i = e % kTB;
-            if (i < bi) E::store(d + ((size_t)(j0 + j) * dsc + (i0 + i)) * ED, smem[i][j]);
-          }
-          __syncthreads();
-        }
-      }
+// Cooperative execution of one tile by the worker warps (thread t of nth).
+template <int ES, int ED, typename SmemT>
+__device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __restrict__ extras, uint64_t dst_add,
+                                          SmemT& smem, uint32_t t) {
+  using E = Elem<ES, ED>;
+  constexpr uint32_t nth = kWorkers;
+  const char* s = f.s;
+  char* d = f.d;
+  const uint32_t nr = f.nr, nc = f.nc, ssr = f.ssr, ssc = f.ssc, dsr = f.dsr, dsc = f.dsc;
+  if (f.kind == KIND_ROWS && f.n_extra == 0) {
+    if (nr == 1) {
+      copy_run<ES, ED>(s, d, nc, t, nth);
     } else {
-      // element-wise: arbitrary strides, any number of destinations
-      const uint32_t cnt = nr * nc;
-      for (uint32_t e = t; e < cnt; e += kThreads) {
-        const uint32_t i = e / nc, j = e - i * nc;
-        const typename E::V v = E::load(s + ((size_t)i * ssr + (size_t)j * ssc) * ES);
-        E::store(d + ((size_t)i * dsr + (size_t)j * dsc) * ED, v);
-        for (uint32_t x = 0; x < n_extra; ++x) {
-          const DDst o = extras[extra + x];
-          E::store(reinterpret_cast<char*>(o.dst + dst_add) + ((size_t)i * o.sr + (size_t)j * o.sc) * ED, v);
+      const bool aligned = (((uintptr_t)d & 15u) == 0) && ((((size_t)dsr * ED) & 15u) == 0) &&
+                           (((uintptr_t)s & (Unit<ES, ED>::SRC_ALIGN - 1)) == 0) &&
+                           ((((size_t)ssr * ES) & (Unit<ES, ED>::SRC_ALIGN - 1)) == 0);
+      if (aligned) {
+        copy_rows_aligned<ES, ED>(s, d, nr, nc, ssr, dsr, t, nth);
+      } else if (nc >= 128) {
+        const uint32_t lane = t & 31, warp = t >> 5;
+        for (uint32_t row = warp; row < nr; row += nth / 32)
+          copy_run<ES, ED>(s + (size_t)row * ssr * ES, d + (size_t)row * dsr * ED, nc, lane, 32);
+      } else {
+        const uint32_t cnt = nr * nc;
+        for (uint32_t e = t; e < cnt; e += nth) {
+          const uint32_t i = e / nc, j = e - i * nc;
+          E::store(d + ((size_t)i * dsr + j) * ED, E::load(s + ((size_t)i * ssr + j) * ES));
         }
+      }
+    }
+  } else if (f.kind == KIND_TRANS && f.n_extra == 0) {
+    // dst[j*dsc + i] = src[i*ssr + j]; 64x64 blocks through shared memory
+    for (uint32_t i0 = 0; i0 < nr; i0 += kTB) {
+      for (uint32_t j0 = 0; j0 < nc; j0 += kTB) {
+        const uint32_t bi = min((uint32_t)kTB, nr - i0), bj = min((uint32_t)kTB, nc - j0);
+        for (uint32_t e = t; e < bi * kTB; e += nth) {       // j fastest: coalesced on the source
+          const uint32_t i = e / kTB, j = e % kTB;
+          if (j < bj) smem[i][j] = E::load(s + ((size_t)(i0 + i) * ssr + (j0 + j)) * ES);
+        }
+        worker_sync();
+        for (uint32_t e = t; e < bj * kTB; e += nth) {       // i fastest: coalesced on the destination
+          const uint32_t j = e / kTB, i = e % kTB;
+          if (i < bi) E::store(d + ((size_t)(j0 + j) * dsc + (i0 + i)) * ED, smem[i][j]);
+        }
+        worker_sync();
+      }
+    }
+  } else {
+    // element-wise: arbitrary strides, any number of destinations
+    const uint32_t cnt = nr * nc;
+    for (uint32_t e = t; e < cnt; e += nth) {
+      const uint32_t i = e / nc, j = e - i * nc;
+      const typename E::V v = E::load(s + ((size_t)i * ssr + (size_t)j * ssc) * ES);
+      E::store(d + ((size_t)i * dsr + (size_t)j * dsc) * ED, v);
+      for (uint32_t x = 0; x < f.n_extra; ++x) {
+        const DDst o = extras[f.extra + x];
+        E::store(reinterpret_cast<char*>(o.dst + dst_add) + ((size_t)i * o.sr + (size_t)j * o.sc) * ED, v);
       }
     }
   }
 }
 
+// Error codes written to the plan's device error word.
+enum : uint32_t { ERR_NONE = 0, ERR_WAIT_LOAD = 1, ERR_WAIT_DESC_EMPTY = 2, ERR_WAIT_DESC_FULL = 3 };
+
+// The persistent executor: one thread block per SM walks its range of the tile table.
+//   warp 0, lane 0   "producer": moves direct tiles itself through a ring of bulk (TMA) copies
+//                    global -> shared -> global, and hands every other tile to the workers
+//                    through a small queue of tile indices.
+//   warps 1..        "workers": execute queued tiles cooperatively (vector loads/stores with the
+//                    cast in registers, shared-memory transposes, element-wise fan-out).
+template <int ES, int ED>
+__global__ void __launch_bounds__(kThreads, 1)
+wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta_begin,
+               const DDst* __restrict__ extras, uint64_t src_add, uint64_t dst_add, uint32_t* __restrict__ err) {
+  using E = Elem<ES, ED>;
+  extern __shared__ __align__(128) char ring[];                       // kDirectStages x kDirectBytes
+  __shared__ typename E::V tsmem[kTB][kTB + (ED == 2 ? 2 : 1)];
+  __shared__ __align__(8) uint64_t full_bar[kDirectStages];
+  __shared__ __align__(8) uint64_t desc_full[kDescSlots], desc_empty[kDescSlots];
+  __shared__ uint32_t desc_tile[kDescSlots];
+
+  const uint32_t begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
+  if (begin >= end) return;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kDirectStages; ++i) mbar_init(&full_bar[i], 1);
+    for (int i = 0; i < kDescSlots; ++i) { mbar_init(&desc_full[i], 1); mbar_init(&desc_empty[i], kWorkers / 32); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (threadIdx.x >= 32) {
+    // ------------------------------- workers -------------------------------------------------
+    const uint32_t t = threadIdx.x - 32;
+    for (uint32_t n = 0;; ++n) {
+      const uint32_t q = n % kDescSlots;
+      uint32_t ok = 1;
+      if ((t & 31) == 0) ok = mbar_wait(&desc_full[q], (n / kDescSlots) & 1);   // one poller per warp
+      ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+      if (!ok) { if (t == 0) atomicMax(err, ERR_WAIT_DESC_FULL); return; }
+      const uint32_t k = desc_tile[q];
+      if (k == kEndOfWork) return;
+      const TileFields f = decode(load_tile(tiles + k), src_add, dst_add);
+      coop_tile<ES, ED>(f, extras, dst_add, tsmem, t);
+      __syncwarp();
+      if ((t & 31) == 0) mbar_arrive(&desc_empty[q]);
+    }
+  }
+  if (threadIdx.x != 0) return;
+
+  // --------------------------------- producer ---------------------------------------------------
+  uint32_t n_desc = 0;                  // tiles queued so far
+  uint32_t n_load = 0, n_store = 0;     // bulk loads issued / bulk stores issued (ring positions)
+  char* q_dst[kDirectStages] = {};
+  uint32_t q_bytes[kDirectStages] = {};
+  bool failed = false;
+
+  auto push_desc = [&](uint32_t k) {
+    const uint32_t q = n_desc % kDescSlots;
+    if (n_desc >= kDescSlots && !mbar_wait(&desc_empty[q], ((n_desc / kDescSlots) - 1) & 1)) {
+      atomicMax(err, ERR_WAIT_DESC_EMPTY); failed = true; return;
+    }
+    desc_tile[q] = k;
+    mbar_arrive(&desc_full[q]);         // release: the tile index is visible to whoever sees the phase
+    ++n_desc;
+  };
+  // store the oldest loaded chunk; then, one store behind, its stage is free for the next load
+  auto store_oldest = [&]() {
+    const uint32_t st = n_store % kDirectStages;
+    if (!mbar_wait(&full_bar[st], (n_store / kDirectStages) & 1)) { atomicMax(err, ERR_WAIT_LOAD); failed = true; return; }
+    fence_async_smem();
+    bulk_store(q_dst[st], ring + (size_t)st * kDirectBytes, q_bytes[st]);
+    bulk_commit();
+    ++n_store;
+  };
+  auto load_chunk = [&](const char* src, char* dst, uint32_t bytes) {
+    // ring full: retire one chunk and wait until the store before it has drained its stage
+    while (!failed && n_load - n_store >= (uint32_t)kDirectStages - 1) { store_oldest(); bulk_wait_read_1(); }
+    if (failed) return;
+    const uint32_t st = n_load % kDirectStages;
+    q_dst[st] = dst;
+    q_bytes[st] = bytes;
+    mbar_expect_tx(&full_bar[st], bytes);
+    bulk_load(ring + (size_t)st * kDirectBytes, src, bytes, &full_bar[st]);
+    ++n_load;
+  };
+
+  TileRegs nxt = load_tile(tiles + begin);
+  for (uint32_t k = begin; k < end && !failed; ++k) {
+    const TileFields f = decode(nxt, src_add, dst_add);
+    if (k + 1 < end) nxt = load_tile(tiles + k + 1);
+    if (!direct_ok<ES, ED>(f)) { push_desc(k); continue; }
+    for (uint32_t i = 0; i < f.nr && !failed; ++i) {
+      const char* s = f.s + (size_t)i * f.ssr * ES;
+      char* d = f.d + (size_t)i * f.dsr * ED;
+      size_t n = (size_t)f.nc * ES;
+      // bytes before the first / after the last 16-byte boundary: element copies
+      size_t head = (16u - ((uintptr_t)d & 15u)) & 15u;
+      if (head > n) head = n;
+      for (size_t b = 0; b < head; b += ES) Elem<ES, ED>::store(d + b, Elem<ES, ED>::load(s + b));
+      s += head; d += head; n -= head;
+      const size_t body = n & ~(size_t)15;
+      for (size_t b = body; b < n; b += ES) Elem<ES, ED>::store(d + b, Elem<ES, ED>::load(s + b));
+      for (size_t off = 0; off < body && !failed; off += kDirectBytes)
+        load_chunk(s + off, d + off, (uint32_t)min((size_t)kDirectBytes, body - off));
+    }
+  }
+  while (!failed && n_store < n_load) store_oldest();
+  if (!failed) push_desc(kEndOfWork);
+  bulk_wait_all();
+}
+
 // ---------------------------------------------------------------------------------------------
 // launch
 // ---------------------------------------------------------------------------------------------
+constexpr size_t kDynSmem = (size_t)kDirectStages * kDirectBytes;
+
+template <int ES, int ED>
+cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add, uint64_t dst_add,
+                       cudaStream_t stream) {
+  static bool configured[16] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 16 && !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(wb_exec_kernel<ES, ED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kDynSmem);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  wb_exec_kernel<ES, ED><<<dim3(plan->grid), dim3(kThreads), kDynSmem, stream>>>(
+      T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err);
+  return cudaGetLastError();
+}
+
 wb_status launch_table(const wb_plan* plan, const TileTable& T, uint64_t src_add, uint64_t dst_add,
                        uint32_t es, uint32_t ed, cudaStream_t stream) {
   if (T.tiles.empty()) return WB_OK;
-  const dim3 grid(plan->grid), block(kThreads);
-  if (es == 2 && ed == 2)
-    wb_exec_kernel<2, 2><<<grid, block, 0, stream>>>(T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add);
-  else if (es == 4 && ed == 4)
-    wb_exec_kernel<4, 4><<<grid, block, 0, stream>>>(T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add);
-  else if (es == 4 && ed == 2)
-    wb_exec_kernel<4, 2><<<grid, block, 0, stream>>>(T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add);
-  else
-    wb_exec_kernel<2, 4><<<grid, block, 0, stream>>>(T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add);
-  return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
+  cudaError_t e;
+  if (es == 2 && ed == 2) e = launch_one<2, 2>(plan, T, src_add, dst_add, stream);
+  else if (es == 4 && ed == 4) e = launch_one<4, 4>(plan, T, src_add, dst_add, stream);
+  else if (es == 4 && ed == 2) e = launch_one<4, 2>(plan, T, src_add, dst_add, stream);
+  else e = launch_one<2, 4>(plan, T, src_add, dst_add, stream);
+  return e == cudaSuccess ? WB_OK : WB_ERR_CUDA;
 }
 
 inline uint32_t esize(uint32_t dt) { return dt == WB_F32 ? 4u : 2u; }
@@ -353,7 +546,8 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
     for (TileTable* T : tabs)
       bytes += up256(T->tiles.size() * sizeof(DTile)) + up256(T->extras.size() * sizeof(DDst)) +
                up256(T->cta_begin.size() * sizeof(uint32_t));
-    bytes = up256(bytes + 256);
+    const size_t err_off = up256(bytes);
+    bytes = up256(err_off + 256);
     std::vector<char> host(bytes, 0);
     if (!plan->d_arena || plan->arena_bytes != bytes) {
       wbi::release_device_tables(plan);
@@ -362,6 +556,7 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
     }
     if (cudaGetDevice(&plan->device) != cudaSuccess) return WB_ERR_CUDA;
     char* dbase = static_cast<char*>(plan->d_arena);
+    plan->d_err = reinterpret_cast<uint32_t*>(dbase + err_off);
     size_t off = 0;
     for (size_t ti = 0; ti < tabs.size(); ++ti) {
       TileTable* T = tabs[ti];
@@ -404,6 +599,14 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
   }
   plan->bound = true;
   return WB_OK;
+}
+
+extern "C" wb_status wb_plan_check(const wb_plan* plan) {
+  if (!plan) return WB_ERR_INVALID_ARG;
+  if (!plan->bound) return WB_ERR_NOT_BOUND;
+  uint32_t e = 0;
+  if (cudaMemcpy(&e, plan->d_err, sizeof(e), cudaMemcpyDeviceToHost) != cudaSuccess) return WB_ERR_CUDA;
+  return e == 0 ? WB_OK : WB_ERR_INTERNAL;
 }
 
 extern "C" wb_status wb_remap(const wb_plan* plan, void* cuda_stream) {

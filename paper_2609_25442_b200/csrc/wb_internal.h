@@ -68,7 +68,7 @@ enum : uint32_t { KIND_ROWS = 0, KIND_TRANS = 1, KIND_ELEM = 2 };
 // Resident thread blocks per SM the executor kernel is compiled for; the planner's default
 // grid is kNumSMs * kCtasPerSM so that one launch is exactly one wave on a B200.
 constexpr uint32_t kNumSMs = 148;
-constexpr uint32_t kCtasPerSM = 3;
+constexpr uint32_t kCtasPerSM = 1;
 
 // Host form of a tile: tensor indices and element offsets (resolved to addresses at bind).
 struct HTile {
@@ -157,6 +157,7 @@ struct wb_plan {
   std::vector<const void*> src_base;
   std::vector<void*> dst_base;
   void* d_arena = nullptr;              // one device allocation holding every table
+  uint32_t* d_err = nullptr;            // sticky device error word (inside the arena)
   size_t arena_bytes = 0;
 };
 
