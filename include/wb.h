@@ -55,7 +55,8 @@ typedef enum {
   WB_ERR_OOM = 8,              /* host or device allocation failed                           */
   WB_ERR_CUDA = 9,             /* a CUDA runtime call failed                                 */
   WB_ERR_NOT_BOUND = 10,       /* execution requested before wb_plan_bind                    */
-  WB_ERR_INTERNAL = 11         /* a plan invariant does not hold (wb_plan_verify)            */
+  WB_ERR_INTERNAL = 11,        /* a plan invariant does not hold (wb_plan_verify)            */
+  WB_ERR_STATIC_LIMIT = 12     /* the plan's tile table exceeds WB_STATIC_SCRATCH_BYTES       */
 } wb_status;
 
 typedef enum { WB_F32 = 0, WB_BF16 = 1 } wb_dtype;
@@ -236,6 +237,44 @@ wb_status wb_plan_check(const wb_plan* plan);
  * tensors in table order.  Errors: INVALID_ARG, NOT_BOUND, CUDA. */
 wb_status wb_remap_host(const wb_plan* plan, const void* const* host_src, size_t n_src,
                         void* const* host_dst, size_t n_dst, void* cuda_stream);
+
+/* wb_remap_static: wb_remap for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a deployment convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a rollout engine that has
+ * already handed all free HBM to its KV-cache pool, a weight update triggered from inside a
+ * region where the allocator must not be entered, a process whose memory budget is fixed at
+ * start-up.  wb_plan_bind allocates a device arena for the tile tables, so such callers cannot
+ * use it.  Here the tables and the error word live in a fixed array of
+ * WB_STATIC_SCRATCH_BYTES (4 MiB) that is part of the library image: every GPU that loads the
+ * library holds those 4 MiB until the process exits, and nothing is ever allocated or freed.
+ * The function calls no cudaMalloc / cudaFree / allocating routine, and the plan need not be
+ * bound.
+ *
+ * plan      built by wb_plan_build (host object; its remap table is used)
+ * src_base  host array of n_src DEVICE addresses of the trainer tensors, in table order
+ * dst_base  host array of n_dst DEVICE addresses of the rollout tensors; the caller still owns
+ *           and passes all inputs and outputs
+ * flags     0, or WB_STATIC_SYNC_CHECK: synchronise the stream after the launch and return
+ *           WB_ERR_INTERNAL if a bounded wait inside the kernel ran out
+ *
+ * Limits and rules:
+ *   - A plan whose remap table (48 B per tile + 16 B per fan-out record + 4 B per thread block
+ *     + 512 B) does not fit in 4 MiB -- about 87,000 tiles, e.g. 40 GB moved at the default
+ *     512 KiB tile size -- is refused with WB_ERR_STATIC_LIMIT and nothing is launched; build
+ *     the plan with a larger tile_bytes, or use wb_plan_bind + wb_remap.
+ *   - The first call on each device resolves the array's device address and configures the
+ *     kernels (no allocation).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents: each
+ *     call rewrites the table it needs and zeroes the error word, in stream order.  Two calls
+ *     whose GPU work can overlap (different streams without an ordering between them) race on
+ *     the array; order them on one stream or with events.  Host-side preparation is serialised
+ *     internally.
+ * Errors: INVALID_ARG, STATIC_LIMIT, CUDA, INTERNAL (only with WB_STATIC_SYNC_CHECK). */
+#define WB_STATIC_SCRATCH_BYTES (4u << 20)
+#define WB_STATIC_SYNC_CHECK 1u
+wb_status wb_remap_static(const wb_plan* plan, const void* const* src_base, size_t n_src,
+                          void* const* dst_base, size_t n_dst, uint32_t flags, void* cuda_stream);
 
 /* Number of kernels wb_remap / wb_pack / wb_unpack launch per call (always 1). */
 int wb_launches_per_call(void);

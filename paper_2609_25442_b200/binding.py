@@ -24,7 +24,7 @@ STATUS_NAMES = {
     0: "WB_OK", 1: "WB_ERR_INVALID_ARG", 2: "WB_ERR_DTYPE", 3: "WB_ERR_SHAPE_MISMATCH",
     4: "WB_ERR_OUT_OF_RANGE", 5: "WB_ERR_DST_OVERLAP", 6: "WB_ERR_UNCOVERED",
     7: "WB_ERR_BUCKET_TOO_SMALL", 8: "WB_ERR_OOM", 9: "WB_ERR_CUDA", 10: "WB_ERR_NOT_BOUND",
-    11: "WB_ERR_INTERNAL",
+    11: "WB_ERR_INTERNAL", 12: "WB_ERR_STATIC_LIMIT",
 }
 
 
@@ -77,7 +77,7 @@ EXPORTS = [
     "wb_layout_describe", "wb_layout_free", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
-    "wb_remap_host", "wb_plan_check", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -115,6 +115,7 @@ def load() -> C.CDLL:
     lib.wb_pack.argtypes = [vp, sz, vp, vp]
     lib.wb_unpack.argtypes = [vp, sz, vp, vp]
     lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
+    lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
     lib.wb_launches_per_call.restype = C.c_int
     lib.wb_status_str.argtypes = [C.c_int]
@@ -234,6 +235,22 @@ class Plan:
         a, b = _ptr_array(host_src_ptrs), _ptr_array(host_dst_ptrs)
         _check(_lib.wb_remap_host(self.handle, a, len(host_src_ptrs), b, len(host_dst_ptrs), stream),
                "wb_remap_host")
+
+
+WB_STATIC_SCRATCH_BYTES = 4 << 20
+WB_STATIC_SYNC_CHECK = 1
+
+
+def wb_remap_static(plan: Plan, src_ptrs: Sequence[int], dst_ptrs: Sequence[int], flags: int = 0,
+                    stream: int = 0) -> None:
+    """wb_remap without any device allocation: the plan is not bound; its tile table goes into
+    the library's fixed 4 MiB device array (see include/wb.h for who needs this and the rules:
+    first call per device outside stream capture, overlapping calls race, larger plans are
+    refused with WB_ERR_STATIC_LIMIT)."""
+    load()
+    a, b = _ptr_array(src_ptrs), _ptr_array(dst_ptrs)
+    _check(_lib.wb_remap_static(plan.handle, a, len(src_ptrs), b, len(dst_ptrs), flags, stream),
+           "wb_remap_static")
 
 
 def wb_plan_build(trainer: Layout, rollout: Layout, **opts) -> Plan:

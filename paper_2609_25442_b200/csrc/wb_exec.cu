@@ -15,6 +15,7 @@
 //   ELEM   anything else (strided vectors, fan-out): one element per thread.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 #include <cstring>
 #include <new>
@@ -648,6 +649,116 @@ extern "C" wb_status wb_remap_host(const wb_plan* plan, const void* const* host_
     if (!host_dst[i]) return WB_ERR_INVALID_ARG;
     if (cudaMemcpyAsync(host_dst[i], plan->dst_base[i], plan->dst.tensors[i].numel * ed,
                         cudaMemcpyDeviceToHost, stream) != cudaSuccess) return WB_ERR_CUDA;
+  }
+  return WB_OK;
+}
+
+
+// =================================================================================================
+// wb_remap_static: the fused remap for callers that must not allocate device memory.
+//
+// The executor kernel needs scratch beyond the caller's tensors: the tile table it walks and an
+// error word.  wb_plan_bind puts those in a cudaMalloc'd arena.  This entry point instead keeps
+// them in the fixed array below, which every GPU that loads the library holds until the process
+// exits.  It never calls cudaMalloc, cudaFree or any allocating routine.
+// =================================================================================================
+static __device__ __align__(256) unsigned char g_static_scratch[WB_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxStaticDevices = 64;
+void* g_static_ptr[kMaxStaticDevices] = {};     // device address of g_static_scratch, per device
+unsigned char g_static_stage[WB_STATIC_SCRATCH_BYTES];   // host image of the scratch, built per call
+struct SpinLock {
+  std::atomic_flag f = ATOMIC_FLAG_INIT;
+  void lock() { while (f.test_and_set(std::memory_order_acquire)) {} }
+  void unlock() { f.clear(std::memory_order_release); }
+} g_static_lock;
+
+// Set-up, once per device, with that device current: resolve the array's device address (in host
+// code the array's name is only a stand-in, not a device address) and let the kernels use their
+// dynamic shared memory.
+template <int ES, int ED>
+cudaError_t static_setup_kernel() {
+  return cudaFuncSetAttribute(wb_exec_kernel<ES, ED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+}
+wb_status static_setup(int dev) {
+  if (g_static_ptr[dev]) return WB_OK;
+  void* ptr = nullptr;
+  if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return WB_ERR_CUDA;
+  if (static_setup_kernel<2, 2>() != cudaSuccess || static_setup_kernel<4, 4>() != cudaSuccess ||
+      static_setup_kernel<4, 2>() != cudaSuccess || static_setup_kernel<2, 4>() != cudaSuccess)
+    return WB_ERR_CUDA;
+  g_static_ptr[dev] = ptr;
+  return WB_OK;
+}
+}  // namespace
+
+extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src_base, size_t n_src,
+                                     void* const* dst_base, size_t n_dst, uint32_t flags, void* cuda_stream) {
+  if (!plan || !src_base || !dst_base || (flags & ~WB_STATIC_SYNC_CHECK)) return WB_ERR_INVALID_ARG;
+  if (n_src != plan->src.tensors.size() || n_dst != plan->dst.tensors.size()) return WB_ERR_INVALID_ARG;
+  const uint32_t es = esize(plan->src.dtype), ed = esize(plan->dst.dtype);
+  for (size_t i = 0; i < n_src; ++i)
+    if (!src_base[i] || ((uintptr_t)src_base[i] % es)) return WB_ERR_INVALID_ARG;
+  for (size_t i = 0; i < n_dst; ++i)
+    if (!dst_base[i] || ((uintptr_t)dst_base[i] % ed)) return WB_ERR_INVALID_ARG;
+  const TileTable& T = plan->remap;
+  if (T.tiles.empty()) return WB_OK;
+  // layout of the scratch: [error word | tiles | fan-out records | per-block tile ranges]
+  const size_t off_tiles = 256;
+  const size_t off_extras = off_tiles + up256(T.tiles.size() * sizeof(DTile));
+  const size_t off_begin = off_extras + up256(T.extras.size() * sizeof(DDst));
+  const size_t total = off_begin + up256(T.cta_begin.size() * sizeof(uint32_t));
+  if (total > (size_t)WB_STATIC_SCRATCH_BYTES) return WB_ERR_STATIC_LIMIT;
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxStaticDevices) return WB_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  g_static_lock.lock();
+  wb_status st = static_setup(dev);
+  if (st != WB_OK) { g_static_lock.unlock(); return st; }
+  char* dbase = static_cast<char*>(g_static_ptr[dev]);
+  // the array keeps the previous call's contents: rebuild everything this launch reads, and
+  // zero the error word
+  std::memset(g_static_stage, 0, off_tiles);
+  DTile* ht = reinterpret_cast<DTile*>(g_static_stage + off_tiles);
+  for (size_t k = 0; k < T.tiles.size(); ++k) {
+    const HTile& h = T.tiles[k];
+    DTile dt{};
+    dt.src = (uint64_t)(uintptr_t)src_base[h.src_tensor] + h.src_off * es;
+    dt.dst = (uint64_t)(uintptr_t)dst_base[h.dst_tensor] + h.dst_off * ed;
+    dt.nr = h.nr; dt.nc = h.nc; dt.ssr = h.ssr; dt.ssc = h.ssc; dt.dsr = h.dsr; dt.dsc = h.dsc;
+    dt.kind_extra = h.kind | (h.n_extra << 8);
+    dt.extra = h.extra;
+    ht[k] = dt;
+  }
+  DDst* hx = reinterpret_cast<DDst*>(g_static_stage + off_extras);
+  for (size_t k = 0; k < T.extras.size(); ++k) {
+    const HDst& h = T.extras[k];
+    hx[k] = DDst{(uint64_t)(uintptr_t)dst_base[h.tensor] + h.off * ed, h.sr, h.sc};
+  }
+  std::memcpy(g_static_stage + off_begin, T.cta_begin.data(), T.cta_begin.size() * sizeof(uint32_t));
+  // pageable source: the runtime has taken its copy of the image when this returns, so the host
+  // image can be reused by the next call
+  cudaError_t e = cudaMemcpyAsync(dbase, g_static_stage, total, cudaMemcpyHostToDevice, stream);
+  g_static_lock.unlock();
+  if (e != cudaSuccess) return WB_ERR_CUDA;
+
+  const DTile* d_tiles = reinterpret_cast<const DTile*>(dbase + off_tiles);
+  const DDst* d_extras = reinterpret_cast<const DDst*>(dbase + off_extras);
+  const uint32_t* d_begin = reinterpret_cast<const uint32_t*>(dbase + off_begin);
+  uint32_t* d_err = reinterpret_cast<uint32_t*>(dbase);
+  const dim3 grid(plan->grid), block(kThreads);
+  if (es == 2 && ed == 2) wb_exec_kernel<2, 2><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  else if (es == 4 && ed == 4) wb_exec_kernel<4, 4><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  else if (es == 4 && ed == 2) wb_exec_kernel<4, 2><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  else wb_exec_kernel<2, 4><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
+  if (flags & WB_STATIC_SYNC_CHECK) {
+    uint32_t err = 0;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaMemcpy(&err, d_err, sizeof(err), cudaMemcpyDeviceToHost) != cudaSuccess) return WB_ERR_CUDA;
+    if (err) return WB_ERR_INTERNAL;
   }
   return WB_OK;
 }
