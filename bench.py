@@ -260,11 +260,13 @@ def main():
         sampler.start()
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     launches = 0
+    torch.cuda.nvtx.range_push("timed")
     evs[0].record()
     for k in range(args.steps):
         launches += step()
         evs[k + 1].record()
     barrier()
+    torch.cuda.nvtx.range_pop()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = evs[0].elapsed_time(evs[-1])
     per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]

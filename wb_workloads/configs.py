@@ -572,23 +572,29 @@ _TINY = ModelSpec(L=2, H=256, nq=4, nkv=2, hd=64, F=688, V=1024)
 _SHAPES = {
     # config: {scale: spec}
     "cfg2": {"full": ModelSpec(32, 4096, 32, 8, 128, 14336, 128256),
+             "large": ModelSpec(4, 4096, 32, 8, 128, 14336, 16032),      # ~2 GB per side
              "medium": ModelSpec(2, 1024, 16, 4, 64, 3576, 8200),
              "small": ModelSpec(2, 256, 8, 2, 32, 696, 1000)},
     "cfg3": {"full": ModelSpec(32, 4096, 32, 8, 128, 14336, 128256),
+             "large": ModelSpec(4, 4096, 32, 8, 128, 14336, 16032),
              "medium": ModelSpec(4, 1024, 16, 8, 64, 3584, 8192),
              "small": ModelSpec(4, 256, 8, 4, 32, 704, 1024)},
     "cfg4": {"full": ModelSpec(48, 2048, 32, 4, 128, 0, 151936, E=128, Fe=768),
+             "large": ModelSpec(2, 2048, 32, 4, 128, 0, 16032, E=128, Fe=768),
              "medium": ModelSpec(2, 512, 8, 2, 64, 0, 8200, E=32, Fe=192),
              "small": ModelSpec(2, 128, 8, 2, 32, 0, 1000, E=16, Fe=48)},
 }
 _STRESS = {"full": (4000, 16, 512.0, 1 << 26),
+           "large": (500, 16, 512.0, 1 << 26),
            "medium": (600, 8, 256.0, 1 << 22),
            "small": (300, 4, 64.0, 1 << 20)}
 
 
 def make_workload(name: str, scale: str = "full") -> Workload:
-    """Build a named configuration.  `scale` is 'full' (the benchmark shape), or a
-    shrunken 'medium' / 'small' copy of the same layout family for parity tests
+    """Build a named configuration.  `scale` is 'full' (the benchmark shape), 'large' (the
+    same shapes with fewer layers / tensors, a few GB: larger than L2 but small enough for a
+    profiler capture), or a shrunken 'medium' / 'small' copy of the same layout family for
+    parity tests
     (cfg1, cfg1b and cfg1c are already tiny and ignore it)."""
     if name in ("cfg1", "cfg1b", "cfg1c"):
         s = _TINY
