@@ -27,7 +27,10 @@ using namespace wbi;
 
 namespace {
 
-constexpr int kThreads = 512;   // warp 0: producer; warps 1..15: workers
+#ifndef WB_THREADS
+#define WB_THREADS 512
+#endif
+constexpr int kThreads = WB_THREADS;   // warp 0: producer; the other warps: workers
 
 // ---------------------------------------------------------------------------------------------
 // memory access helpers: streaming (evict-first) loads and stores, the data is touched once
@@ -125,7 +128,7 @@ __device__ __forceinline__ uint4 gather_unit(const char* s) {
   }
 }
 
-template <int ES, int ED> struct Unroll { static constexpr int U = (ES == 4 && ED == 2) ? 4 : 8; };
+template <int ES, int ED> struct Unroll { static constexpr int U = (ES == 4 && ED == 2) ? 2 : 4; };
 
 // Copy one run of n contiguous elements with `nth` cooperating threads (this thread is `t`).
 template <int ES, int ED>
@@ -242,6 +245,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// One poll of the barrier.  (Giving try_wait an explicit suspend-time hint was measured to wake
+// waiting warps late and cost 30 % of the staged paths' bandwidth, so the default is used.)
 __device__ __forceinline__ bool mbar_try(uint32_t addr, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -272,14 +277,58 @@ __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-constexpr int kWorkers = kThreads - 32;       // warps 1.. run the cooperative tile code
-constexpr int kDirectStages = 4;              // bulk ring of the direct (load -> store) path
-constexpr int kDirectBytes = 16384;
-constexpr int kDescSlots = 8;                 // producer -> worker tile queue
-constexpr int kTB = 64;                       // transpose block edge
-constexpr uint32_t kEndOfWork = 0xFFFFFFFFu;
+constexpr int kWorkers = kThreads - 32;       // warps 1.. convert staged chunks and run queued tiles
+// Shared-memory rings (tuned on B200; the direct ring is very sensitive: 3 x 32 KiB moves 5 % more
+// than 4 x 16 KiB).  Kernels whose element sizes differ never use the direct ring and give all of
+// it to the worker ring.
+#ifndef WB_DIRECT_STAGES
+#define WB_DIRECT_STAGES 3
+#endif
+#ifndef WB_DIRECT_BYTES
+#define WB_DIRECT_BYTES 32768
+#endif
+#ifndef WB_SLOTS_SAME
+#define WB_SLOTS_SAME 3
+#endif
+#ifndef WB_SLOT_BYTES_SAME
+#define WB_SLOT_BYTES_SAME 32768
+#endif
+#ifndef WB_SLOTS_CAST
+#define WB_SLOTS_CAST 4
+#endif
+#ifndef WB_SLOT_BYTES_CAST
+#define WB_SLOT_BYTES_CAST 49152
+#endif
+constexpr int kDirectStages = WB_DIRECT_STAGES;   // bulk ring of the direct (load -> store) path
+constexpr int kDirectBytes = WB_DIRECT_BYTES;
+constexpr int kMaxSlots = WB_SLOTS_SAME > WB_SLOTS_CAST ? WB_SLOTS_SAME : WB_SLOTS_CAST;
+template <int ES, int ED> struct Rings {      // worker ring: staged chunks and queued tiles
+  static constexpr int kSlots = ES == ED ? WB_SLOTS_SAME : WB_SLOTS_CAST;
+  static constexpr int kSlotBytes = ES == ED ? WB_SLOT_BYTES_SAME : WB_SLOT_BYTES_CAST;
+  static constexpr size_t kDirect = ES == ED ? (size_t)kDirectStages * kDirectBytes : 0;
+  static constexpr size_t kDyn = kDirect + (size_t)kSlots * kSlotBytes;
+};
+constexpr int kTB = 64;                       // transpose block edge of the fallback path
+constexpr int kTransRowBytes = 256;           // staged transpose: source bytes per row segment
+constexpr int kTransSeg = 32;                 // staged transpose: rows per thread task
+
+enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_TRANS = 3 };
+
+// What the producer tells the workers about one ring slot.
+struct ChunkDesc {
+  uint32_t mode;
+  uint32_t tile;      // MODE_COOP: index of the tile to run
+  uint32_t nr, nc;    // staged chunk: rows in the stage, elements per row
+  uint32_t pitch;     // bytes between rows in the stage
+  uint32_t pad;
+  uint64_t src;       // global address of the chunk's first source element (alignment arithmetic only)
+  uint64_t dst;       // global address of the chunk's first destination element
+  uint64_t sps;       // source row pitch in bytes
+  uint64_t dps;       // destination pitch in bytes: between rows (ROWS) or between columns (TRANS)
+};
 
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
+__device__ __forceinline__ uint32_t roundup16(uint32_t x) { return (x + 15u) & ~15u; }
 
 struct TileFields {
   const char* s;
@@ -304,6 +353,131 @@ __device__ __forceinline__ bool direct_ok(const TileFields& f) {
   if ((((uintptr_t)f.s ^ (uintptr_t)f.d) & 15u) != 0) return false;
   if (f.nr > 1 && (((((size_t)f.ssr - (size_t)f.dsr) * ES) & 15u) != 0 || (size_t)f.nc * ES < 1024)) return false;
   return (size_t)f.nc * ES >= 256;
+}
+
+// 16 bytes starting `s` bytes into the 32-byte concatenation of v0 and v1 (s a multiple of 2).
+__device__ __forceinline__ uint4 shift16(uint4 v0, uint4 v1, uint32_t s) {
+  const uint32_t sb = (s & 3u) * 8u;
+  uint32_t w0, w1, w2, w3, w4;
+  switch (s >> 2) {
+    case 0: w0 = v0.x; w1 = v0.y; w2 = v0.z; w3 = v0.w; w4 = v1.x; break;
+    case 1: w0 = v0.y; w1 = v0.z; w2 = v0.w; w3 = v1.x; w4 = v1.y; break;
+    case 2: w0 = v0.z; w1 = v0.w; w2 = v1.x; w3 = v1.y; w4 = v1.z; break;
+    default: w0 = v0.w; w1 = v1.x; w2 = v1.y; w3 = v1.z; w4 = v1.w; break;
+  }
+  return make_uint4(__funnelshift_r(w0, w1, sb), __funnelshift_r(w1, w2, sb),
+                    __funnelshift_r(w2, w3, sb), __funnelshift_r(w3, w4, sb));
+}
+
+// One full destination vector (NV elements) from a staged row: `row` is the 16-byte aligned
+// shared-memory base of the row, `o` the byte offset of the first source element in it.
+template <int ES, int ED>
+__device__ __forceinline__ uint4 staged_unit(const char* row, uint32_t o) {
+  const uint4* q = reinterpret_cast<const uint4*>(row + (o & ~15u));
+  const uint32_t s = o & 15u;
+  if constexpr (ES == ED) {
+    const uint4 v0 = q[0];
+    if (s == 0) return v0;
+    return shift16(v0, q[1], s);
+  } else if constexpr (ES == 4) {   // 32 source bytes -> 16 destination bytes
+    uint4 a = q[0], b = q[1];
+    if (s != 0) {
+      const uint4 c = q[2];
+      a = shift16(a, b, s);
+      b = shift16(b, c, s);
+    }
+    return make_uint4(f32x2_to_bf16x2(a.x, a.y), f32x2_to_bf16x2(a.z, a.w),
+                      f32x2_to_bf16x2(b.x, b.y), f32x2_to_bf16x2(b.z, b.w));
+  } else {                          // 8 source bytes -> 16 destination bytes
+    uint4 a = q[0];
+    if (s != 0) a = shift16(a, (s > 8) ? q[1] : a, s);
+    return make_uint4(a.x << 16, a.x & 0xFFFF0000u, a.y << 16, a.y & 0xFFFF0000u);
+  }
+}
+
+// Workers: rows staged in shared memory -> destination rows.  Every row is cut into 16-byte
+// aligned destination slots; full slots are one vector store, ragged first/last slots are
+// element stores.  A group of G lanes (G = 32, 16 or 8 by row length) takes G consecutive slots
+// of one row; groups are independent (no barrier).  `t` is the rotated worker thread index.
+template <int ES, int ED>
+__device__ __forceinline__ void staged_rows(const ChunkDesc& d, const char* stage, uint32_t t) {
+  using E = Elem<ES, ED>;
+  constexpr uint32_t NV = 16 / ED;
+  const uint32_t n = d.nc;
+  const uint32_t smax = (n + 2 * NV - 2) / NV;     // slots a row can touch
+  const uint32_t gs = smax > 16 ? 5u : (smax > 8 ? 4u : 3u);
+  const uint32_t G = 1u << gs;
+  const uint32_t nb = (smax + G - 1) >> gs;        // slot blocks per row
+  const uint32_t tasks = d.nr * nb;
+  const uint32_t lead0 = (uint32_t)d.src & 15u, dlead = (uint32_t)d.sps & 15u;
+  const uint32_t lig = t & (G - 1);
+  for (uint32_t task = t >> gs; task < tasks; task += (uint32_t)kWorkers >> gs) {
+    const uint32_t r = task / nb, k = (task - r * nb) * G + lig;
+    const uint64_t D = d.dst + (uint64_t)r * d.dps;
+    const uint32_t a = (uint32_t)(D & 15u) / ED;   // elements of slot 0 that precede the row
+    const int32_t e0 = (int32_t)(k * NV) - (int32_t)a;
+    if (e0 >= (int32_t)n) continue;
+    const char* row = stage + r * d.pitch;
+    const uint32_t lead = (lead0 + r * dlead) & 15u;
+    if (e0 >= 0 && (uint32_t)e0 + NV <= n) {
+      st16(reinterpret_cast<char*>((D & ~(uint64_t)15) + 16u * k), staged_unit<ES, ED>(row, lead + (uint32_t)e0 * ES));
+    } else {
+      const uint32_t lo = e0 < 0 ? 0u : (uint32_t)e0;
+      const uint32_t hi = min(n, (uint32_t)(e0 + (int32_t)NV));
+      for (uint32_t e = lo; e < hi; ++e)
+        E::store(reinterpret_cast<char*>(D) + (size_t)e * ED, E::load(row + lead + e * ES));
+    }
+  }
+}
+
+// Workers: a staged block of source rows -> destination columns (dst[j*dps + i] = src[i][j]).
+// A thread task is one destination run: column j, kTransSeg consecutive rows; it peels to a
+// 16-byte boundary, writes vectors, then the tail.  Consecutive lanes take consecutive columns,
+// so shared-memory reads of a warp fall in consecutive words.
+template <int ES, int ED>
+__device__ __forceinline__ void staged_trans(const ChunkDesc& d, const char* stage, uint32_t t) {
+  using E = Elem<ES, ED>;
+  constexpr uint32_t NV = 16 / ED;
+  const uint32_t ni = d.nr, nj = d.nc;
+  const uint32_t segs = (ni + kTransSeg - 1) / kTransSeg;
+  const uint32_t total = segs * nj;
+  const uint32_t lead0 = (uint32_t)d.src & 15u, dlead = (uint32_t)d.sps & 15u, pitch = d.pitch;
+  for (uint32_t idx = t; idx < total; idx += kWorkers) {
+    const uint32_t sg = idx / nj, j = idx - sg * nj;
+    const uint32_t i0 = sg * kTransSeg, len = min((uint32_t)kTransSeg, ni - i0);
+    char* out = reinterpret_cast<char*>(d.dst + (uint64_t)j * d.dps) + (size_t)i0 * ED;
+    // element i of the column lives at stage + i*pitch + ((src + i*sps) & 15) + j*ES; walk it
+    const char* p = stage + i0 * pitch + j * ES;
+    uint32_t lead = (lead0 + i0 * dlead) & 15u;
+    auto next = [&]() -> typename E::V {
+      const typename E::V v = E::load(p + lead);
+      p += pitch;
+      lead = (lead + dlead) & 15u;
+      return v;
+    };
+    uint32_t head = (uint32_t)((16u - ((uintptr_t)out & 15u)) & 15u) / ED;
+    if (head > len) head = len;
+    for (uint32_t e = 0; e < head; ++e) E::store(out + e * ED, next());
+    const uint32_t nvec = (len - head) / NV;
+    char* o = out + head * ED;
+    for (uint32_t v = 0; v < nvec; ++v, o += 16) {
+      uint4 x;
+      if constexpr (ED == 2) {
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t lo = next(), hi = next();
+          w[q] = lo | (hi << 16);
+        }
+        x = make_uint4(w[0], w[1], w[2], w[3]);
+      } else {
+        const uint32_t w0 = next(), w1 = next(), w2 = next(), w3 = next();
+        x = make_uint4(w0, w1, w2, w3);
+      }
+      st16(o, x);
+    }
+    for (uint32_t e = head + nvec * NV; e < len; ++e) E::store(out + e * ED, next());
+  }
 }
 
 // Cooperative execution of one tile by the worker warps (thread t of nth).
@@ -369,30 +543,38 @@ __device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __res
 }
 
 // Error codes written to the plan's device error word.
-enum : uint32_t { ERR_NONE = 0, ERR_WAIT_LOAD = 1, ERR_WAIT_DESC_EMPTY = 2, ERR_WAIT_DESC_FULL = 3 };
+enum : uint32_t { ERR_NONE = 0, ERR_WAIT_LOAD = 1, ERR_WAIT_SLOT_EMPTY = 2, ERR_WAIT_SLOT_FULL = 3 };
 
 // The persistent executor: one thread block per SM walks its range of the tile table.
-//   warp 0, lane 0   "producer": moves direct tiles itself through a ring of bulk (TMA) copies
-//                    global -> shared -> global, and hands every other tile to the workers
-//                    through a small queue of tile indices.
-//   warps 1..        "workers": execute queued tiles cooperatively (vector loads/stores with the
-//                    cast in registers, shared-memory transposes, element-wise fan-out).
+//   warp 0   "producer".  Lane 0 moves direct tiles by itself through a ring of bulk (TMA) copies
+//            global -> shared -> global.  For every other tile the warp feeds the worker ring:
+//            either the tile's rows are staged into a ring slot with bulk loads (one per row, the
+//            16-byte aligned superset of the row), or the tile index is queued as is.
+//   warps 1.. "workers".  Take ring slots in order: convert staged rows (cast in registers,
+//            realignment by funnel shifts, 16-byte vector stores), transpose staged blocks, or
+//            run a queued tile cooperatively (element-wise fan-out and other rare shapes).
 template <int ES, int ED>
 __global__ void __launch_bounds__(kThreads, 1)
 wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta_begin,
                const DDst* __restrict__ extras, uint64_t src_add, uint64_t dst_add, uint32_t* __restrict__ err) {
   using E = Elem<ES, ED>;
-  extern __shared__ __align__(128) char ring[];                       // kDirectStages x kDirectBytes
+  extern __shared__ __align__(128) char dyn_smem[];
+  constexpr int kSlots = Rings<ES, ED>::kSlots;
+  constexpr int kSlotBytes = Rings<ES, ED>::kSlotBytes;
+  char* const ring = dyn_smem;                                         // kDirectStages x kDirectBytes
+  char* const wring = dyn_smem + Rings<ES, ED>::kDirect;               // kSlots x kSlotBytes
   __shared__ typename E::V tsmem[kTB][kTB + (ED == 2 ? 2 : 1)];
-  __shared__ __align__(8) uint64_t full_bar[kDirectStages];
-  __shared__ __align__(8) uint64_t desc_full[kDescSlots], desc_empty[kDescSlots];
-  __shared__ uint32_t desc_tile[kDescSlots];
+  __shared__ __align__(8) uint64_t direct_full[kDirectStages];
+  __shared__ __align__(8) uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots];
+  __shared__ __align__(16) ChunkDesc desc[kMaxSlots];
+  __shared__ char* q_dst[kDirectStages];        // direct ring: where each loaded stage goes
+  __shared__ uint32_t q_bytes[kDirectStages];
 
   const uint32_t begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
   if (begin >= end) return;
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kDirectStages; ++i) mbar_init(&full_bar[i], 1);
-    for (int i = 0; i < kDescSlots; ++i) { mbar_init(&desc_full[i], 1); mbar_init(&desc_empty[i], kWorkers / 32); }
+    for (int i = 0; i < kDirectStages; ++i) mbar_init(&direct_full[i], 1);
+    for (int i = 0; i < kSlots; ++i) { mbar_init(&slot_full[i], 1); mbar_init(&slot_empty[i], kWorkers / 32); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -401,55 +583,96 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     // ------------------------------- workers -------------------------------------------------
     const uint32_t t = threadIdx.x - 32;
     for (uint32_t n = 0;; ++n) {
-      const uint32_t q = n % kDescSlots;
+      const uint32_t slot = n % kSlots;
       uint32_t ok = 1;
-      if ((t & 31) == 0) ok = mbar_wait(&desc_full[q], (n / kDescSlots) & 1);   // one poller per warp
+      if ((t & 31) == 0) ok = mbar_wait(&slot_full[slot], (n / kSlots) & 1);   // one poller per warp
       ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-      if (!ok) { if (t == 0) atomicMax(err, ERR_WAIT_DESC_FULL); return; }
-      const uint32_t k = desc_tile[q];
-      if (k == kEndOfWork) return;
-      const TileFields f = decode(load_tile(tiles + k), src_add, dst_add);
-      coop_tile<ES, ED>(f, extras, dst_add, tsmem, t);
+      if (!ok) { if (t == 0) atomicMax(err, ERR_WAIT_SLOT_FULL); return; }
+      const ChunkDesc d = desc[slot];
+      if (d.mode == MODE_END) return;
+      const char* stage = wring + (size_t)slot * kSlotBytes;
+      // small chunks have fewer tasks than workers: rotate which warps take them
+      uint32_t tr = t + (n * 256u) % kWorkers;
+      if (tr >= (uint32_t)kWorkers) tr -= kWorkers;
+      if (d.mode == MODE_ROWS) {
+        staged_rows<ES, ED>(d, stage, tr);
+      } else if (d.mode == MODE_TRANS) {
+        staged_trans<ES, ED>(d, stage, tr);
+      } else {
+        const TileFields f = decode(load_tile(tiles + d.tile), src_add, dst_add);
+        coop_tile<ES, ED>(f, extras, dst_add, tsmem, t);
+      }
       __syncwarp();
-      if ((t & 31) == 0) mbar_arrive(&desc_empty[q]);
+      if ((t & 31) == 0) mbar_arrive(&slot_empty[slot]);
     }
   }
-  if (threadIdx.x != 0) return;
 
-  // --------------------------------- producer ---------------------------------------------------
-  uint32_t n_desc = 0;                  // tiles queued so far
-  uint32_t n_load = 0, n_store = 0;     // bulk loads issued / bulk stores issued (ring positions)
-  char* q_dst[kDirectStages] = {};
-  uint32_t q_bytes[kDirectStages] = {};
-  bool failed = false;
+  // --------------------------------- producer warp -----------------------------------------------
+  const uint32_t lane = threadIdx.x;
+  uint32_t n_w = 0;                     // worker-ring slots handed out so far (warp-uniform)
+  uint32_t n_load = 0, n_store = 0;     // direct ring positions (lane 0)
+  bool failed = false;                  // warp-uniform
 
-  auto push_desc = [&](uint32_t k) {
-    const uint32_t q = n_desc % kDescSlots;
-    if (n_desc >= kDescSlots && !mbar_wait(&desc_empty[q], ((n_desc / kDescSlots) - 1) & 1)) {
-      atomicMax(err, ERR_WAIT_DESC_EMPTY); failed = true; return;
-    }
-    desc_tile[q] = k;
-    mbar_arrive(&desc_full[q]);         // release: the tile index is visible to whoever sees the phase
-    ++n_desc;
+  // wait until the workers have released the slot that position n_w maps to
+  auto acquire_slot = [&]() -> bool {
+    uint32_t ok = 1;
+    if (lane == 0 && n_w >= kSlots) ok = mbar_wait(&slot_empty[n_w % kSlots], ((n_w / kSlots) - 1) & 1);
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    if (!ok) { if (lane == 0) atomicMax(err, ERR_WAIT_SLOT_EMPTY); failed = true; }
+    return ok != 0;
   };
-  // store the oldest loaded chunk; then, one store behind, its stage is free for the next load
+  auto push_simple = [&](uint32_t mode, uint32_t tile) {
+    if (!acquire_slot()) return;
+    const uint32_t slot = n_w % kSlots;
+    if (lane == 0) {
+      desc[slot].mode = mode;
+      desc[slot].tile = tile;
+      mbar_arrive(&slot_full[slot]);    // release: the descriptor is visible to whoever sees the phase
+    }
+    ++n_w;
+  };
+  // stage R rows of n elements (row r starts at src + r*sps) into the next slot
+  auto push_staged = [&](uint32_t mode, const char* src, char* dst, uint32_t R, uint32_t n, uint64_t sps,
+                         uint64_t dps, uint32_t pitch) {
+    if (!acquire_slot()) return;
+    const uint32_t slot = n_w % kSlots;
+    char* stage = wring + (size_t)slot * kSlotBytes;
+    uint32_t mine = 0;
+    for (uint32_t r = lane; r < R; r += 32)
+      mine += roundup16((uint32_t)(((uintptr_t)src + (uint64_t)r * sps) & 15u) + n * ES);
+    const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if (lane == 0) {
+      ChunkDesc c;
+      c.mode = mode; c.tile = 0; c.nr = R; c.nc = n; c.pitch = pitch; c.pad = 0;
+      c.src = (uint64_t)(uintptr_t)src; c.dst = (uint64_t)(uintptr_t)dst; c.sps = sps; c.dps = dps;
+      desc[slot] = c;
+      mbar_expect_tx(&slot_full[slot], total);     // the producer's arrival + the bytes to come
+    }
+    __syncwarp();
+    for (uint32_t r = lane; r < R; r += 32) {
+      const uintptr_t a = (uintptr_t)src + (uint64_t)r * sps;
+      bulk_load(stage + (size_t)r * pitch, reinterpret_cast<const void*>(a & ~(uintptr_t)15),
+                roundup16((uint32_t)(a & 15u) + n * ES), &slot_full[slot]);
+    }
+    ++n_w;
+  };
+  // direct ring (lane 0): store the oldest loaded chunk; one store behind, its stage is free again
   auto store_oldest = [&]() {
     const uint32_t st = n_store % kDirectStages;
-    if (!mbar_wait(&full_bar[st], (n_store / kDirectStages) & 1)) { atomicMax(err, ERR_WAIT_LOAD); failed = true; return; }
+    if (!mbar_wait(&direct_full[st], (n_store / kDirectStages) & 1)) { atomicMax(err, ERR_WAIT_LOAD); failed = true; return; }
     fence_async_smem();
     bulk_store(q_dst[st], ring + (size_t)st * kDirectBytes, q_bytes[st]);
     bulk_commit();
     ++n_store;
   };
   auto load_chunk = [&](const char* src, char* dst, uint32_t bytes) {
-    // ring full: retire one chunk and wait until the store before it has drained its stage
     while (!failed && n_load - n_store >= (uint32_t)kDirectStages - 1) { store_oldest(); bulk_wait_read_1(); }
     if (failed) return;
     const uint32_t st = n_load % kDirectStages;
     q_dst[st] = dst;
     q_bytes[st] = bytes;
-    mbar_expect_tx(&full_bar[st], bytes);
-    bulk_load(ring + (size_t)st * kDirectBytes, src, bytes, &full_bar[st]);
+    mbar_expect_tx(&direct_full[st], bytes);
+    bulk_load(ring + (size_t)st * kDirectBytes, src, bytes, &direct_full[st]);
     ++n_load;
   };
 
@@ -457,31 +680,62 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
   for (uint32_t k = begin; k < end && !failed; ++k) {
     const TileFields f = decode(nxt, src_add, dst_add);
     if (k + 1 < end) nxt = load_tile(tiles + k + 1);
-    if (!direct_ok<ES, ED>(f)) { push_desc(k); continue; }
-    for (uint32_t i = 0; i < f.nr && !failed; ++i) {
-      const char* s = f.s + (size_t)i * f.ssr * ES;
-      char* d = f.d + (size_t)i * f.dsr * ED;
-      size_t n = (size_t)f.nc * ES;
-      // bytes before the first / after the last 16-byte boundary: element copies
-      size_t head = (16u - ((uintptr_t)d & 15u)) & 15u;
-      if (head > n) head = n;
-      for (size_t b = 0; b < head; b += ES) Elem<ES, ED>::store(d + b, Elem<ES, ED>::load(s + b));
-      s += head; d += head; n -= head;
-      const size_t body = n & ~(size_t)15;
-      for (size_t b = body; b < n; b += ES) Elem<ES, ED>::store(d + b, Elem<ES, ED>::load(s + b));
-      for (size_t off = 0; off < body && !failed; off += kDirectBytes)
-        load_chunk(s + off, d + off, (uint32_t)min((size_t)kDirectBytes, body - off));
+    if (direct_ok<ES, ED>(f)) {
+      if (lane == 0) {
+        for (uint32_t i = 0; i < f.nr && !failed; ++i) {
+          const char* s = f.s + (size_t)i * f.ssr * ES;
+          char* d = f.d + (size_t)i * f.dsr * ED;
+          size_t n = (size_t)f.nc * ES;
+          // bytes before the first / after the last 16-byte boundary: element copies
+          size_t head = (16u - ((uintptr_t)d & 15u)) & 15u;
+          if (head > n) head = n;
+          for (size_t b = 0; b < head; b += ES) E::store(d + b, E::load(s + b));
+          s += head; d += head; n -= head;
+          const size_t body = n & ~(size_t)15;
+          for (size_t b = body; b < n; b += ES) E::store(d + b, E::load(s + b));
+          for (size_t off = 0; off < body && !failed; off += kDirectBytes)
+            load_chunk(s + off, d + off, (uint32_t)min((size_t)kDirectBytes, body - off));
+        }
+      }
+      failed = __shfl_sync(0xFFFFFFFFu, (uint32_t)failed, 0) != 0;
+    } else if (f.kind == KIND_ROWS && f.n_extra == 0 && (size_t)f.nc * ES >= 128) {
+      const uint32_t row_bytes = f.nc * ES + 16;                 // worst-case aligned superset of a row
+      if (row_bytes <= (uint32_t)kSlotBytes) {
+        const uint32_t pitch = roundup16(row_bytes);
+        const uint32_t per = f.nr == 1 ? 1u : min(f.nr, (uint32_t)kSlotBytes / pitch);
+        for (uint32_t r0 = 0; r0 < f.nr && !failed; r0 += per)
+          push_staged(MODE_ROWS, f.s + (size_t)r0 * f.ssr * ES, f.d + (size_t)r0 * f.dsr * ED,
+                      min(per, f.nr - r0), f.nc, (uint64_t)f.ssr * ES, (uint64_t)f.dsr * ED, pitch);
+      } else {
+        const uint32_t piece = ((uint32_t)kSlotBytes - 32) / ES / 64 * 64;   // elements per column piece
+        for (uint32_t r = 0; r < f.nr && !failed; ++r)
+          for (uint32_t c = 0; c < f.nc && !failed; c += piece)
+            push_staged(MODE_ROWS, f.s + ((size_t)r * f.ssr + c) * ES, f.d + ((size_t)r * f.dsr + c) * ED, 1,
+                        min(piece, f.nc - c), 0, 0, (uint32_t)kSlotBytes);
+      }
+    } else if (f.kind == KIND_TRANS && f.n_extra == 0 && f.nc * ES >= 64 && f.nr >= 4) {
+      const uint32_t cj = min(f.nc, (uint32_t)kTransRowBytes / ES);
+      const uint32_t pitch = roundup16(cj * ES + 16);
+      const uint32_t ri = min(f.nr, (uint32_t)kSlotBytes / pitch / 8 * 8);
+      for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += ri)
+        for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cj)
+          push_staged(MODE_TRANS, f.s + ((size_t)i0 * f.ssr + j0) * ES, f.d + ((size_t)j0 * f.dsc + i0) * ED,
+                      min(ri, f.nr - i0), min(cj, f.nc - j0), (uint64_t)f.ssr * ES, (uint64_t)f.dsc * ED, pitch);
+    } else {
+      push_simple(MODE_COOP, k);
     }
   }
-  while (!failed && n_store < n_load) store_oldest();
-  if (!failed) push_desc(kEndOfWork);
-  bulk_wait_all();
+  if (lane == 0) {
+    while (!failed && n_store < n_load) store_oldest();
+  }
+  failed = __shfl_sync(0xFFFFFFFFu, (uint32_t)failed, 0) != 0;
+  if (!failed) push_simple(MODE_END, 0);
+  if (lane == 0) bulk_wait_all();
 }
 
 // ---------------------------------------------------------------------------------------------
 // launch
 // ---------------------------------------------------------------------------------------------
-constexpr size_t kDynSmem = (size_t)kDirectStages * kDirectBytes;
 
 template <int ES, int ED>
 cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add, uint64_t dst_add,
@@ -491,11 +745,11 @@ cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add
   cudaGetDevice(&dev);
   if (dev >= 0 && dev < 16 && !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(wb_exec_kernel<ES, ED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kDynSmem);
+                                         (int)Rings<ES, ED>::kDyn);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  wb_exec_kernel<ES, ED><<<dim3(plan->grid), dim3(kThreads), kDynSmem, stream>>>(
+  wb_exec_kernel<ES, ED><<<dim3(plan->grid), dim3(kThreads), Rings<ES, ED>::kDyn, stream>>>(
       T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err);
   return cudaGetLastError();
 }
@@ -679,7 +933,8 @@ struct SpinLock {
 // dynamic shared memory.
 template <int ES, int ED>
 cudaError_t static_setup_kernel() {
-  return cudaFuncSetAttribute(wb_exec_kernel<ES, ED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+  return cudaFuncSetAttribute(wb_exec_kernel<ES, ED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)Rings<ES, ED>::kDyn);
 }
 wb_status static_setup(int dev) {
   if (g_static_ptr[dev]) return WB_OK;
@@ -749,10 +1004,10 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
   const uint32_t* d_begin = reinterpret_cast<const uint32_t*>(dbase + off_begin);
   uint32_t* d_err = reinterpret_cast<uint32_t*>(dbase);
   const dim3 grid(plan->grid), block(kThreads);
-  if (es == 2 && ed == 2) wb_exec_kernel<2, 2><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
-  else if (es == 4 && ed == 4) wb_exec_kernel<4, 4><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
-  else if (es == 4 && ed == 2) wb_exec_kernel<4, 2><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
-  else wb_exec_kernel<2, 4><<<grid, block, kDynSmem, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  if (es == 2 && ed == 2) wb_exec_kernel<2, 2><<<grid, block, Rings<2, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  else if (es == 4 && ed == 4) wb_exec_kernel<4, 4><<<grid, block, Rings<4, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  else if (es == 4 && ed == 2) wb_exec_kernel<4, 2><<<grid, block, Rings<4, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  else wb_exec_kernel<2, 4><<<grid, block, Rings<2, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
   if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
   if (flags & WB_STATIC_SYNC_CHECK) {
     uint32_t err = 0;
