@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--grid-ctas", type=int, default=0)
     ap.add_argument("--path", default="remap", choices=["remap", "pack_unpack"])
+    ap.add_argument("--static-schedule", action="store_true",
+                    help="fixed per-block tile ranges instead of run-time batches")
     return ap.parse_args()
 
 
@@ -220,7 +222,8 @@ def main():
     t0 = time.perf_counter()
     tl = wb.Layout(wl.trainer.tensors, wl.trainer.slices)
     rl = wb.Layout(wl.rollout.tensors, wl.rollout.slices)
-    plan = wb.Plan(tl, rl, tile_bytes=args.tile_bytes, grid_ctas=args.grid_ctas)
+    plan = wb.Plan(tl, rl, tile_bytes=args.tile_bytes, grid_ctas=args.grid_ctas,
+                   flags=wb.WB_PLAN_STATIC_SCHEDULE if args.static_schedule else 0)
     plan_s = time.perf_counter() - t0
     stats = plan.stats()
     src = RankArenas(wl.trainer.tensors, dev, fill_byte=0)
@@ -343,6 +346,7 @@ def main():
                           "slabs": stats["n_slabs"], "rounds": stats["n_rounds"],
                           "grid_ctas": stats["grid_ctas"], "tile_bytes": stats["tile_bytes"],
                           "plan_build_s": plan_s, "replicas_per_gpu": 1,
+                          "schedule": "static" if args.static_schedule else "dynamic",
                           "multi_gpu": "independent replicas, no collective"},
                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                "gpu_launches": launches, "pct_of_8TBs_nominal": 100.0 * value / world / 8000.0}

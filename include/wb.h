@@ -103,6 +103,9 @@ typedef struct {
 
 #define WB_PLAN_NO_REPLICA_SPLIT 1u /* read replicated source regions from the lowest rank
                                        only instead of a distinct slice per replica        */
+#define WB_PLAN_STATIC_SCHEDULE 2u  /* every thread block walks the fixed, byte-balanced tile
+                                       range the planner gave it, instead of drawing batches
+                                       of tiles from a shared counter at run time          */
 
 typedef struct {
   uint64_t n_ckpt_tensors;      /* checkpoint tensors the destination consumes              */

@@ -10,8 +10,8 @@
 //          16-byte vector loads and stores with the cast done in registers; unaligned
 //          heads/tails are peeled per run; rows whose pitches keep every run 16-byte
 //          aligned are flattened into one vector index space.
-//   TRANS  source contiguous along j, destination contiguous along i: staged through a
-//          padded shared-memory block so that both sides stay coalesced.
+//   TRANS  source contiguous along j, destination contiguous along i: each warp transposes
+//          32-column blocks through a private shared-memory patch.
 //   ELEM   anything else (strided vectors, fan-out): one element per thread.
 #include <cuda_runtime.h>
 
@@ -308,9 +308,7 @@ template <int ES, int ED> struct Rings {      // worker ring: staged chunks and 
   static constexpr size_t kDirect = ES == ED ? (size_t)kDirectStages * kDirectBytes : 0;
   static constexpr size_t kDyn = kDirect + (size_t)kSlots * kSlotBytes;
 };
-constexpr int kTB = 64;                       // transpose block edge of the fallback path
-constexpr int kTransRowBytes = 256;           // staged transpose: source bytes per row segment
-constexpr int kTransSeg = 32;                 // staged transpose: rows per thread task
+constexpr int kWorkerWarps = kWorkers / 32;
 
 enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_TRANS = 3 };
 
@@ -327,7 +325,6 @@ struct ChunkDesc {
   uint64_t dps;       // destination pitch in bytes: between rows (ROWS) or between columns (TRANS)
 };
 
-__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
 __device__ __forceinline__ uint32_t roundup16(uint32_t x) { return (x + 15u) & ~15u; }
 
 struct TileFields {
@@ -430,60 +427,128 @@ __device__ __forceinline__ void staged_rows(const ChunkDesc& d, const char* stag
   }
 }
 
-// Workers: a staged block of source rows -> destination columns (dst[j*dps + i] = src[i][j]).
-// A thread task is one destination run: column j, kTransSeg consecutive rows; it peels to a
-// 16-byte boundary, writes vectors, then the tail.  Consecutive lanes take consecutive columns,
-// so shared-memory reads of a warp fall in consecutive words.
+// Raw source element from shared memory (32-bit shared-space address) and its cast.
+template <int ES> __device__ __forceinline__ uint32_t lds_raw(uint32_t saddr) {
+  uint32_t v;
+  if constexpr (ES == 4) {
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
+  } else {
+    uint16_t h;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(saddr));
+    v = h;
+  }
+  return v;
+}
+template <int ES, int ED> __device__ __forceinline__ typename Elem<ES, ED>::V cast_raw(uint32_t raw) {
+  if constexpr (ES == ED) return (typename Elem<ES, ED>::V)raw;
+  else if constexpr (ES == 4) return f32_to_bf16(raw);
+  else return raw << 16;
+}
+// two consecutive 2-byte destination elements packed in one word
+template <int ES> __device__ __forceinline__ uint32_t pack_pair16(uint32_t lo, uint32_t hi) {
+  if constexpr (ES == 4) return f32x2_to_bf16x2(lo, hi);
+  else return lo | (hi << 16);
+}
+
+// Workers: transposing tile, dst[j*dsc + i] = cast(src[i*ssr + j]).  No block-wide step: every
+// warp takes 32-column x RB-row blocks of the tile on its own.
+//   phase A  lane = source column.  The warp reads row after row (32 consecutive elements per
+//            load instruction, 16 loads in flight per lane), casts, and writes each value into
+//            its private patch of the ring slot, laid out as destination rows: T[lane][row].
+//   phase B  lane = destination row.  Each row (RB elements, any 2-/4-byte alignment in global
+//            memory) is cut into 16-byte aligned slots: full slots are one vector store assembled
+//            from shared memory with funnel shifts, ragged end slots are element stores.
+// The patch pitch is odd in 32-bit words, so lanes hit distinct banks in both phases.
 template <int ES, int ED>
-__device__ __forceinline__ void staged_trans(const ChunkDesc& d, const char* stage, uint32_t t) {
+__device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratch, uint32_t scratch_bytes,
+                                               uint32_t warp, uint32_t lane) {
   using E = Elem<ES, ED>;
   constexpr uint32_t NV = 16 / ED;
-  const uint32_t ni = d.nr, nj = d.nc;
-  const uint32_t segs = (ni + kTransSeg - 1) / kTransSeg;
-  const uint32_t total = segs * nj;
-  const uint32_t lead0 = (uint32_t)d.src & 15u, dlead = (uint32_t)d.sps & 15u, pitch = d.pitch;
-  for (uint32_t idx = t; idx < total; idx += kWorkers) {
-    const uint32_t sg = idx / nj, j = idx - sg * nj;
-    const uint32_t i0 = sg * kTransSeg, len = min((uint32_t)kTransSeg, ni - i0);
-    char* out = reinterpret_cast<char*>(d.dst + (uint64_t)j * d.dps) + (size_t)i0 * ED;
-    // element i of the column lives at stage + i*pitch + ((src + i*sps) & 15) + j*ES; walk it
-    const char* p = stage + i0 * pitch + j * ES;
-    uint32_t lead = (lead0 + i0 * dlead) & 15u;
-    auto next = [&]() -> typename E::V {
-      const typename E::V v = E::load(p + lead);
-      p += pitch;
-      lead = (lead + dlead) & 15u;
-      return v;
-    };
-    uint32_t head = (uint32_t)((16u - ((uintptr_t)out & 15u)) & 15u) / ED;
-    if (head > len) head = len;
-    for (uint32_t e = 0; e < head; ++e) E::store(out + e * ED, next());
-    const uint32_t nvec = (len - head) / NV;
-    char* o = out + head * ED;
-    for (uint32_t v = 0; v < nvec; ++v, o += 16) {
-      uint4 x;
-      if constexpr (ED == 2) {
-        uint32_t w[4];
+  constexpr uint32_t PER_WORD = 4 / ED;                     // destination elements per 32-bit word
+  // rows per block: as many as the warp's share of the slot allows (multiple of 8, at most 64)
+  const uint32_t share = scratch_bytes / kWorkerWarps / 4;  // words
+  uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD) & ~7u);
+  const uint32_t pitch_w = rb / PER_WORD + 1;               // odd: rb/PER_WORD is even
+  uint32_t* T = reinterpret_cast<uint32_t*>(scratch) + warp * (32 * pitch_w);
+  const uint32_t tbase = smem_u32(T);
+  const uint32_t nbi = (f.nr + rb - 1) / rb, nbj = (f.nc + 31) / 32;
+  for (uint32_t b = warp; b < nbi * nbj; b += kWorkerWarps) {
+    const uint32_t bi = b / nbj, bj = b - bi * nbj;
+    const uint32_t i0 = bi * rb, j0 = bj * 32;
+    const uint32_t ni = min(rb, f.nr - i0), nj = min(32u, f.nc - j0);
+    // ---- phase A
+    if (lane < nj) {
+      const char* src = f.s + ((size_t)i0 * f.ssr + j0 + lane) * ES;
+      const size_t sps = (size_t)f.ssr * ES;
+      const uint32_t trow = tbase + lane * pitch_w * 4;
+      constexpr int UA = 16;                                  // loads in flight per lane
+      for (uint32_t r0 = 0; r0 < ni; r0 += UA) {
+        uint32_t raw[UA];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint32_t lo = next(), hi = next();
-          w[q] = lo | (hi << 16);
+        for (int u = 0; u < UA; ++u) {
+          raw[u] = 0;
+          if (r0 + u < ni) {
+            if constexpr (ES == 4) raw[u] = __ldcs(reinterpret_cast<const uint32_t*>(src + (size_t)(r0 + u) * sps));
+            else raw[u] = __ldcs(reinterpret_cast<const uint16_t*>(src + (size_t)(r0 + u) * sps));
+          }
         }
-        x = make_uint4(w[0], w[1], w[2], w[3]);
-      } else {
-        const uint32_t w0 = next(), w1 = next(), w2 = next(), w3 = next();
-        x = make_uint4(w0, w1, w2, w3);
+        if constexpr (ED == 2) {
+#pragma unroll
+          for (int u = 0; u < UA; u += 2)
+            if (r0 + u < ni)
+              asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 2), "r"(pack_pair16<ES>(raw[u], raw[u + 1])));
+        } else {
+#pragma unroll
+          for (int u = 0; u < UA; ++u)
+            if (r0 + u < ni)
+              asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 4), "r"((uint32_t)cast_raw<ES, ED>(raw[u])));
+        }
       }
-      st16(o, x);
     }
-    for (uint32_t e = head + nvec * NV; e < len; ++e) E::store(out + e * ED, next());
+    __syncwarp();
+    // ---- phase B
+    {
+      const uint32_t smax = (ni + 2 * NV - 2) / NV;             // slots a row can touch
+      for (uint32_t task = lane; task < nj * smax; task += 32) {
+        const uint32_t k = task / nj, j = task - k * nj;         // consecutive lanes: consecutive rows
+        char* out = f.d + ((size_t)(j0 + j) * f.dsc + i0) * ED;   // first element of this run
+        const uint32_t a = (uint32_t)((uintptr_t)out & 15u) / ED;
+        const int32_t e0 = (int32_t)(k * NV) - (int32_t)a;
+        if (e0 >= (int32_t)ni) continue;
+        const uint32_t trow = tbase + j * pitch_w * 4;
+        if (e0 >= 0 && (uint32_t)e0 + NV <= ni) {
+          uint4 x;
+          if constexpr (ED == 4) {
+            x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
+            x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
+          } else {
+            const uint32_t w = trow + ((uint32_t)e0 >> 1) * 4;
+            const uint32_t w0 = lds_raw<4>(w), w1 = lds_raw<4>(w + 4), w2 = lds_raw<4>(w + 8), w3 = lds_raw<4>(w + 12);
+            if (e0 & 1) {
+              const uint32_t w4 = lds_raw<4>(w + 16);
+              x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
+                             __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
+            } else {
+              x = make_uint4(w0, w1, w2, w3);
+            }
+          }
+          st16(reinterpret_cast<char*>(((uintptr_t)out & ~(uintptr_t)15) + 16u * k), x);
+        } else {
+          const uint32_t lo = e0 < 0 ? 0u : (uint32_t)e0;
+          const uint32_t hi = min(ni, (uint32_t)(e0 + (int32_t)NV));
+          for (uint32_t e = lo; e < hi; ++e)
+            E::store(out + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
+        }
+      }
+    }
+    __syncwarp();
   }
 }
 
 // Cooperative execution of one tile by the worker warps (thread t of nth).
-template <int ES, int ED, typename SmemT>
+template <int ES, int ED>
 __device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __restrict__ extras, uint64_t dst_add,
-                                          SmemT& smem, uint32_t t) {
+                                          uint32_t t) {
   using E = Elem<ES, ED>;
   constexpr uint32_t nth = kWorkers;
   const char* s = f.s;
@@ -508,23 +573,6 @@ __device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __res
           const uint32_t i = e / nc, j = e - i * nc;
           E::store(d + ((size_t)i * dsr + j) * ED, E::load(s + ((size_t)i * ssr + j) * ES));
         }
-      }
-    }
-  } else if (f.kind == KIND_TRANS && f.n_extra == 0) {
-    // dst[j*dsc + i] = src[i*ssr + j]; 64x64 blocks through shared memory
-    for (uint32_t i0 = 0; i0 < nr; i0 += kTB) {
-      for (uint32_t j0 = 0; j0 < nc; j0 += kTB) {
-        const uint32_t bi = min((uint32_t)kTB, nr - i0), bj = min((uint32_t)kTB, nc - j0);
-        for (uint32_t e = t; e < bi * kTB; e += nth) {       // j fastest: coalesced on the source
-          const uint32_t i = e / kTB, j = e % kTB;
-          if (j < bj) smem[i][j] = E::load(s + ((size_t)(i0 + i) * ssr + (j0 + j)) * ES);
-        }
-        worker_sync();
-        for (uint32_t e = t; e < bj * kTB; e += nth) {       // i fastest: coalesced on the destination
-          const uint32_t j = e / kTB, i = e % kTB;
-          if (i < bi) E::store(d + ((size_t)(j0 + j) * dsc + (i0 + i)) * ED, smem[i][j]);
-        }
-        worker_sync();
       }
     }
   } else {
@@ -556,22 +604,25 @@ enum : uint32_t { ERR_NONE = 0, ERR_WAIT_LOAD = 1, ERR_WAIT_SLOT_EMPTY = 2, ERR_
 template <int ES, int ED>
 __global__ void __launch_bounds__(kThreads, 1)
 wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta_begin,
-               const DDst* __restrict__ extras, uint64_t src_add, uint64_t dst_add, uint32_t* __restrict__ err) {
+               const DDst* __restrict__ extras, uint64_t src_add, uint64_t dst_add, uint32_t* __restrict__ err,
+               uint32_t n_tiles, uint32_t* __restrict__ sched) {
   using E = Elem<ES, ED>;
   extern __shared__ __align__(128) char dyn_smem[];
   constexpr int kSlots = Rings<ES, ED>::kSlots;
   constexpr int kSlotBytes = Rings<ES, ED>::kSlotBytes;
   char* const ring = dyn_smem;                                         // kDirectStages x kDirectBytes
   char* const wring = dyn_smem + Rings<ES, ED>::kDirect;               // kSlots x kSlotBytes
-  __shared__ typename E::V tsmem[kTB][kTB + (ED == 2 ? 2 : 1)];
   __shared__ __align__(8) uint64_t direct_full[kDirectStages];
   __shared__ __align__(8) uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots];
   __shared__ __align__(16) ChunkDesc desc[kMaxSlots];
   __shared__ char* q_dst[kDirectStages];        // direct ring: where each loaded stage goes
   __shared__ uint32_t q_bytes[kDirectStages];
 
-  const uint32_t begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
-  if (begin >= end) return;
+  // Scheduling: with `sched` the blocks draw batches of consecutive tiles from a shared counter
+  // (large batches first, shrinking towards the end); without it each block walks the fixed
+  // range the planner assigned to it.
+  const uint32_t begin = sched ? 0u : cta_begin[blockIdx.x], end = sched ? 0u : cta_begin[blockIdx.x + 1];
+  if (!sched && begin >= end) return;
   if (threadIdx.x == 0) {
     for (int i = 0; i < kDirectStages; ++i) mbar_init(&direct_full[i], 1);
     for (int i = 0; i < kSlots; ++i) { mbar_init(&slot_full[i], 1); mbar_init(&slot_empty[i], kWorkers / 32); }
@@ -596,11 +647,12 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
       if (tr >= (uint32_t)kWorkers) tr -= kWorkers;
       if (d.mode == MODE_ROWS) {
         staged_rows<ES, ED>(d, stage, tr);
-      } else if (d.mode == MODE_TRANS) {
-        staged_trans<ES, ED>(d, stage, tr);
       } else {
         const TileFields f = decode(load_tile(tiles + d.tile), src_add, dst_add);
-        coop_tile<ES, ED>(f, extras, dst_add, tsmem, t);
+        if (d.mode == MODE_TRANS)
+          warp_transpose<ES, ED>(f, const_cast<char*>(stage), kSlotBytes, tr >> 5, t & 31);
+        else
+          coop_tile<ES, ED>(f, extras, dst_add, t);
       }
       __syncwarp();
       if ((t & 31) == 0) mbar_arrive(&slot_empty[slot]);
@@ -676,10 +728,35 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     ++n_load;
   };
 
-  TileRegs nxt = load_tile(tiles + begin);
-  for (uint32_t k = begin; k < end && !failed; ++k) {
+  uint32_t bk = begin, bend = end;      // current batch [bk, bend)
+  bool first = true;
+  auto next_batch = [&]() -> bool {
+    if (!sched) {
+      const bool ok = first;
+      first = false;
+      return ok;
+    }
+    uint32_t s0 = n_tiles, b = 0;
+    if (lane == 0) {
+      const uint32_t cur = *reinterpret_cast<volatile uint32_t*>(&sched[0]);
+      if (cur < n_tiles) {
+        b = max(1u, (n_tiles - cur) / (gridDim.x * 4u));
+        s0 = atomicAdd(&sched[0], b);
+      }
+    }
+    s0 = __shfl_sync(0xFFFFFFFFu, s0, 0);
+    b = __shfl_sync(0xFFFFFFFFu, b, 0);
+    if (s0 >= n_tiles) return false;
+    bk = s0;
+    bend = min(s0 + b, n_tiles);
+    return true;
+  };
+
+  while (!failed && next_batch()) {
+  TileRegs nxt = load_tile(tiles + bk);
+  for (uint32_t k = bk; k < bend && !failed; ++k) {
     const TileFields f = decode(nxt, src_add, dst_add);
-    if (k + 1 < end) nxt = load_tile(tiles + k + 1);
+    if (k + 1 < bend) nxt = load_tile(tiles + k + 1);
     if (direct_ok<ES, ED>(f)) {
       if (lane == 0) {
         for (uint32_t i = 0; i < f.nr && !failed; ++i) {
@@ -713,24 +790,30 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
             push_staged(MODE_ROWS, f.s + ((size_t)r * f.ssr + c) * ES, f.d + ((size_t)r * f.dsr + c) * ED, 1,
                         min(piece, f.nc - c), 0, 0, (uint32_t)kSlotBytes);
       }
-    } else if (f.kind == KIND_TRANS && f.n_extra == 0 && f.nc * ES >= 64 && f.nr >= 4) {
-      const uint32_t cj = min(f.nc, (uint32_t)kTransRowBytes / ES);
-      const uint32_t pitch = roundup16(cj * ES + 16);
-      const uint32_t ri = min(f.nr, (uint32_t)kSlotBytes / pitch / 8 * 8);
-      for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += ri)
-        for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cj)
-          push_staged(MODE_TRANS, f.s + ((size_t)i0 * f.ssr + j0) * ES, f.d + ((size_t)j0 * f.dsc + i0) * ED,
-                      min(ri, f.nr - i0), min(cj, f.nc - j0), (uint64_t)f.ssr * ES, (uint64_t)f.dsc * ED, pitch);
+    } else if (f.kind == KIND_TRANS && f.n_extra == 0) {
+      push_simple(MODE_TRANS, k);         // no staging: the workers use the slot as scratch
     } else {
       push_simple(MODE_COOP, k);
     }
+  }
   }
   if (lane == 0) {
     while (!failed && n_store < n_load) store_oldest();
   }
   failed = __shfl_sync(0xFFFFFFFFu, (uint32_t)failed, 0) != 0;
   if (!failed) push_simple(MODE_END, 0);
-  if (lane == 0) bulk_wait_all();
+  if (lane == 0) {
+    bulk_wait_all();
+    if (sched) {
+      // the last block to finish re-arms the counters for the next launch of this table
+      __threadfence();
+      if (atomicAdd(&sched[1], 1u) == gridDim.x - 1) {
+        sched[0] = 0;
+        sched[1] = 0;
+        __threadfence();
+      }
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -750,7 +833,8 @@ cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add
     configured[dev] = true;
   }
   wb_exec_kernel<ES, ED><<<dim3(plan->grid), dim3(kThreads), Rings<ES, ED>::kDyn, stream>>>(
-      T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err);
+      T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err, (uint32_t)T.tiles.size(),
+      (plan->opts.flags & WB_PLAN_STATIC_SCHEDULE) ? nullptr : T.d_sched);
   return cudaGetLastError();
 }
 
@@ -800,7 +884,7 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
     size_t bytes = 0;
     for (TileTable* T : tabs)
       bytes += up256(T->tiles.size() * sizeof(DTile)) + up256(T->extras.size() * sizeof(DDst)) +
-               up256(T->cta_begin.size() * sizeof(uint32_t));
+               up256(T->cta_begin.size() * sizeof(uint32_t)) + 256;
     const size_t err_off = up256(bytes);
     bytes = up256(err_off + 256);
     std::vector<char> host(bytes, 0);
@@ -846,6 +930,8 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
       T->d_cta_begin = reinterpret_cast<uint32_t*>(dbase + off);
       std::memcpy(host.data() + off, T->cta_begin.data(), T->cta_begin.size() * sizeof(uint32_t));
       off += up256(T->cta_begin.size() * sizeof(uint32_t));
+      T->d_sched = reinterpret_cast<uint32_t*>(dbase + off);   // {next tile, blocks done}, zero
+      off += 256;
     }
     if (cudaMemcpy(plan->d_arena, host.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess)
       return WB_ERR_CUDA;
@@ -974,7 +1060,7 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
   if (st != WB_OK) { g_static_lock.unlock(); return st; }
   char* dbase = static_cast<char*>(g_static_ptr[dev]);
   // the array keeps the previous call's contents: rebuild everything this launch reads, and
-  // zero the error word
+  // zero the error word and the scheduling counters (first 256 bytes)
   std::memset(g_static_stage, 0, off_tiles);
   DTile* ht = reinterpret_cast<DTile*>(g_static_stage + off_tiles);
   for (size_t k = 0; k < T.tiles.size(); ++k) {
@@ -1003,11 +1089,13 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
   const DDst* d_extras = reinterpret_cast<const DDst*>(dbase + off_extras);
   const uint32_t* d_begin = reinterpret_cast<const uint32_t*>(dbase + off_begin);
   uint32_t* d_err = reinterpret_cast<uint32_t*>(dbase);
+  uint32_t* d_sched = (plan->opts.flags & WB_PLAN_STATIC_SCHEDULE) ? nullptr : reinterpret_cast<uint32_t*>(dbase + 64);
+  const uint32_t n_tiles = (uint32_t)T.tiles.size();
   const dim3 grid(plan->grid), block(kThreads);
-  if (es == 2 && ed == 2) wb_exec_kernel<2, 2><<<grid, block, Rings<2, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
-  else if (es == 4 && ed == 4) wb_exec_kernel<4, 4><<<grid, block, Rings<4, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
-  else if (es == 4 && ed == 2) wb_exec_kernel<4, 2><<<grid, block, Rings<4, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
-  else wb_exec_kernel<2, 4><<<grid, block, Rings<2, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err);
+  if (es == 2 && ed == 2) wb_exec_kernel<2, 2><<<grid, block, Rings<2, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
+  else if (es == 4 && ed == 4) wb_exec_kernel<4, 4><<<grid, block, Rings<4, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
+  else if (es == 4 && ed == 2) wb_exec_kernel<4, 2><<<grid, block, Rings<4, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
+  else wb_exec_kernel<2, 4><<<grid, block, Rings<2, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
   if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
   if (flags & WB_STATIC_SYNC_CHECK) {
     uint32_t err = 0;

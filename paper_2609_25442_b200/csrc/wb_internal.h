@@ -117,6 +117,7 @@ struct TileTable {
   DTile* d_tiles = nullptr;
   DDst* d_extras = nullptr;
   uint32_t* d_cta_begin = nullptr;
+  uint32_t* d_sched = nullptr;        // {next tile, blocks done} for dynamic scheduling
 };
 
 struct Slab {
