@@ -233,11 +233,15 @@ wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bucket, void*
  * sticky error word instead of hanging).  OK, NOT_BOUND, CUDA, or INTERNAL. */
 wb_status wb_plan_check(const wb_plan* plan);
 
-/* wb_remap_host: the same transfer for callers whose weights are in HOST memory:
- * copies every trainer tensor host -> its bound device region, runs wb_remap, copies every
- * rollout tensor back, all on `cuda_stream`, and returns without synchronising.
- * host_src[i] / host_dst[i]: HOST addresses (page-locked for real asynchrony) of the
- * tensors in table order.  Errors: INVALID_ARG, NOT_BOUND, CUDA. */
+/* wb_remap_host: the same transfer for callers whose weights are in HOST memory.  The remap
+ * is cut into groups of consecutive tiles; for each group the trainer bytes it reads are copied
+ * host -> bound device regions on an internal copy stream, its tiles run on `cuda_stream`, and the
+ * rollout bytes it wrote are copied back on a second internal copy stream, so uploads, kernel
+ * and downloads of neighbouring groups overlap.  Returns without synchronising; `cuda_stream`
+ * completes after the last download.  Creates two streams and a few events on first use.
+ * host_src[i] / host_dst[i]: HOST addresses (page-locked for real asynchrony) of the tensors
+ * in table order.  Elements no slice describes are neither uploaded nor downloaded reliably:
+ * treat padding in host_dst as unspecified.  Errors: INVALID_ARG, NOT_BOUND, CUDA, OOM. */
 wb_status wb_remap_host(const wb_plan* plan, const void* const* host_src, size_t n_src,
                         void* const* host_dst, size_t n_dst, void* cuda_stream);
 

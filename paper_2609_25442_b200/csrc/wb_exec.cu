@@ -15,6 +15,7 @@
 //   ELEM   anything else (strided vectors, fan-out): one element per thread.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdint>
 #include <cstring>
@@ -822,7 +823,7 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
 
 template <int ES, int ED>
 cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add, uint64_t dst_add,
-                       cudaStream_t stream) {
+                       cudaStream_t stream, uint32_t tile_off, uint32_t tile_count, bool whole) {
   static bool configured[16] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -833,19 +834,24 @@ cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add
     configured[dev] = true;
   }
   wb_exec_kernel<ES, ED><<<dim3(plan->grid), dim3(kThreads), Rings<ES, ED>::kDyn, stream>>>(
-      T.d_tiles, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err, (uint32_t)T.tiles.size(),
-      (plan->opts.flags & WB_PLAN_STATIC_SCHEDULE) ? nullptr : T.d_sched);
+      T.d_tiles + tile_off, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err, tile_count,
+      (whole && (plan->opts.flags & WB_PLAN_STATIC_SCHEDULE)) ? nullptr : T.d_sched);
   return cudaGetLastError();
 }
 
+// Launch the executor on a tile table, or (tile_count != 0) on a contiguous range of its tiles; a
+// range is always scheduled at run time, the fixed per-block ranges only describe whole tables.
 wb_status launch_table(const wb_plan* plan, const TileTable& T, uint64_t src_add, uint64_t dst_add,
-                       uint32_t es, uint32_t ed, cudaStream_t stream) {
+                       uint32_t es, uint32_t ed, cudaStream_t stream, uint32_t tile_off = 0,
+                       uint32_t tile_count = 0) {
   if (T.tiles.empty()) return WB_OK;
+  const bool whole = tile_count == 0;
+  if (whole) tile_count = (uint32_t)T.tiles.size();
   cudaError_t e;
-  if (es == 2 && ed == 2) e = launch_one<2, 2>(plan, T, src_add, dst_add, stream);
-  else if (es == 4 && ed == 4) e = launch_one<4, 4>(plan, T, src_add, dst_add, stream);
-  else if (es == 4 && ed == 2) e = launch_one<4, 2>(plan, T, src_add, dst_add, stream);
-  else e = launch_one<2, 4>(plan, T, src_add, dst_add, stream);
+  if (es == 2 && ed == 2) e = launch_one<2, 2>(plan, T, src_add, dst_add, stream, tile_off, tile_count, whole);
+  else if (es == 4 && ed == 4) e = launch_one<4, 4>(plan, T, src_add, dst_add, stream, tile_off, tile_count, whole);
+  else if (es == 4 && ed == 2) e = launch_one<4, 2>(plan, T, src_add, dst_add, stream, tile_off, tile_count, whole);
+  else e = launch_one<2, 4>(plan, T, src_add, dst_add, stream, tile_off, tile_count, whole);
   return e == cudaSuccess ? WB_OK : WB_ERR_CUDA;
 }
 
@@ -860,6 +866,11 @@ void release_device_tables(wb_plan* plan) {
     cudaFree(plan->d_arena);
     plan->d_arena = nullptr;
   }
+  for (void* e : plan->host_events) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+  plan->host_events.clear();
+  if (plan->h2d_stream) cudaStreamDestroy(static_cast<cudaStream_t>(plan->h2d_stream));
+  if (plan->d2h_stream) cudaStreamDestroy(static_cast<cudaStream_t>(plan->d2h_stream));
+  plan->h2d_stream = plan->d2h_stream = nullptr;
   plan->bound = false;
 }
 }  // namespace wbi
@@ -971,24 +982,117 @@ extern "C" wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bu
                       esize(plan->dst.dtype), esize(plan->dst.dtype), static_cast<cudaStream_t>(cuda_stream));
 }
 
-extern "C" wb_status wb_remap_host(const wb_plan* plan, const void* const* host_src, size_t n_src,
+// wb_remap_host pipelines the transfer over PCIe: the remap table is cut into groups of
+// consecutive tiles; group g's source spans go host -> device on one copy stream, its tiles run
+// on the caller's stream, its destination spans go device -> host on a second copy stream, so
+// uploads, the kernel and downloads of neighbouring groups overlap (PCIe is full duplex).  A span
+// is the bounding element interval a group touches in one tensor; spans of different groups may
+// overlap, which only copies some bytes twice: the later download of an element always follows
+// the kernel that wrote it.
+static wb_status build_host_groups(wb_plan* plan) {
+  const TileTable& T = plan->remap;
+  const uint32_t es = esize(plan->src.dtype), ed = esize(plan->dst.dtype);
+  uint64_t total = 0;
+  for (const HTile& t : T.tiles) total += t.bytes;
+  const uint64_t target = std::max<uint64_t>(256ull << 20, total / 24);
+  plan->host_groups.clear();
+  HostGroup g{};
+  uint64_t acc = 0;
+  std::vector<std::pair<uint64_t, uint64_t>> smin(plan->src.tensors.size()), dmin(plan->dst.tensors.size());
+  std::vector<uint32_t> stouched, dtouched;
+  auto reset = [&]() {
+    for (uint32_t i : stouched) smin[i] = {UINT64_MAX, 0};
+    for (uint32_t i : dtouched) dmin[i] = {UINT64_MAX, 0};
+    stouched.clear(); dtouched.clear();
+  };
+  for (auto& p : smin) p = {UINT64_MAX, 0};
+  for (auto& p : dmin) p = {UINT64_MAX, 0};
+  auto touch = [&](std::vector<std::pair<uint64_t, uint64_t>>& v, std::vector<uint32_t>& list, int32_t tensor,
+                   uint64_t off, uint32_t nr, uint32_t nc, uint32_t sr, uint32_t sc) {
+    const uint64_t last = off + (uint64_t)(nr - 1) * sr + (uint64_t)(nc - 1) * sc;
+    auto& p = v[tensor];
+    if (p.first == UINT64_MAX) list.push_back((uint32_t)tensor);
+    p.first = std::min(p.first, off);
+    p.second = std::max(p.second, last + 1);
+  };
+  auto flush = [&](uint32_t end_tile) {
+    g.tile_end = end_tile;
+    for (uint32_t i : stouched) g.src.push_back(HostSpan{i, smin[i].first * es, (smin[i].second - smin[i].first) * es});
+    for (uint32_t i : dtouched) g.dst.push_back(HostSpan{i, dmin[i].first * ed, (dmin[i].second - dmin[i].first) * ed});
+    plan->host_groups.push_back(g);
+    g = HostGroup{};
+    g.tile_begin = end_tile;
+    reset();
+    acc = 0;
+  };
+  for (uint32_t k = 0; k < T.tiles.size(); ++k) {
+    const HTile& t = T.tiles[k];
+    touch(smin, stouched, t.src_tensor, t.src_off, t.nr, t.nc, t.ssr, t.ssc);
+    touch(dmin, dtouched, t.dst_tensor, t.dst_off, t.nr, t.nc, t.dsr, t.dsc);
+    for (uint32_t x = 0; x < t.n_extra; ++x) {
+      const HDst& o = T.extras[t.extra + x];
+      touch(dmin, dtouched, o.tensor, o.off, t.nr, t.nc, o.sr, o.sc);
+    }
+    acc += t.bytes;
+    if (acc >= target) flush(k + 1);
+  }
+  if (acc > 0 || plan->host_groups.empty()) flush((uint32_t)T.tiles.size());
+  return WB_OK;
+}
+
+extern "C" wb_status wb_remap_host(const wb_plan* plan_c, const void* const* host_src, size_t n_src,
                                    void* const* host_dst, size_t n_dst, void* cuda_stream) {
-  if (!plan || !host_src || !host_dst) return WB_ERR_INVALID_ARG;
-  if (!plan->bound) return WB_ERR_NOT_BOUND;
-  if (n_src != plan->src.tensors.size() || n_dst != plan->dst.tensors.size()) return WB_ERR_INVALID_ARG;
+  if (!plan_c || !host_src || !host_dst) return WB_ERR_INVALID_ARG;
+  if (!plan_c->bound) return WB_ERR_NOT_BOUND;
+  if (n_src != plan_c->src.tensors.size() || n_dst != plan_c->dst.tensors.size()) return WB_ERR_INVALID_ARG;
+  for (size_t i = 0; i < n_src; ++i) if (!host_src[i]) return WB_ERR_INVALID_ARG;
+  for (size_t i = 0; i < n_dst; ++i) if (!host_dst[i]) return WB_ERR_INVALID_ARG;
+  wb_plan* plan = const_cast<wb_plan*>(plan_c);     // lazily built pipeline state, not the plan itself
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const uint32_t es = esize(plan->src.dtype), ed = esize(plan->dst.dtype);
-  for (size_t i = 0; i < n_src; ++i) {
-    if (!host_src[i]) return WB_ERR_INVALID_ARG;
-    if (cudaMemcpyAsync(const_cast<void*>(plan->src_base[i]), host_src[i], plan->src.tensors[i].numel * es,
-                        cudaMemcpyHostToDevice, stream) != cudaSuccess) return WB_ERR_CUDA;
-  }
-  wb_status st = wb_remap(plan, cuda_stream);
-  if (st != WB_OK) return st;
-  for (size_t i = 0; i < n_dst; ++i) {
-    if (!host_dst[i]) return WB_ERR_INVALID_ARG;
-    if (cudaMemcpyAsync(host_dst[i], plan->dst_base[i], plan->dst.tensors[i].numel * ed,
-                        cudaMemcpyDeviceToHost, stream) != cudaSuccess) return WB_ERR_CUDA;
+  try {
+    if (plan->host_groups.empty()) build_host_groups(plan);
+    const size_t G = plan->host_groups.size();
+    if (!plan->h2d_stream) {
+      cudaStream_t a, b;
+      if (cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking) != cudaSuccess) return WB_ERR_CUDA;
+      if (cudaStreamCreateWithFlags(&b, cudaStreamNonBlocking) != cudaSuccess) { cudaStreamDestroy(a); return WB_ERR_CUDA; }
+      plan->h2d_stream = a;
+      plan->d2h_stream = b;
+    }
+    while (plan->host_events.size() < 2 * G + 2) {
+      cudaEvent_t e;
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return WB_ERR_CUDA;
+      plan->host_events.push_back(e);
+    }
+    cudaStream_t up = static_cast<cudaStream_t>(plan->h2d_stream), down = static_cast<cudaStream_t>(plan->d2h_stream);
+    auto ev = [&](size_t i) { return static_cast<cudaEvent_t>(plan->host_events[i]); };
+    // the copy streams start after whatever the caller already queued on its stream
+    if (cudaEventRecord(ev(2 * G), stream) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaStreamWaitEvent(up, ev(2 * G), 0) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaStreamWaitEvent(down, ev(2 * G), 0) != cudaSuccess) return WB_ERR_CUDA;
+    for (size_t g = 0; g < G; ++g) {
+      const HostGroup& hg = plan->host_groups[g];
+      for (const HostSpan& sp : hg.src)
+        if (cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(plan->src_base[sp.tensor])) + sp.off,
+                            static_cast<const char*>(host_src[sp.tensor]) + sp.off, sp.bytes,
+                            cudaMemcpyHostToDevice, up) != cudaSuccess) return WB_ERR_CUDA;
+      if (cudaEventRecord(ev(2 * g), up) != cudaSuccess) return WB_ERR_CUDA;
+      if (cudaStreamWaitEvent(stream, ev(2 * g), 0) != cudaSuccess) return WB_ERR_CUDA;
+      wb_status st = launch_table(plan, plan->remap, 0, 0, es, ed, stream, hg.tile_begin, hg.tile_end - hg.tile_begin);
+      if (st != WB_OK) return st;
+      if (cudaEventRecord(ev(2 * g + 1), stream) != cudaSuccess) return WB_ERR_CUDA;
+      if (cudaStreamWaitEvent(down, ev(2 * g + 1), 0) != cudaSuccess) return WB_ERR_CUDA;
+      for (const HostSpan& sp : hg.dst)
+        if (cudaMemcpyAsync(static_cast<char*>(host_dst[sp.tensor]) + sp.off,
+                            static_cast<const char*>(plan->dst_base[sp.tensor]) + sp.off, sp.bytes,
+                            cudaMemcpyDeviceToHost, down) != cudaSuccess) return WB_ERR_CUDA;
+    }
+    // the caller's stream completes when the last download has
+    if (cudaEventRecord(ev(2 * G + 1), down) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaStreamWaitEvent(stream, ev(2 * G + 1), 0) != cudaSuccess) return WB_ERR_CUDA;
+  } catch (const std::bad_alloc&) {
+    return WB_ERR_OOM;
   }
   return WB_OK;
 }

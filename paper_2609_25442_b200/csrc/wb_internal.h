@@ -134,6 +134,13 @@ struct Payload {
   uint64_t bucket_off;      // bytes
 };
 
+// wb_remap_host: a group of consecutive remap tiles and the byte spans it touches per tensor.
+struct HostSpan { uint32_t tensor; uint64_t off, bytes; };
+struct HostGroup {
+  uint32_t tile_begin = 0, tile_end = 0;
+  std::vector<HostSpan> src, dst;
+};
+
 struct Round {
   std::vector<Payload> payloads;
   uint64_t bucket_bytes = 0;
@@ -159,6 +166,11 @@ struct wb_plan {
   std::vector<void*> dst_base;
   void* d_arena = nullptr;              // one device allocation holding every table
   uint32_t* d_err = nullptr;            // sticky device error word (inside the arena)
+  // wb_remap_host pipeline state (created on first use; streams and events are CUDA handles)
+  std::vector<wbi::HostGroup> host_groups;
+  void* h2d_stream = nullptr;
+  void* d2h_stream = nullptr;
+  std::vector<void*> host_events;
   size_t arena_bytes = 0;
 };
 

@@ -5,6 +5,8 @@ The output must equal what the ordinary bind + wb_remap path writes, bit for bit
 in a row that use different plans (so stale contents of the shared array would show).
 
 This file is named to be collected last."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -34,11 +36,13 @@ def test_static_scratch_matches_bound_remap_twice_in_a_row():
     stream = torch.cuda.current_stream().cuda_stream
     a_case, a_plan, a_want = _reference_and_static(device, "cfg3", "small")      # fp32 -> bf16, fan-out
     b_case, b_plan, b_want = _reference_and_static(device, "cfg1b", "full")      # padding, replicas
+    gc.collect()                                  # plans of earlier tests free their arenas now, not later
+    torch.cuda.synchronize()
     free_before = torch.cuda.mem_get_info()[0]
     wb.wb_remap_static(a_plan, a_case.src.pointers(), a_case.dst.pointers(), 0, stream)
     wb.wb_remap_static(b_plan, b_case.src.pointers(), b_case.dst.pointers(), wb.WB_STATIC_SYNC_CHECK, stream)
     torch.cuda.synchronize()
-    assert torch.cuda.mem_get_info()[0] == free_before            # no device memory was taken
+    assert torch.cuda.mem_get_info()[0] >= free_before            # no device memory was taken
     for got, want in zip(a_case.dst_bits(), a_want):
         assert np.array_equal(got, want)
     for got, want in zip(b_case.dst_bits(), b_want):
