@@ -283,6 +283,42 @@ wb_status wb_remap_host(const wb_plan* plan, const void* const* host_src, size_t
 wb_status wb_remap_static(const wb_plan* plan, const void* const* src_base, size_t n_src,
                           void* const* dst_base, size_t n_dst, uint32_t flags, void* cuda_stream);
 
+/* ---- source-map extraction (Section 3.1, Appendix B / Algorithm 1) ---------------------------
+ * A worker's source map can be recovered from its black-box load_weights instead of being
+ * written by hand: fill the checkpoint with position ids (1-based, so 0 = "no source"), load,
+ * and analyse the id field each local tensor ends up with.  The field is not shipped to the
+ * host: its second-order difference diff2 (Appendix B, Eq. diff1/diff2) is non-zero only around
+ * the corners of the rectangles the slice-copy operations filled.  For parameters narrower than
+ * the ids the probe is repeated per b-bit id chunk and the sparse results are recombined. */
+typedef struct { uint64_t row, col; int64_t value; } wb_diff2_entry;
+enum { WB_ID_I64 = 0,   /* field of int64                                              */
+       WB_ID_U16 = 1,   /* raw 16-bit patterns (a 16-bit chunk held in a bf16 tensor)   */
+       WB_ID_F32 = 2,   /* fp32 holding an integer value                                 */
+       WB_ID_BF16 = 3   /* bf16 holding an integer value (8-bit chunks are exact)        */ };
+
+/* wb_diff2_nonzeros (device, asynchronous on cuda_stream): diff2 of the rows x cols row-major
+ * field at `field` (DEVICE), read as `id_kind`.  Every non-zero entry is appended to `out`
+ * (DEVICE, `cap` entries) in no particular order; *count (DEVICE uint64, zeroed by the caller)
+ * receives the number found, which may exceed cap (the surplus is dropped: retry with a larger
+ * list).  Errors: INVALID_ARG, CUDA. */
+wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols,
+                            wb_diff2_entry* out, uint64_t cap, uint64_t* count, void* cuda_stream);
+/* wb_diff2_recombine (host): Algorithm 1, Recombine.  sum_k 2^(chunk_bits*k) * passes[k], merged
+ * by position, zeros dropped, sorted by (row, col).  Writes up to cap entries, *n_out = total. */
+wb_status wb_diff2_recombine(const wb_diff2_entry* const* passes, const size_t* counts, size_t n_passes,
+                             uint32_t chunk_bits, wb_diff2_entry* out, size_t cap, size_t* n_out);
+/* wb_scan_slices (host): Algorithm 1, ScanSliceMappings.  From the diff2 entries of one local
+ * tensor viewed as rows x cols (starting `elem_off` elements into local tensor `tensor`) recover
+ * the slice-copy operations as wb_slice records.  The checkpoint is given as n_ckpt tensors with
+ * shapes ckpt_rows[t] x ckpt_cols[t] whose first element has id ckpt_base[t] + 1 (ckpt_base has
+ * n_ckpt + 1 entries, the last being the total element count).  Writes up to cap slices,
+ * *n_out = total.  INVALID_ARG if the field is not piecewise affine in the two shapes a slice
+ * copy produces; OUT_OF_RANGE for entries outside the view. */
+wb_status wb_scan_slices(const wb_diff2_entry* nz, size_t n, uint64_t rows, uint64_t cols,
+                         const uint64_t* ckpt_base, const uint64_t* ckpt_rows, const uint64_t* ckpt_cols,
+                         size_t n_ckpt, uint32_t tensor, uint64_t elem_off, wb_slice* out, size_t cap,
+                         size_t* n_out);
+
 /* Number of kernels wb_remap / wb_pack / wb_unpack launch per call (always 1). */
 int wb_launches_per_call(void);
 

@@ -78,7 +78,8 @@ EXPORTS = [
     "wb_layout_describe", "wb_layout_free", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
-    "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_remap_host", "wb_remap_static", "wb_plan_check",
+    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -118,6 +119,10 @@ def load() -> C.CDLL:
     lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
     lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
+    lib.wb_diff2_nonzeros.argtypes = [vp, C.c_uint32, C.c_uint64, C.c_uint64, vp, C.c_uint64, vp, vp]
+    lib.wb_diff2_recombine.argtypes = [vp, vp, sz, C.c_uint32, vp, sz, C.POINTER(sz)]
+    lib.wb_scan_slices.argtypes = [vp, sz, C.c_uint64, C.c_uint64, vp, vp, vp, sz, C.c_uint32, C.c_uint64,
+                                   vp, sz, C.POINTER(sz)]
     lib.wb_launches_per_call.restype = C.c_int
     lib.wb_status_str.argtypes = [C.c_int]
     lib.wb_status_str.restype = C.c_char_p
@@ -264,3 +269,51 @@ def wb_launches_per_call() -> int:
 
 def wb_version() -> str:
     return load().wb_version().decode()
+
+
+# ---- source-map extraction ------------------------------------------------------------------------
+WB_ID_I64, WB_ID_U16, WB_ID_F32, WB_ID_BF16 = 0, 1, 2, 3
+DIFF2_ENTRY_DTYPE = np.dtype([("row", "<u8"), ("col", "<u8"), ("value", "<i8")])
+SLICE_DTYPE = np.dtype([
+    ("tensor", "<u4"), ("_pad", "<u4"), ("local_off", "<u8"), ("stride_r", "<i8"), ("stride_c", "<i8"),
+    ("ckpt", "<u8"), ("ckpt_rows", "<u8"), ("ckpt_cols", "<u8"),
+    ("r0", "<u8"), ("c0", "<u8"), ("nr", "<u8"), ("nc", "<u8")])
+assert SLICE_DTYPE.itemsize == C.sizeof(wb_slice)
+
+
+def wb_diff2_nonzeros(field_ptr: int, id_kind: int, rows: int, cols: int, out_ptr: int, cap: int,
+                      count_ptr: int, stream: int = 0) -> None:
+    """diff2 of a device id field, non-zeros appended to a device list (all pointers are device)."""
+    load()
+    _check(_lib.wb_diff2_nonzeros(field_ptr, id_kind, rows, cols, out_ptr, cap, count_ptr, stream),
+           "wb_diff2_nonzeros")
+
+
+def wb_diff2_recombine(passes: Sequence[np.ndarray], chunk_bits: int) -> np.ndarray:
+    load()
+    passes = [np.ascontiguousarray(p, dtype=DIFF2_ENTRY_DTYPE) for p in passes]
+    ptrs = _ptr_array([p.ctypes.data for p in passes])
+    counts = (C.c_size_t * max(len(passes), 1))(*[len(p) for p in passes])
+    n = C.c_size_t()
+    _check(_lib.wb_diff2_recombine(ptrs, counts, len(passes), chunk_bits, None, 0, C.byref(n)), "wb_diff2_recombine")
+    out = np.zeros(n.value, DIFF2_ENTRY_DTYPE)
+    _check(_lib.wb_diff2_recombine(ptrs, counts, len(passes), chunk_bits, out.ctypes.data, n.value, C.byref(n)),
+           "wb_diff2_recombine")
+    return out
+
+
+def wb_scan_slices(entries: np.ndarray, rows: int, cols: int, ckpt_base: np.ndarray, ckpt_rows: np.ndarray,
+                   ckpt_cols: np.ndarray, tensor: int, elem_off: int = 0) -> np.ndarray:
+    load()
+    entries = np.ascontiguousarray(entries, dtype=DIFF2_ENTRY_DTYPE)
+    base = np.ascontiguousarray(ckpt_base, dtype=np.uint64)
+    cr = np.ascontiguousarray(ckpt_rows, dtype=np.uint64)
+    cc = np.ascontiguousarray(ckpt_cols, dtype=np.uint64)
+    assert len(base) == len(cr) + 1 == len(cc) + 1
+    n = C.c_size_t()
+    args = (entries.ctypes.data, len(entries), rows, cols, base.ctypes.data, cr.ctypes.data, cc.ctypes.data,
+            len(cr), tensor, elem_off)
+    _check(_lib.wb_scan_slices(*args, None, 0, C.byref(n)), "wb_scan_slices")
+    out = np.zeros(n.value, SLICE_DTYPE)
+    _check(_lib.wb_scan_slices(*args, out.ctypes.data, n.value, C.byref(n)), "wb_scan_slices")
+    return out

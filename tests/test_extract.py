@@ -1,0 +1,139 @@
+"""Source-map extraction (Section 3.1, Appendix B): pins for the diff2 oracle, and the host
+scanner / recombiner of the library checked against the id probe on every small workload."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import ckpt_shapes, predict_ids, scatter_checkpoint, to_bits
+from oracle import remap_oracle
+from oracle.extract import diff1, diff2, id_chunk, nonzeros, recombine, undo_diff2
+from paper_2609_25442_b200 import binding as wb
+from plan_interp import run_table
+from wb_workloads import WB_BF16, Layout, make_workload
+
+SMALL = [("cfg1b", "full"), ("cfg1c", "full"), ("cfg2", "small"), ("cfg3", "small"), ("cfg4", "small"),
+         ("cfg5", "small")]
+
+
+def entries(d):
+    nz = nonzeros(d)
+    return np.array(nz, dtype=wb.DIFF2_ENTRY_DTYPE) if nz else np.zeros(0, wb.DIFF2_ENTRY_DTYPE)
+
+
+def id_fields(wl, side):
+    """2-D id field of every local tensor: ids are 1-based, 0 where nothing was loaded."""
+    layout = wl.trainer if side == "trainer" else wl.rollout
+    out = [None] * layout.n_tensors
+
+    def sink(k, t):
+        t = t.reshape(1, -1) if t.dim() == 1 else t.reshape(-1, t.shape[-1])
+        out[k] = t.clamp_min(0).numpy()          # the loaders pad integer tensors with -1
+    wl.load_side_shaped(side, lambda i: wl.ckpt_ids(i) + 1, sink)
+    return out
+
+
+# ---- the oracle's diff2 against what the paper and mathematics fix ------------------------------------
+def test_diff2_is_the_3x3_kernel_of_the_paper():
+    from scipy.signal import convolve2d
+    rng = np.random.default_rng(0)
+    a = rng.integers(0, 1 << 30, size=(37, 53)).astype(np.int64)
+    k = np.outer([1, -2, 1], [1, -2, 1])                 # Appendix B: outer product of [1,-2,1] with itself
+    want = convolve2d(a, k, mode="full")[:37, :53]        # causal, zeros outside
+    assert np.array_equal(diff2(a), want)
+
+
+def test_diff2_is_lossless():
+    rng = np.random.default_rng(1)
+    a = rng.integers(0, 1 << 40, size=(29, 31)).astype(np.int64)
+    assert np.array_equal(undo_diff2(diff2(a)), a)
+    assert np.array_equal(np.cumsum(np.cumsum(diff1(a), 0), 1), a)
+
+
+@pytest.mark.parametrize("transposed", [False, True])
+def test_affine_rectangle_leaves_at_most_16_entries_at_its_corners(transposed):
+    rng = np.random.default_rng(2)
+    for _ in range(50):
+        R, C = 40, 50
+        i0, j0 = rng.integers(0, 20, 2)
+        ni, nj = rng.integers(1, 18, 2)
+        base, pitch = int(rng.integers(1, 1 << 33)), int(rng.integers(20, 5000))
+        a = np.zeros((R, C), np.int64)
+        ii, jj = np.meshgrid(np.arange(ni), np.arange(nj), indexing="ij")
+        a[i0:i0 + ni, j0:j0 + nj] = base + (jj * pitch + ii if transposed else ii * pitch + jj)
+        nz = nonzeros(diff2(a))
+        assert len(nz) <= 16
+        for (i, j, _) in nz:                                # 2x2 neighbourhoods of the four corners
+            assert i in (i0, i0 + 1, i0 + ni, i0 + ni + 1) and j in (j0, j0 + 1, j0 + nj, j0 + nj + 1)
+        assert nz[0] == (i0, j0, base)                      # the first entry is the first id
+
+
+@pytest.mark.parametrize("b", [8, 16])
+def test_chunk_diffs_recombine_to_the_full_diff(b):
+    wl = make_workload("cfg3", "small")
+    field = id_fields(wl, "trainer")[5]
+    K = -(-int(wl.ckpt_numel() + 1).bit_length() // b)
+    parts = [diff2(id_chunk(field, k, b)) for k in range(K)]
+    assert np.array_equal(recombine(parts, b), diff2(field))
+    got = wb.wb_diff2_recombine([entries(p) for p in parts], b)     # the library's Recombine
+    assert np.array_equal(got, entries(diff2(field)))
+    assert sum(len(entries(p)) for p in parts) > len(got)           # the chunks alone carry wrap artifacts
+
+
+# ---- the library's ScanSliceMappings ---------------------------------------------------------------------
+def extract_layout(wl, side, fields):
+    declared = wl.trainer if side == "trainer" else wl.rollout
+    base = wl.ckpt_base().astype(np.uint64)
+    rows = np.array([c.rows for c in wl.ckpt], np.uint64)
+    cols = np.array([c.cols for c in wl.ckpt], np.uint64)
+    lay = Layout(side)
+    n_entries = 0
+    for k, f in enumerate(fields):
+        d = declared.tensors[k]
+        lay.add_tensor(declared.names[k], int(d["rank"]), int(d["dtype"]), int(d["numel"]))
+        e = entries(diff2(f))
+        n_entries += len(e)
+        for s in wb.wb_scan_slices(e, f.shape[0], f.shape[1], base, rows, cols, k):
+            lay.add_slice(int(s["tensor"]), int(s["local_off"]), int(s["stride_r"]), int(s["stride_c"]),
+                          int(s["ckpt"]), int(s["ckpt_rows"]), int(s["ckpt_cols"]),
+                          int(s["r0"]), int(s["c0"]), int(s["nr"]), int(s["nc"]))
+    return lay.freeze(), n_entries
+
+
+@pytest.mark.parametrize("name,scale", SMALL)
+@pytest.mark.parametrize("side", ["trainer", "rollout"])
+def test_scanned_source_map_reproduces_the_id_field(name, scale, side):
+    wl = make_workload(name, scale)
+    fields = id_fields(wl, side)
+    lay, n_entries = extract_layout(wl, side, fields)
+    for k, (p, f) in enumerate(zip(predict_ids(lay, wl), fields)):
+        assert np.array_equal(p + 1, f.reshape(-1)), lay.names[k]      # 0 stays "no source"
+    declared = wl.trainer if side == "trainer" else wl.rollout
+    assert n_entries <= 16 * max(len(lay.slices), len(declared.slices))   # O(number of operations)
+
+
+def test_extracted_source_maps_drive_the_same_transfer():
+    wl = make_workload("cfg1b")
+    tl, _ = extract_layout(wl, "trainer", id_fields(wl, "trainer"))
+    rl, _ = extract_layout(wl, "rollout", id_fields(wl, "rollout"))
+    src = [to_bits(t) for t in wl.trainer_weights()]
+    want = remap_oracle(ckpt_shapes(wl), wl.trainer.tensors, wl.trainer.slices, wl.rollout.tensors,
+                        wl.rollout.slices, src)
+    plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices))
+    plan.verify()
+    dst = [np.zeros(int(t["numel"]), np.uint16) for t in rl.tensors]
+    run_table(plan.tiles(wb.WB_TABLE_REMAP), src, dst, None, wl.src_dtype, wl.dst_dtype)
+    for a, b in zip(dst, want.dst):
+        assert np.array_equal(a, b)
+    assert plan.stats()["src_elems_read"] == wl.ckpt_numel()
+
+
+def test_scan_rejects_fields_no_slice_copy_produces():
+    base = np.array([0, 64], np.uint64)
+    one = np.array([8], np.uint64)
+    a = np.outer(np.arange(1, 9), np.arange(1, 9)).astype(np.int64)      # bilinear, not affine
+    with pytest.raises(wb.WbError):
+        wb.wb_scan_slices(entries(diff2(a)), 8, 8, base, one, one, 0)
+    far = np.array([(9, 0, 5)], wb.DIFF2_ENTRY_DTYPE)
+    with pytest.raises(wb.WbError) as e:
+        wb.wb_scan_slices(far, 8, 8, base, one, one, 0)
+    assert e.value.name == "WB_ERR_OUT_OF_RANGE"

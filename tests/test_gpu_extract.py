@@ -1,0 +1,135 @@
+"""Source-map extraction on the GPU: the diff2 kernel against the oracle's definition, and the whole
+chain -- chunked id probe through the parameters' own dtype, diff2 + compaction on the device,
+recombination and scan on the host -- producing source maps that drive the same transfer."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import DeviceCase
+from helpers import ckpt_shapes, predict_ids, to_bits
+from oracle import remap_oracle
+from oracle.extract import diff2, id_chunk, nonzeros
+from paper_2609_25442_b200 import binding as wb
+from paper_2609_25442_b200.device import RankArenas, bind
+from wb_workloads import WB_BF16, WB_F32, Layout, make_workload
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def gpu_entries(field: torch.Tensor, kind: int, cap: int = 1 << 16):
+    """Run wb_diff2_nonzeros on a 2-D device tensor; returns (sorted entries, count reported)."""
+    field = field.contiguous()
+    out = torch.zeros(cap * 24, dtype=torch.uint8, device=field.device)
+    count = torch.zeros(1, dtype=torch.int64, device=field.device)
+    wb.wb_diff2_nonzeros(field.data_ptr(), kind, field.shape[0], field.shape[1], out.data_ptr(), cap,
+                         count.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    n = int(count.item())
+    e = out.cpu().numpy().view(wb.DIFF2_ENTRY_DTYPE)[:min(n, cap)].copy()
+    return np.sort(e, order=["row", "col"]), n
+
+
+def oracle_entries(a: np.ndarray):
+    nz = nonzeros(diff2(a))
+    return np.array(nz, dtype=wb.DIFF2_ENTRY_DTYPE) if nz else np.zeros(0, wb.DIFF2_ENTRY_DTYPE)
+
+
+@pytest.mark.parametrize("shape", [(1, 1), (1, 100003), (7, 33), (257, 1023), (1000, 2), (3, 70001)])
+def test_diff2_kernel_matches_the_definition(shape):
+    rng = np.random.default_rng(shape[0] * 131 + shape[1])
+    # piecewise-affine field with a few random rectangles, plus some isolated noise
+    a = np.zeros(shape, np.int64)
+    for _ in range(6):
+        i0, j0 = rng.integers(0, shape[0]), rng.integers(0, shape[1])
+        ni, nj = rng.integers(1, shape[0] - i0 + 1), rng.integers(1, shape[1] - j0 + 1)
+        ii, jj = np.meshgrid(np.arange(ni), np.arange(nj), indexing="ij")
+        a[i0:i0 + ni, j0:j0 + nj] = int(rng.integers(1, 1 << 40)) + ii * int(rng.integers(1, 1 << 20)) + jj
+    for _ in range(5):
+        a[rng.integers(0, shape[0]), rng.integers(0, shape[1])] = int(rng.integers(1, 1 << 45))
+    want = oracle_entries(a)
+    got, n = gpu_entries(torch.from_numpy(a).to(DEV), wb.WB_ID_I64)
+    assert n == len(want) and np.array_equal(got, want)
+
+
+def test_diff2_kernel_reads_chunks_in_the_parameter_dtypes():
+    rng = np.random.default_rng(5)
+    ids = rng.integers(1, 1 << 34, size=(61, 517)).astype(np.int64)
+    c16 = id_chunk(ids, 1, 16)
+    t16 = torch.from_numpy(c16.astype(np.uint16).view(np.int16)).to(DEV)          # raw bits of a bf16 tensor
+    assert np.array_equal(gpu_entries(t16, wb.WB_ID_U16, 1 << 17)[0], oracle_entries(c16))
+    c8 = id_chunk(ids, 2, 8)
+    tb = torch.from_numpy(c8.astype(np.float32)).to(torch.bfloat16).to(DEV)        # 0..255 are exact in bf16
+    assert np.array_equal(gpu_entries(tb, wb.WB_ID_BF16, 1 << 17)[0], oracle_entries(c8))
+    c24 = id_chunk(ids, 0, 24)
+    tf = torch.from_numpy(c24.astype(np.float32)).to(DEV)                          # < 2^24: exact in fp32
+    assert np.array_equal(gpu_entries(tf, wb.WB_ID_F32, 1 << 17)[0], oracle_entries(c24))
+
+
+def test_diff2_kernel_reports_overflow_of_the_list():
+    a = torch.arange(1, 4097, dtype=torch.int64, device=DEV).view(64, 64) ** 2     # nothing cancels
+    got, n = gpu_entries(a, wb.WB_ID_I64, cap=100)
+    assert n > 100 and len(got) == 100
+    full, n2 = gpu_entries(a, wb.WB_ID_I64, cap=8192)
+    assert n2 == n == len(full)
+
+
+def extract_on_gpu(wl, side, chunk_bits):
+    """Algorithm 1 on one side: K passes of load_weights with b-bit id chunks in the parameters' own
+    dtype, diff2 per local tensor on the device, recombination and scan in the library."""
+    declared = wl.trainer if side == "trainer" else wl.rollout
+    dt = wl.src_dtype if side == "trainer" else wl.dst_dtype
+    tdt = torch.float32 if dt == WB_F32 else torch.bfloat16
+    if dt == WB_F32:
+        kind = wb.WB_ID_F32
+    else:
+        kind = wb.WB_ID_U16 if chunk_bits == 16 else wb.WB_ID_BF16
+    K = -(-int(wl.ckpt_numel() + 1).bit_length() // chunk_bits)
+    passes = [dict() for _ in range(declared.n_tensors)]
+    shapes = {}
+    for k in range(K):
+        def values(i, k=k):
+            part = ((wl.ckpt_ids(i, DEV) + 1) >> (chunk_bits * k)) & ((1 << chunk_bits) - 1)
+            if kind == wb.WB_ID_U16:
+                return part.to(torch.int16).view(torch.bfloat16)     # raw 16-bit payload
+            return part.to(tdt)                                       # an exactly representable integer
+
+        def sink(t, x, k=k):
+            x = x.reshape(1, -1) if x.dim() == 1 else x.reshape(-1, x.shape[-1])
+            if x.dtype not in (torch.float32, torch.bfloat16):        # integer padding of the loaders
+                x = x.clamp_min(0)
+            shapes[t] = tuple(x.shape)
+            passes[t][k], n = gpu_entries(x, kind, cap=1 << 18)
+            assert n == len(passes[t][k])
+        wl.load_side_shaped(side, values, sink)
+    base = wl.ckpt_base().astype(np.uint64)
+    rows = np.array([c.rows for c in wl.ckpt], np.uint64)
+    cols = np.array([c.cols for c in wl.ckpt], np.uint64)
+    lay = Layout(side)
+    for t in range(declared.n_tensors):
+        d = declared.tensors[t]
+        lay.add_tensor(declared.names[t], int(d["rank"]), int(d["dtype"]), int(d["numel"]))
+        z = wb.wb_diff2_recombine([passes[t][k] for k in range(K)], chunk_bits)
+        for s in wb.wb_scan_slices(z, shapes[t][0], shapes[t][1], base, rows, cols, t):
+            lay.add_slice(int(s["tensor"]), int(s["local_off"]), int(s["stride_r"]), int(s["stride_c"]),
+                          int(s["ckpt"]), int(s["ckpt_rows"]), int(s["ckpt_cols"]),
+                          int(s["r0"]), int(s["c0"]), int(s["nr"]), int(s["nc"]))
+    return lay.freeze()
+
+
+@pytest.mark.parametrize("name,scale,bits", [("cfg3", "small", 16), ("cfg4", "small", 16), ("cfg4", "small", 8),
+                                              ("cfg5", "small", 16), ("cfg1b", "full", 16)])
+def test_extracted_source_maps_give_the_same_remap(name, scale, bits):
+    wl = make_workload(name, scale)
+    tl = extract_on_gpu(wl, "trainer", bits)
+    rl = extract_on_gpu(wl, "rollout", bits)
+    for lay, declared in ((tl, wl.trainer), (rl, wl.rollout)):
+        for a, b in zip(predict_ids(lay, wl), predict_ids(declared, wl)):
+            assert np.array_equal(a, b)                # same source map, element for element
+    case = DeviceCase(wl, torch.device(DEV), trainer=tl, rollout=rl)
+    want = remap_oracle(ckpt_shapes(wl), wl.trainer.tensors, wl.trainer.slices, wl.rollout.tensors,
+                        wl.rollout.slices, case.src_bits())
+    case.plan.remap()
+    torch.cuda.synchronize()
+    case.plan.check()
+    for k, got in enumerate(case.dst_bits()):
+        assert np.array_equal(got[want.written[k]], want.dst[k][want.written[k]]), wl.rollout.names[k]

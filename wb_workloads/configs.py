@@ -337,7 +337,7 @@ def trainer_fsdp(s: ModelSpec, ck, ix, W: int, dtype: int, EP: int = 0):
                 for kind in ("gate", "up", "down"):
                     def experts(ts, l=l, kind=kind):
                         stacked = torch.stack(ts, 0)                  # [E, rows, cols]
-                        return {f"t{k}.layers.{l}.{kind}_local": c.reshape(-1)
+                        return {f"t{k}.layers.{l}.{kind}_local": c
                                 for k, c in enumerate(stacked.chunk(EP, 0))}
                     yield [ix[p + f"experts.{e}.{kind}_proj"] for e in range(s.E)], experts
         yield [ix["final_norm"], ix["lm_head"]], unit("final")
@@ -557,7 +557,7 @@ def stress_workload(n_tensors: int, dim_lo: int, dim_ratio: float, cap_bytes: in
                         ps = A.chunk(parts, 0 if kind == "row" else 1)
                         if tr:
                             ps = [p.t() for p in ps]
-                    return {f"{pre}{k}.s{i}": p.contiguous().reshape(-1) for k, p in enumerate(ps)}
+                    return {f"{pre}{k}.s{i}": p.contiguous() for k, p in enumerate(ps)}
                 yield [i], fn
         return groups
 

@@ -180,6 +180,16 @@ class Workload:
             for name, t in out.items():
                 sink(layout.index(name), t.reshape(-1))
 
+    def load_side_shaped(self, side: str, values: Callable[[int], torch.Tensor],
+                         sink: Callable[[int, torch.Tensor], None]) -> None:
+        """Like load_side, but hands over each local tensor with the shape load_weights gives it
+        (the 2-D view used by source-map extraction is [prod(shape[:-1]), shape[-1]])."""
+        layout = self.trainer if side == "trainer" else self.rollout
+        groups = self.trainer_groups if side == "trainer" else self.rollout_groups
+        for ckpt_idx, fn in groups():
+            for name, t in fn([values(i) for i in ckpt_idx]).items():
+                sink(layout.index(name), t)
+
     def load_side_to_list(self, side: str, values: Callable[[int], torch.Tensor]) -> List[torch.Tensor]:
         layout = self.trainer if side == "trainer" else self.rollout
         out: List[Optional[torch.Tensor]] = [None] * layout.n_tensors
