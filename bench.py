@@ -48,7 +48,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--grid-ctas", type=int, default=0)
-    ap.add_argument("--path", default="remap", choices=["remap", "pack_unpack"])
+    ap.add_argument("--path", default="remap", choices=["remap", "pack_unpack", "extract"])
     ap.add_argument("--static-schedule", action="store_true",
                     help="fixed per-block tile ranges instead of run-time batches")
     return ap.parse_args()
@@ -197,11 +197,69 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+def run_extract(args):
+    """--path extract: the diff2 + compaction kernel of source-map extraction over the int64 id
+    fields the trainer's load_weights produces (first loader groups, up to ~4 GB of ids)."""
+    from paper_2609_25442_b200 import binding as wb
+    from paper_2609_25442_b200.device import require_cuda
+    require_cuda()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    wl = make_workload(args.workload, args.scale)
+    fields, total = [], 0
+    for ckpt_idx, fn in wl.trainer_groups():
+        for _, t in fn([wl.ckpt_ids(i, dev) + 1 for i in ckpt_idx]).items():
+            t = (t.reshape(1, -1) if t.dim() == 1 else t.reshape(-1, t.shape[-1])).clamp_min(0).contiguous()
+            fields.append(t)
+            total += t.numel()
+        if total * 8 >= 4e9:
+            break
+    cap = 1 << 20
+    out = torch.zeros(cap * 24, dtype=torch.uint8, device=dev)
+    count = torch.zeros(1, dtype=torch.int64, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step():
+        count.zero_()
+        for f in fields:
+            wb.wb_diff2_nonzeros(f.data_ptr(), wb.WB_ID_I64, f.shape[0], f.shape[1], out.data_ptr(), cap,
+                                 count.data_ptr(), stream)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    gbs = total * 8 / (ms * 1e-3) / 1e9
+    peak = FALLBACK_HBM_GBS
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak = float(json.load(f)["hbm_gbs"])
+    except Exception:
+        pass
+    print(json.dumps({"metric": "diff2 id-field scan GB/s (int64 ids read)", "value": gbs, "unit": "GB/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "int64", "data": "synthetic",
+                      "config": {"workload": wl.name, "path": "extract", "fields": len(fields),
+                                 "elements": total, "nonzeros": int(count.item()),
+                                 "l2": "inputs_larger_than_l2"},
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                                   "frac": gbs / peak, "traffic": None, "kernel": "wb_diff2_kernel"},
+                      "gpu_launches": args.steps * len(fields)}))
+
+
 # ------------------------------------------------------------------------------------------------
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.path == "extract":
+        run_extract(args)
         return
 
     from paper_2609_25442_b200 import binding as wb

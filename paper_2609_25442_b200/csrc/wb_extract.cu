@@ -28,46 +28,90 @@ template <> __device__ __forceinline__ long long field_at<WB_ID_BF16>(const void
   return (long long)__float2ll_rn(__uint_as_float(bits));
 }
 
-// One thread per element, grid-stride over the row-major field.  A thread reads the 3x3 causal
-// neighbourhood (the neighbours are L1/L2 hits: DRAM sees every element about once) and, if the
-// stencil is non-zero, takes a slot in the output list; slots are claimed once per warp.
+// A warp task is a strip of kStrip = 32*kV columns marched down up to kRowsPerTask rows.  Lane l
+// owns columns c0 + l + 32 k (k < kV), so each of its kV loads per row is a fully coalesced warp
+// access and all kV are in flight together.  The two values to the left of a column come from
+// lanes l-1 and l-2 by shuffle (from the previous k for lanes 0 and 1; from memory at the strip's
+// left edge), and the horizontal second difference h(i,j) = A(i,j) - 2 A(i,j-1) + A(i,j-2) of the
+// two rows above stays in registers, so diff2(i,j) = h(i,j) - 2 h(i-1,j) + h(i-2,j) costs one
+// global load per element (plus two halo rows per task).  Non-zeros are rare: a warp vote skips
+// the compaction for almost every row.
+constexpr int kRowsPerTask = 64;
+constexpr int kV = 8;
+constexpr int kStrip = 32 * kV;
+
+template <int KIND>
+__device__ __forceinline__ void row_h(const void* field, unsigned long long row_base, unsigned long long cols,
+                                      unsigned long long c0, unsigned lane, long long h[kV]) {
+  long long a[kV];
+#pragma unroll
+  for (int k = 0; k < kV; ++k) {
+    const unsigned long long c = c0 + lane + 32u * k;
+    a[k] = c < cols ? field_at<KIND>(field, row_base + c) : 0;
+  }
+  // halo: the two columns left of the strip (read by lanes 0 and 1, both end up needing them)
+  long long e1 = 0, e2 = 0;                                  // A[c0-1], A[c0-2]
+  if (lane < 2) {
+    if (c0 >= 1) e1 = field_at<KIND>(field, row_base + c0 - 1);
+    if (c0 >= 2) e2 = field_at<KIND>(field, row_base + c0 - 2);
+  }
+  long long prev30 = e2, prev31 = e1;                          // "lanes 30 / 31 of k-1"; uniform per warp below
+  prev30 = __shfl_sync(0xFFFFFFFFu, prev30, 0);
+  prev31 = __shfl_sync(0xFFFFFFFFu, prev31, 0);
+#pragma unroll
+  for (int k = 0; k < kV; ++k) {
+    long long l1 = __shfl_up_sync(0xFFFFFFFFu, a[k], 1), l2 = __shfl_up_sync(0xFFFFFFFFu, a[k], 2);
+    if (lane == 0) { l1 = prev31; l2 = prev30; }
+    if (lane == 1) l2 = prev31;
+    h[k] = a[k] - 2 * l1 + l2;
+    prev30 = __shfl_sync(0xFFFFFFFFu, a[k], 30);
+    prev31 = __shfl_sync(0xFFFFFFFFu, a[k], 31);
+  }
+}
+
 template <int KIND>
 __global__ void __launch_bounds__(256)
 wb_diff2_kernel(const void* __restrict__ field, unsigned long long rows, unsigned long long cols,
                 wb_diff2_entry* __restrict__ out, unsigned long long cap, unsigned long long* __restrict__ count) {
-  const unsigned long long n = rows * cols;
-  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned lane = threadIdx.x & 31;
-  // whole warps iterate together so that the ballot below always has all lanes
-  for (unsigned long long base = (unsigned long long)blockIdx.x * blockDim.x + (threadIdx.x & ~31u); base < n;
-       base += stride) {
-    const unsigned long long e = base + lane;
-    long long d = 0;
-    unsigned long long i = 0, j = 0;
-    if (e < n) {
-      i = e / cols;
-      j = e - i * cols;
-      long long acc[3] = {0, 0, 0};       // [1,-2,1] along j for rows i, i-1, i-2
+  const unsigned long long strips = (cols + kStrip - 1) / kStrip, blocks = (rows + kRowsPerTask - 1) / kRowsPerTask;
+  const unsigned long long n_tasks = strips * blocks;
+  const unsigned long long warp0 = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const unsigned long long n_warps = ((unsigned long long)gridDim.x * blockDim.x) >> 5;
+  for (unsigned long long task = warp0; task < n_tasks; task += n_warps) {
+    const unsigned long long rb = task / strips, cs = task - rb * strips;   // neighbouring warps: neighbouring strips
+    const unsigned long long i0 = rb * kRowsPerTask;
+    const unsigned long long i1 = i0 + kRowsPerTask < rows ? i0 + kRowsPerTask : rows;
+    const unsigned long long c0 = cs * kStrip;
+    long long hm1[kV], hm2[kV];
 #pragma unroll
-      for (int a = 0; a < 3; ++a) {
-        if (i >= (unsigned long long)a) {
-          const unsigned long long r = e - (unsigned long long)a * cols;
-          long long v = field_at<KIND>(field, r);
-          if (j >= 1) v -= 2 * field_at<KIND>(field, r - 1);
-          if (j >= 2) v += field_at<KIND>(field, r - 2);
-          acc[a] = v;
-        }
+    for (int k = 0; k < kV; ++k) hm1[k] = hm2[k] = 0;
+    if (i0 >= 2) row_h<KIND>(field, (i0 - 2) * cols, cols, c0, lane, hm2);
+    if (i0 >= 1) row_h<KIND>(field, (i0 - 1) * cols, cols, c0, lane, hm1);
+    for (unsigned long long i = i0; i < i1; ++i) {
+      long long h[kV], d[kV];
+      row_h<KIND>(field, i * cols, cols, c0, lane, h);
+      long long any = 0;
+#pragma unroll
+      for (int k = 0; k < kV; ++k) {
+        d[k] = (c0 + lane + 32u * k < cols) ? h[k] - 2 * hm1[k] + hm2[k] : 0;
+        hm2[k] = hm1[k];
+        hm1[k] = h[k];
+        any |= d[k];
       }
-      d = acc[0] - 2 * acc[1] + acc[2];
-    }
-    const unsigned mask = __ballot_sync(0xFFFFFFFFu, d != 0);
-    if (mask) {
-      unsigned long long slot0 = 0;
-      if (lane == 0) slot0 = atomicAdd(count, (unsigned long long)__popc(mask));
-      slot0 = __shfl_sync(0xFFFFFFFFu, slot0, 0);
-      if (d != 0) {
-        const unsigned long long slot = slot0 + __popc(mask & ((1u << lane) - 1));
-        if (slot < cap) out[slot] = wb_diff2_entry{i, j, d};
+      if (__any_sync(0xFFFFFFFFu, any != 0)) {
+#pragma unroll
+        for (int k = 0; k < kV; ++k) {
+          const unsigned mask = __ballot_sync(0xFFFFFFFFu, d[k] != 0);
+          if (!mask) continue;
+          unsigned long long slot0 = 0;
+          if (lane == 0) slot0 = atomicAdd(count, (unsigned long long)__popc(mask));
+          slot0 = __shfl_sync(0xFFFFFFFFu, slot0, 0);
+          if (d[k] != 0) {
+            const unsigned long long slot = slot0 + __popc(mask & ((1u << lane) - 1));
+            if (slot < cap) out[slot] = wb_diff2_entry{i, c0 + lane + 32u * k, d[k]};
+          }
+        }
       }
     }
   }
@@ -81,9 +125,9 @@ extern "C" wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint
   if (rows == 0 || cols == 0) return WB_OK;
   if (rows > (1ull << 40) || cols > (1ull << 40) || rows * cols > (1ull << 48)) return WB_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const unsigned long long n = rows * cols;
-  const unsigned long long want = (n + 255) / 256;
-  const unsigned grid = (unsigned)(want < 148ull * 16 ? want : 148ull * 16);
+  const unsigned long long tasks = ((cols + kStrip - 1) / kStrip) * ((rows + kRowsPerTask - 1) / kRowsPerTask);
+  const unsigned long long want = (tasks + 7) / 8;                 // 8 warps per block
+  const unsigned grid = (unsigned)(want < 148ull * 8 ? want : 148ull * 8);
   auto* cnt = reinterpret_cast<unsigned long long*>(count);
   switch (id_kind) {
     case WB_ID_I64: wb_diff2_kernel<WB_ID_I64><<<grid, 256, 0, stream>>>(field, rows, cols, out, cap, cnt); break;
