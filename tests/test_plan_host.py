@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol():
     lib = wb.load()
     header = open(os.path.join(ROOT, "include", "wb.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(wb_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(wb_[a-z0-9_]+)\s*\(", header))
     assert {"wb_layout_describe", "wb_plan_build", "wb_pack", "wb_unpack", "wb_remap"} <= declared
     for name in declared:
         assert hasattr(lib, name), name
