@@ -265,16 +265,12 @@ def main():
     from paper_2609_25442_b200 import binding as wb
     from paper_2609_25442_b200.device import RankArenas, bind, require_cuda
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2609_25442_b200 import dist as wbdist
+    rank, local_rank, world = wbdist.rank_info()
     require_cuda()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    dist = wbdist.init("nccl", dev)
 
     # ---- inputs: resident in HBM before the timed region -------------------------------------
     wl = make_workload(args.workload, args.scale)
@@ -310,9 +306,7 @@ def main():
         return 2 * n_rounds
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
+        wbdist.barrier(dist, cuda=True)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -332,12 +326,9 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     total_ms = evs[0].elapsed_time(evs[-1])
     per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = wbdist.max_over_ranks(dist, total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * bytes_step / (ms_per_step * 1e-3) / 1e9
+    value = wbdist.aggregate_gbs(world, bytes_step, ms_per_step)
 
     # ---- roofline of the dominant (only) kernel --------------------------------------------------
     peak, peak_src = FALLBACK_HBM_GBS, "fallback"
@@ -380,12 +371,8 @@ def main():
         b.record()
         barrier()
         e_ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e_ms /= args.e2e_steps
-        e2e = {"value": world * bytes_step / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+        e_ms = wbdist.max_over_ranks(dist, e_ms, dev) / args.e2e_steps
+        e2e = {"value": wbdist.aggregate_gbs(world, bytes_step, e_ms), "unit": UNIT,
                "h2d_bytes_per_step": src.total_bytes(), "d2h_bytes_per_step": dst.total_bytes(),
                "ms_per_step": e_ms, "steps": args.e2e_steps, "pinned": pinned}
         del host_src, host_dst
