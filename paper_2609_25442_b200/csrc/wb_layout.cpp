@@ -50,9 +50,9 @@ static wb_status normalise(const wb_slice& s, const wb_tensor_desc& t, NSlice* o
   } else {
     return WB_ERR_INVALID_ARG;
   }
-  if (pitch >= (1ull << 32)) return WB_ERR_INVALID_ARG;
   // last element touched
   const uint64_t outer = transposed ? nc : nr, inner = transposed ? nr : nc;
+  if (outer > 1 && pitch >= (1ull << 32)) return WB_ERR_INVALID_ARG;   // a single run has no pitch
   // overflow-safe: outer, pitch < 2^63 / numel checks below
   const unsigned __int128 last = (unsigned __int128)s.local_off +
                                  (unsigned __int128)(outer - 1) * pitch + (inner - 1);

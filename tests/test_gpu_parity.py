@@ -228,3 +228,68 @@ def test_remap_from_host_buffers(device):
     torch.cuda.synchronize()
     for k, t in enumerate(host_dst):
         assert np.array_equal(to_bits(t), want.dst[k])
+
+
+def test_empty_layouts_launch_nothing(device):
+    tl, rl = Layout("t"), Layout("r")
+    tl.add_tensor("T", 0, WB_F32, 16)
+    rl.add_tensor("R", 0, WB_BF16, 16)
+    tl.freeze(); rl.freeze()
+    plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices))
+    plan.verify()
+    st = plan.stats()
+    assert st["n_tiles_remap"] == 0 and st["src_elems_read"] == 0 and plan.num_rounds() == 1
+    src = RankArenas(tl.tensors, device, fill_byte=1)
+    dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+    bind(plan, src, dst)
+    plan.remap()
+    bucket = torch.zeros(64, dtype=torch.uint8, device=device)
+    plan.pack(0, bucket.data_ptr())
+    plan.unpack(0, bucket.data_ptr())
+    torch.cuda.synchronize()
+    plan.check()
+    assert (to_bits(dst.tensors[0]) == 0xCDCD).all()
+
+
+def test_offsets_beyond_32_bits(device):
+    """One tensor of 4.4 G elements (8.8 GB a side): element offsets, tile counts and bucket offsets
+    need 64 bits.  Trainer: two flat shards; rollout: one tensor, so slabs start deep inside."""
+    n = (1 << 32) + 123_456_789
+    if torch.cuda.mem_get_info()[0] < 2 * 2 * n + (8 << 30):
+        pytest.skip("needs ~26 GB of free device memory")
+    half = n // 2 + 7
+    tl, rl = Layout("t"), Layout("r")
+    tl.add_tensor("T0", 0, WB_BF16, half)
+    tl.add_tensor("T1", 1, WB_BF16, n - half)
+    rl.add_tensor("R", 0, WB_BF16, n)
+    tl.add_slice(0, 0, n, 1, 0, 1, n, 0, 0, 1, half)
+    tl.add_slice(1, 0, n, 1, 0, 1, n, 0, half, 1, n - half)
+    rl.add_slice(0, 0, n, 1, 0, 1, n, 0, 0, 1, n)
+    tl.freeze(); rl.freeze()
+    plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices))
+    plan.verify()
+    assert plan.stats()["src_elems_read"] == n and plan.num_rounds() >= 3
+    src = RankArenas(tl.tensors, device)
+    dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+    g = torch.Generator(device=device); g.manual_seed(3)
+    for t in src.tensors:                       # random 16-bit patterns, generated in pieces
+        v = t.view(torch.int16)
+        for a in range(0, v.numel(), 1 << 28):
+            b = min(a + (1 << 28), v.numel())
+            v[a:b] = torch.randint(-32768, 32767, (b - a,), dtype=torch.int16, device=device, generator=g)
+    bind(plan, src, dst)
+    plan.remap()
+    torch.cuda.synchronize()
+    out = dst.tensors[0].view(torch.int16)
+    assert torch.equal(out[:half], src.tensors[0].view(torch.int16))
+    assert torch.equal(out[half:], src.tensors[1].view(torch.int16))
+    # the two-pass path over the same range
+    dst.arenas[0].fill_(CANARY)
+    bucket = torch.empty(max(plan.bucket_bytes(r) for r in range(plan.num_rounds())), dtype=torch.uint8, device=device)
+    for r in range(plan.num_rounds()):
+        plan.pack(r, bucket.data_ptr())
+        plan.unpack(r, bucket.data_ptr())
+    torch.cuda.synchronize()
+    plan.check()
+    assert torch.equal(out[:half], src.tensors[0].view(torch.int16))
+    assert torch.equal(out[half:], src.tensors[1].view(torch.int16))
