@@ -466,83 +466,111 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
   using E = Elem<ES, ED>;
   constexpr uint32_t NV = 16 / ED;
   constexpr uint32_t PER_WORD = 4 / ED;                     // destination elements per 32-bit word
+  constexpr int UA = 16;                                    // rows per batch of loads
   // rows per block: as many as the warp's share of the slot allows (multiple of 8, at most 64)
   const uint32_t share = scratch_bytes / kWorkerWarps / 4;  // words
-  uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD) & ~7u);
+  const uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD) & ~7u);
   const uint32_t pitch_w = rb / PER_WORD + 1;               // odd: rb/PER_WORD is even
   uint32_t* T = reinterpret_cast<uint32_t*>(scratch) + warp * (32 * pitch_w);
   const uint32_t tbase = smem_u32(T);
   const uint32_t nbi = (f.nr + rb - 1) / rb, nbj = (f.nc + 31) / 32;
-  for (uint32_t b = warp; b < nbi * nbj; b += kWorkerWarps) {
+  const uint32_t nb = nbi * nbj;
+  const size_t sps = (size_t)f.ssr * ES;
+  if (warp >= nb) return;
+
+  struct Block { uint32_t i0, j0, ni, nj; };
+  auto block_of = [&](uint32_t b) {
     const uint32_t bi = b / nbj, bj = b - bi * nbj;
-    const uint32_t i0 = bi * rb, j0 = bj * 32;
-    const uint32_t ni = min(rb, f.nr - i0), nj = min(32u, f.nc - j0);
-    // ---- phase A
-    if (lane < nj) {
-      const char* src = f.s + ((size_t)i0 * f.ssr + j0 + lane) * ES;
-      const size_t sps = (size_t)f.ssr * ES;
-      const uint32_t trow = tbase + lane * pitch_w * 4;
-      constexpr int UA = 16;                                  // loads in flight per lane
-      for (uint32_t r0 = 0; r0 < ni; r0 += UA) {
-        uint32_t raw[UA];
+    return Block{bi * rb, bj * 32, min(rb, f.nr - bi * rb), min(32u, f.nc - bj * 32)};
+  };
+  // phase A, loads: UA rows of this lane's column into registers
+  auto issue = [&](const Block& k, uint32_t r0, uint32_t (&dst)[UA]) {
+    const char* src = f.s + ((size_t)(k.i0 + r0) * f.ssr + k.j0 + lane) * ES;
 #pragma unroll
-        for (int u = 0; u < UA; ++u) {
-          raw[u] = 0;
-          if (r0 + u < ni) {
-            if constexpr (ES == 4) raw[u] = __ldcs(reinterpret_cast<const uint32_t*>(src + (size_t)(r0 + u) * sps));
-            else raw[u] = __ldcs(reinterpret_cast<const uint16_t*>(src + (size_t)(r0 + u) * sps));
-          }
-        }
-        if constexpr (ED == 2) {
-#pragma unroll
-          for (int u = 0; u < UA; u += 2)
-            if (r0 + u < ni)
-              asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 2), "r"(pack_pair16<ES>(raw[u], raw[u + 1])));
-        } else {
-#pragma unroll
-          for (int u = 0; u < UA; ++u)
-            if (r0 + u < ni)
-              asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 4), "r"((uint32_t)cast_raw<ES, ED>(raw[u])));
-        }
+    for (int u = 0; u < UA; ++u) {
+      dst[u] = 0;
+      if (lane < k.nj && r0 + u < k.ni) {
+        if constexpr (ES == 4) dst[u] = __ldcs(reinterpret_cast<const uint32_t*>(src + (size_t)u * sps));
+        else dst[u] = __ldcs(reinterpret_cast<const uint16_t*>(src + (size_t)u * sps));
       }
     }
+  };
+  // phase A, stores: cast and write into the patch as destination row `lane`
+  auto consume = [&](const Block& k, uint32_t r0, const uint32_t (&v)[UA]) {
+    if (lane >= k.nj) return;
+    const uint32_t trow = tbase + lane * pitch_w * 4;
+    if constexpr (ED == 2) {
+#pragma unroll
+      for (int u = 0; u < UA; u += 2)
+        if (r0 + u < k.ni)
+          asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 2), "r"(pack_pair16<ES>(v[u], v[u + 1])));
+    } else {
+#pragma unroll
+      for (int u = 0; u < UA; ++u)
+        if (r0 + u < k.ni)
+          asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 4), "r"((uint32_t)cast_raw<ES, ED>(v[u])));
+    }
+  };
+  // phase B: every destination run of the block in 16-byte aligned slots
+  auto phase_b = [&](const Block& k) {
     __syncwarp();
-    // ---- phase B
-    {
-      const uint32_t smax = (ni + 2 * NV - 2) / NV;             // slots a row can touch
-      for (uint32_t task = lane; task < nj * smax; task += 32) {
-        const uint32_t k = task / nj, j = task - k * nj;         // consecutive lanes: consecutive rows
-        char* out = f.d + ((size_t)(j0 + j) * f.dsc + i0) * ED;   // first element of this run
-        const uint32_t a = (uint32_t)((uintptr_t)out & 15u) / ED;
-        const int32_t e0 = (int32_t)(k * NV) - (int32_t)a;
-        if (e0 >= (int32_t)ni) continue;
-        const uint32_t trow = tbase + j * pitch_w * 4;
-        if (e0 >= 0 && (uint32_t)e0 + NV <= ni) {
-          uint4 x;
-          if constexpr (ED == 4) {
-            x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
-            x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
+    const uint32_t smax = (k.ni + 2 * NV - 2) / NV;             // slots a run can touch
+    for (uint32_t task = lane; task < k.nj * smax; task += 32) {
+      const uint32_t s = task / k.nj, j = task - s * k.nj;        // consecutive lanes: consecutive runs
+      char* out = f.d + ((size_t)(k.j0 + j) * f.dsc + k.i0) * ED;
+      const uint32_t a = (uint32_t)((uintptr_t)out & 15u) / ED;
+      const int32_t e0 = (int32_t)(s * NV) - (int32_t)a;
+      if (e0 >= (int32_t)k.ni) continue;
+      const uint32_t trow = tbase + j * pitch_w * 4;
+      if (e0 >= 0 && (uint32_t)e0 + NV <= k.ni) {
+        uint4 x;
+        if constexpr (ED == 4) {
+          x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
+          x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
+        } else {
+          const uint32_t w = trow + ((uint32_t)e0 >> 1) * 4;
+          const uint32_t w0 = lds_raw<4>(w), w1 = lds_raw<4>(w + 4), w2 = lds_raw<4>(w + 8), w3 = lds_raw<4>(w + 12);
+          if (e0 & 1) {
+            const uint32_t w4 = lds_raw<4>(w + 16);
+            x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
+                           __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
           } else {
-            const uint32_t w = trow + ((uint32_t)e0 >> 1) * 4;
-            const uint32_t w0 = lds_raw<4>(w), w1 = lds_raw<4>(w + 4), w2 = lds_raw<4>(w + 8), w3 = lds_raw<4>(w + 12);
-            if (e0 & 1) {
-              const uint32_t w4 = lds_raw<4>(w + 16);
-              x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
-                             __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
-            } else {
-              x = make_uint4(w0, w1, w2, w3);
-            }
+            x = make_uint4(w0, w1, w2, w3);
           }
-          st16(reinterpret_cast<char*>(((uintptr_t)out & ~(uintptr_t)15) + 16u * k), x);
-        } else {
-          const uint32_t lo = e0 < 0 ? 0u : (uint32_t)e0;
-          const uint32_t hi = min(ni, (uint32_t)(e0 + (int32_t)NV));
-          for (uint32_t e = lo; e < hi; ++e)
-            E::store(out + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
         }
+        st16(reinterpret_cast<char*>(((uintptr_t)out & ~(uintptr_t)15) + 16u * s), x);
+      } else {
+        const uint32_t lo = e0 < 0 ? 0u : (uint32_t)e0;
+        const uint32_t hi = min(k.ni, (uint32_t)(e0 + (int32_t)NV));
+        for (uint32_t e = lo; e < hi; ++e)
+          E::store(out + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
       }
     }
     __syncwarp();
+  };
+
+  // The warp's batches in order; the loads of batch q+1 are issued before batch q is consumed, so
+  // they are in flight during the shared-memory writes and during phase B.
+  uint32_t b = warp, r0 = 0;
+  Block blk = block_of(b);
+  auto step = [&](uint32_t (&cur)[UA], uint32_t (&nxt)[UA]) -> bool {
+    uint32_t b2 = b, r2 = r0 + UA;
+    Block blk2 = blk;
+    const bool same = r2 < blk.ni;
+    if (!same) { b2 = b + kWorkerWarps; r2 = 0; }
+    const bool more = same || b2 < nb;
+    if (!same && more) blk2 = block_of(b2);
+    if (more) issue(blk2, r2, nxt);
+    consume(blk, r0, cur);
+    if (!same) phase_b(blk);
+    b = b2; r0 = r2; blk = blk2;
+    return more;
+  };
+  uint32_t bufa[UA], bufb[UA];
+  issue(blk, 0, bufa);
+  for (;;) {
+    if (!step(bufa, bufb)) break;
+    if (!step(bufb, bufa)) break;
   }
 }
 
