@@ -283,6 +283,37 @@ wb_status wb_remap_host(const wb_plan* plan, const void* const* host_src, size_t
 wb_status wb_remap_static(const wb_plan* plan, const void* const* src_base, size_t n_src,
                           void* const* dst_base, size_t n_dst, uint32_t flags, void* cuda_stream);
 
+/* ---- three-stage routing over nodes: traffic accounting (Section 3.2, Eq. 1) ------------------
+ * With virtual ranks placed on nodes, a plan's slabs define the paper's three stages: *receive*
+ * (each slab travels from its trainer rank to its designated rollout rank -- replicas of a tensor
+ * are the designated receivers of distinct slices), *external exchange* (every other rollout node
+ * that needs the slab gets it once, over RDMA, from the designated receiver) and *internal
+ * exchange* (the remaining ranks of a node copy it over NVLink).  Nothing is moved: this returns
+ * the byte counts the stages would carry, to check the plan against the paper's traffic claims --
+ * trainers send exactly one model copy M, node v receives exactly its de-duplicated volume M_v over
+ * RDMA -- and the lower bound T_min = max(M / B_T, max_v M_v / B_v) of Eq. 1.
+ * Bytes are destination-dtype bytes (wb_pack casts before the wire). */
+typedef struct {
+  uint64_t model_bytes;            /* M: every consumed checkpoint element once                    */
+  uint64_t receive_bytes;          /* stage 1, trainers -> designated receivers                    */
+  uint64_t external_bytes;         /* stage 2, between rollout nodes (RDMA)                        */
+  uint64_t internal_bytes;         /* stage 3, inside rollout nodes (NVLink)                       */
+  uint64_t direct_rdma_bytes;      /* without the exchange stages: every rank pulls all it needs   */
+  uint64_t max_trainer_rank_egress;
+  uint64_t max_rollout_rank_rdma_ingress;
+  uint64_t max_node_rdma_ingress;
+  double   t_min_seconds;          /* Eq. 1 with the bandwidths given                              */
+} wb_route_stats_t;
+/* trainer_node[r] / rollout_node[r]: node of virtual trainer / rollout rank r (host arrays; node ids
+ * are small integers, trainer and rollout nodes share one numbering).  trainer_gbs = aggregate
+ * trainer egress bandwidth B_T, node_gbs = ingress bandwidth B_v of a rollout node, in GB/s.
+ * node_rdma_ingress / node_required (host, n_nodes entries each, may be NULL) receive, per node, the
+ * RDMA bytes entering it in stages 1+2 and M_v.  Errors: INVALID_ARG. */
+wb_status wb_route_account(const wb_plan* plan, const uint32_t* trainer_node, size_t n_trainer_ranks,
+                           const uint32_t* rollout_node, size_t n_rollout_ranks, double trainer_gbs,
+                           double node_gbs, wb_route_stats_t* out, uint64_t* node_rdma_ingress,
+                           uint64_t* node_required, size_t n_nodes);
+
 /* ---- source-map extraction (Section 3.1, Appendix B / Algorithm 1) ---------------------------
  * A worker's source map can be recovered from its black-box load_weights instead of being
  * written by hand: fill the checkpoint with position ids (1-based, so 0 = "no source"), load,

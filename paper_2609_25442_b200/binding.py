@@ -79,7 +79,7 @@ EXPORTS = [
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
     "wb_remap_host", "wb_remap_static", "wb_plan_check",
-    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -119,6 +119,7 @@ def load() -> C.CDLL:
     lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
     lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
+    lib.wb_route_account.argtypes = [vp, vp, sz, vp, sz, C.c_double, C.c_double, vp, vp, vp, sz]
     lib.wb_diff2_nonzeros.argtypes = [vp, C.c_uint32, C.c_uint64, C.c_uint64, vp, C.c_uint64, vp, vp]
     lib.wb_diff2_recombine.argtypes = [vp, vp, sz, C.c_uint32, vp, sz, C.POINTER(sz)]
     lib.wb_scan_slices.argtypes = [vp, sz, C.c_uint64, C.c_uint64, vp, vp, vp, sz, C.c_uint32, C.c_uint64,
@@ -317,3 +318,26 @@ def wb_scan_slices(entries: np.ndarray, rows: int, cols: int, ckpt_base: np.ndar
     out = np.zeros(n.value, SLICE_DTYPE)
     _check(_lib.wb_scan_slices(*args, out.ctypes.data, n.value, C.byref(n)), "wb_scan_slices")
     return out
+
+
+# ---- three-stage routing, traffic accounting ---------------------------------------------------------
+class wb_route_stats_t(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in (
+        "model_bytes", "receive_bytes", "external_bytes", "internal_bytes", "direct_rdma_bytes",
+        "max_trainer_rank_egress", "max_rollout_rank_rdma_ingress", "max_node_rdma_ingress")] + \
+        [("t_min_seconds", C.c_double)]
+
+
+def wb_route_account(plan: Plan, trainer_node: Sequence[int], rollout_node: Sequence[int], n_nodes: int,
+                     trainer_gbs: float = 0.0, node_gbs: float = 0.0):
+    """Returns (stats dict, per-node RDMA ingress, per-node required bytes M_v)."""
+    load()
+    tn = np.ascontiguousarray(trainer_node, dtype=np.uint32)
+    rn = np.ascontiguousarray(rollout_node, dtype=np.uint32)
+    st = wb_route_stats_t()
+    ing = np.zeros(n_nodes, np.uint64)
+    req = np.zeros(n_nodes, np.uint64)
+    _check(_lib.wb_route_account(plan.handle, tn.ctypes.data, len(tn), rn.ctypes.data, len(rn), trainer_gbs,
+                                 node_gbs, C.byref(st), ing.ctypes.data, req.ctypes.data, n_nodes),
+           "wb_route_account")
+    return {n: getattr(st, n) for n, _ in st._fields_}, ing, req

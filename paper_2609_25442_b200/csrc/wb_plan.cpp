@@ -766,3 +766,78 @@ extern "C" wb_status wb_plan_verify(const wb_plan* plan) {
   }
   return WB_OK;
 }
+
+
+// =================================================================================================
+// Three-stage routing, traffic accounting (Section 3.2).
+extern "C" wb_status wb_route_account(const wb_plan* plan, const uint32_t* trainer_node, size_t n_trainer_ranks,
+                                      const uint32_t* rollout_node, size_t n_rollout_ranks, double trainer_gbs,
+                                      double node_gbs, wb_route_stats_t* out, uint64_t* node_rdma_ingress,
+                                      uint64_t* node_required, size_t n_nodes) {
+  if (!plan || !trainer_node || !rollout_node || !out || n_nodes == 0) return WB_ERR_INVALID_ARG;
+  if (n_trainer_ranks < plan->egress.size() || n_rollout_ranks < plan->ingress.size()) return WB_ERR_INVALID_ARG;
+  for (size_t r = 0; r < n_trainer_ranks; ++r) if (trainer_node[r] >= n_nodes) return WB_ERR_INVALID_ARG;
+  for (size_t r = 0; r < n_rollout_ranks; ++r) if (rollout_node[r] >= n_nodes) return WB_ERR_INVALID_ARG;
+  try {
+    const uint64_t ed = plan->dst.dtype == WB_F32 ? 4 : 2;
+    wb_route_stats_t st{};
+    std::vector<uint64_t> t_egress(n_trainer_ranks, 0), r_rdma(n_rollout_ranks, 0);
+    std::vector<uint64_t> node_in(n_nodes, 0), node_req(n_nodes, 0);
+    std::vector<uint32_t> nodes, per_node;
+    for (const Slab& sl : plan->slabs) {
+      const uint64_t bytes = sl.rect.area() * ed;
+      st.model_bytes += bytes;
+      // stage 1: trainer rank -> designated receiver
+      st.receive_bytes += bytes;
+      t_egress[sl.sender] += bytes;
+      const uint32_t home = rollout_node[sl.receiver];
+      if (trainer_node[sl.sender] != home) { r_rdma[sl.receiver] += bytes; node_in[home] += bytes; }
+      // the rollout nodes that need this slab, and how many of their ranks do
+      nodes.clear(); per_node.clear();
+      for (uint32_t d = 0; d < sl.dst_count; ++d) {
+        const uint32_t rank = plan->dst.tensors[plan->dst.slices[plan->slab_dsts[sl.dst_begin + d]].tensor].rank;
+        const uint32_t nd = rollout_node[rank];
+        size_t k = 0;
+        while (k < nodes.size() && nodes[k] != nd) ++k;
+        if (k == nodes.size()) { nodes.push_back(nd); per_node.push_back(0); }
+        per_node[k]++;
+        // without exchange stages every rank pulls the slab itself
+        if (trainer_node[sl.sender] != nd) st.direct_rdma_bytes += bytes;
+      }
+      for (size_t k = 0; k < nodes.size(); ++k) {
+        node_req[nodes[k]] += bytes;
+        if (nodes[k] != home) {               // stage 2: once into every other node that needs it
+          st.external_bytes += bytes;
+          node_in[nodes[k]] += bytes;
+          // the designated receiver's counterpart takes it: the destination rank of that node
+          // with the same position (in rank order) as the receiver has in its own node
+          uint32_t pos = 0;
+          std::vector<uint32_t> there;
+          for (uint32_t d = 0; d < sl.dst_count; ++d) {
+            const uint32_t rank = plan->dst.tensors[plan->dst.slices[plan->slab_dsts[sl.dst_begin + d]].tensor].rank;
+            if (rollout_node[rank] == nodes[k]) there.push_back(rank);
+            if (rollout_node[rank] == home && rank < sl.receiver) ++pos;
+          }
+          std::sort(there.begin(), there.end());
+          r_rdma[there[pos % there.size()]] += bytes;
+        }
+        st.internal_bytes += bytes * (per_node[k] - 1);   // stage 3: the node's other ranks
+      }
+    }
+    for (uint64_t v : t_egress) st.max_trainer_rank_egress = std::max(st.max_trainer_rank_egress, v);
+    for (uint64_t v : r_rdma) st.max_rollout_rank_rdma_ingress = std::max(st.max_rollout_rank_rdma_ingress, v);
+    double worst = 0;
+    for (size_t v = 0; v < n_nodes; ++v) {
+      st.max_node_rdma_ingress = std::max(st.max_node_rdma_ingress, node_in[v]);
+      if (node_gbs > 0) worst = std::max(worst, node_req[v] / (node_gbs * 1e9));
+      if (node_rdma_ingress) node_rdma_ingress[v] = node_in[v];
+      if (node_required) node_required[v] = node_req[v];
+    }
+    if (trainer_gbs > 0) worst = std::max(worst, st.model_bytes / (trainer_gbs * 1e9));
+    st.t_min_seconds = worst;
+    *out = st;
+  } catch (const std::bad_alloc&) {
+    return WB_ERR_OOM;
+  }
+  return WB_OK;
+}
