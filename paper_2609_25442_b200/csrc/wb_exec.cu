@@ -454,11 +454,14 @@ template <int ES> __device__ __forceinline__ uint32_t pack_pair16(uint32_t lo, u
 // Workers: transposing tile, dst[j*dsc + i] = cast(src[i*ssr + j]).  No block-wide step: every
 // warp takes 32-column x RB-row blocks of the tile on its own.
 //   phase A  lane = source column.  The warp reads row after row (32 consecutive elements per
-//            load instruction, 16 loads in flight per lane), casts, and writes each value into
-//            its private patch of the ring slot, laid out as destination rows: T[lane][row].
-//   phase B  lane = destination row.  Each row (RB elements, any 2-/4-byte alignment in global
-//            memory) is cut into 16-byte aligned slots: full slots are one vector store assembled
-//            from shared memory with funnel shifts, ragged end slots are element stores.
+//            load instruction, 16 loads in flight per lane, one batch ahead), casts, and writes
+//            each value into its private patch of the ring slot, laid out as destination rows:
+//            T[lane][row].
+//   phase B  lane = destination run.  A run may start at any 2-/4-byte alignment in global memory;
+//            it is written in 16-byte aligned windows.  A block owns the windows that START in its
+//            rows and reads up to NV-1 rows past its end to complete the last one, so neighbouring
+//            blocks never share a window and almost every store is a full vector; only the two
+//            ends of a whole run use element stores.
 // The patch pitch is odd in 32-bit words, so lanes hit distinct banks in both phases.
 template <int ES, int ED>
 __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratch, uint32_t scratch_bytes,
@@ -467,10 +470,13 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
   constexpr uint32_t NV = 16 / ED;
   constexpr uint32_t PER_WORD = 4 / ED;                     // destination elements per 32-bit word
   constexpr int UA = 16;                                    // rows per batch of loads
-  // rows per block: as many as the warp's share of the slot allows (multiple of 8, at most 64)
+  // rows per block: as many as the warp's share of the slot allows next to the NV-1 halo rows
+  // (multiple of 8, at most 64); no halo is needed when every run starts on a 16-byte boundary
   const uint32_t share = scratch_bytes / kWorkerWarps / 4;  // words
-  const uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD) & ~7u);
-  const uint32_t pitch_w = rb / PER_WORD + 1;               // odd: rb/PER_WORD is even
+  const bool aligned = (((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0;
+  const uint32_t halo = aligned ? 0u : NV - 1, room = aligned ? 0u : 8u;
+  const uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD - room) & ~7u);
+  const uint32_t pitch_w = (rb + room) / PER_WORD + 1;      // odd: (rb+room)/PER_WORD is even
   uint32_t* T = reinterpret_cast<uint32_t*>(scratch) + warp * (32 * pitch_w);
   const uint32_t tbase = smem_u32(T);
   const uint32_t nbi = (f.nr + rb - 1) / rb, nbj = (f.nc + 31) / 32;
@@ -478,10 +484,11 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
   const size_t sps = (size_t)f.ssr * ES;
   if (warp >= nb) return;
 
-  struct Block { uint32_t i0, j0, ni, nj; };
+  struct Block { uint32_t i0, j0, ni, nj, nl; };      // nl: rows loaded = own rows + halo
   auto block_of = [&](uint32_t b) {
     const uint32_t bi = b / nbj, bj = b - bi * nbj;
-    return Block{bi * rb, bj * 32, min(rb, f.nr - bi * rb), min(32u, f.nc - bj * 32)};
+    const uint32_t i0 = bi * rb, ni = min(rb, f.nr - i0);
+    return Block{i0, bj * 32, ni, min(32u, f.nc - bj * 32), min(ni + halo, f.nr - i0)};
   };
   // phase A, loads: UA rows of this lane's column into registers
   auto issue = [&](const Block& k, uint32_t r0, uint32_t (&dst)[UA]) {
@@ -489,7 +496,7 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
 #pragma unroll
     for (int u = 0; u < UA; ++u) {
       dst[u] = 0;
-      if (lane < k.nj && r0 + u < k.ni) {
+      if (lane < k.nj && r0 + u < k.nl) {
         if constexpr (ES == 4) dst[u] = __ldcs(reinterpret_cast<const uint32_t*>(src + (size_t)u * sps));
         else dst[u] = __ldcs(reinterpret_cast<const uint16_t*>(src + (size_t)u * sps));
       }
@@ -502,48 +509,57 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
     if constexpr (ED == 2) {
 #pragma unroll
       for (int u = 0; u < UA; u += 2)
-        if (r0 + u < k.ni)
+        if (r0 + u < k.nl)
           asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 2), "r"(pack_pair16<ES>(v[u], v[u + 1])));
     } else {
 #pragma unroll
       for (int u = 0; u < UA; ++u)
-        if (r0 + u < k.ni)
+        if (r0 + u < k.nl)
           asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 4), "r"((uint32_t)cast_raw<ES, ED>(v[u])));
     }
   };
-  // phase B: every destination run of the block in 16-byte aligned slots
+  // phase B: the 16-byte windows of every destination run that start inside the block's rows
   auto phase_b = [&](const Block& k) {
     __syncwarp();
-    const uint32_t smax = (k.ni + 2 * NV - 2) / NV;             // slots a run can touch
+    const uint32_t smax = k.ni / NV + 2;                          // windows per run, upper bound
     for (uint32_t task = lane; task < k.nj * smax; task += 32) {
-      const uint32_t s = task / k.nj, j = task - s * k.nj;        // consecutive lanes: consecutive runs
-      char* out = f.d + ((size_t)(k.j0 + j) * f.dsc + k.i0) * ED;
-      const uint32_t a = (uint32_t)((uintptr_t)out & 15u) / ED;
-      const int32_t e0 = (int32_t)(s * NV) - (int32_t)a;
-      if (e0 >= (int32_t)k.ni) continue;
+      const uint32_t w = task / k.nj, j = task - w * k.nj;        // consecutive lanes: consecutive runs
+      char* run = f.d + (size_t)(k.j0 + j) * f.dsc * ED;          // element (j, 0) of the run
+      const uint32_t a = (uint32_t)(((uintptr_t)run / ED + k.i0) & (NV - 1));   // offset of row i0 in its window
       const uint32_t trow = tbase + j * pitch_w * 4;
-      if (e0 >= 0 && (uint32_t)e0 + NV <= k.ni) {
+      if (w == 0) {
+        // rows before the first window that starts here: the previous block's window covers them,
+        // except at the very start of the run
+        const uint32_t lead = a ? NV - a : 0;
+        if (k.i0 == 0)
+          for (uint32_t e = 0; e < min(lead, k.ni); ++e)
+            E::store(run + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
+        continue;
+      }
+      const uint32_t e0 = (a ? NV - a : 0) + (w - 1) * NV;         // first row (relative to i0) of the window
+      if (e0 >= k.ni) continue;
+      char* out = run + (size_t)(k.i0 + e0) * ED;                 // 16-byte aligned
+      if (e0 + NV <= k.nl) {
         uint4 x;
         if constexpr (ED == 4) {
           x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
           x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
         } else {
-          const uint32_t w = trow + ((uint32_t)e0 >> 1) * 4;
-          const uint32_t w0 = lds_raw<4>(w), w1 = lds_raw<4>(w + 4), w2 = lds_raw<4>(w + 8), w3 = lds_raw<4>(w + 12);
+          const uint32_t p = trow + (e0 >> 1) * 4;
+          const uint32_t w0 = lds_raw<4>(p), w1 = lds_raw<4>(p + 4), w2 = lds_raw<4>(p + 8), w3 = lds_raw<4>(p + 12);
           if (e0 & 1) {
-            const uint32_t w4 = lds_raw<4>(w + 16);
+            const uint32_t w4 = lds_raw<4>(p + 16);
             x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
                            __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
           } else {
             x = make_uint4(w0, w1, w2, w3);
           }
         }
-        st16(reinterpret_cast<char*>(((uintptr_t)out & ~(uintptr_t)15) + 16u * s), x);
+        st16(out, x);
       } else {
-        const uint32_t lo = e0 < 0 ? 0u : (uint32_t)e0;
-        const uint32_t hi = min(k.ni, (uint32_t)(e0 + (int32_t)NV));
-        for (uint32_t e = lo; e < hi; ++e)
-          E::store(out + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
+        // the run ends inside this window
+        for (uint32_t e = e0; e < k.nl; ++e)
+          E::store(run + (size_t)(k.i0 + e) * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
       }
     }
     __syncwarp();
@@ -556,7 +572,7 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
   auto step = [&](uint32_t (&cur)[UA], uint32_t (&nxt)[UA]) -> bool {
     uint32_t b2 = b, r2 = r0 + UA;
     Block blk2 = blk;
-    const bool same = r2 < blk.ni;
+    const bool same = r2 < blk.nl;
     if (!same) { b2 = b + kWorkerWarps; r2 = 0; }
     const bool more = same || b2 < nb;
     if (!same && more) blk2 = block_of(b2);
