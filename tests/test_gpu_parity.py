@@ -293,3 +293,24 @@ def test_offsets_beyond_32_bits(device):
     plan.check()
     assert torch.equal(out[:half], src.tensors[0].view(torch.int16))
     assert torch.equal(out[half:], src.tensors[1].view(torch.int16))
+
+
+@pytest.mark.parametrize("name,scale", [("cfg1b", "full"), ("cfg3", "small"), ("cfg5", "small"), ("cfg2", "medium")])
+def test_static_schedule_gives_the_same_result(device, name, scale):
+    """WB_PLAN_STATIC_SCHEDULE: every thread block walks the planner's fixed tile range instead of
+    drawing batches at run time; the output must not depend on the schedule."""
+    case = DeviceCase(make_workload(name, scale), device, flags=wb.WB_PLAN_STATIC_SCHEDULE,
+                      bucket_budget_bytes=1 << 20)
+    want = oracle_for(case)
+    case.plan.remap()
+    torch.cuda.synchronize()
+    case.plan.check()
+    assert_dst_equals(case, want)
+    case.reset_dst()
+    for r in range(case.plan.num_rounds()):
+        bucket = torch.empty(case.plan.bucket_bytes(r), dtype=torch.uint8, device=device)
+        case.plan.pack(r, bucket.data_ptr())
+        case.plan.unpack(r, bucket.data_ptr())
+    torch.cuda.synchronize()
+    case.plan.check()
+    assert_dst_equals(case, want)
