@@ -233,6 +233,12 @@ wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bucket, void*
  * sticky error word instead of hanging).  OK, NOT_BOUND, CUDA, or INTERNAL. */
 wb_status wb_plan_check(const wb_plan* plan);
 
+/* wb_wait_probe: self-test of the kernels' bounded waits.  Launches one thread that waits on a
+ * barrier nothing ever signals, with a limit of limit_ms (1..2000) milliseconds, and synchronises.
+ * Returns WB_ERR_INTERNAL when the wait gave up as designed (the expected outcome), WB_OK if it
+ * did not have to, CUDA / OOM on runtime errors.  The context stays usable afterwards. */
+wb_status wb_wait_probe(uint32_t limit_ms, void* cuda_stream);
+
 /* wb_remap_host: the same transfer for callers whose weights are in HOST memory.  The remap
  * is cut into groups of consecutive tiles; for each group the trainer bytes it reads are copied
  * host -> bound device regions on an internal copy stream, its tiles run on `cuda_stream`, and the

@@ -79,7 +79,7 @@ EXPORTS = [
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
     "wb_remap_host", "wb_remap_static", "wb_plan_check",
-    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -119,6 +119,7 @@ def load() -> C.CDLL:
     lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
     lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
+    lib.wb_wait_probe.argtypes = [C.c_uint32, vp]
     lib.wb_route_account.argtypes = [vp, vp, sz, vp, sz, C.c_double, C.c_double, vp, vp, vp, sz]
     lib.wb_diff2_nonzeros.argtypes = [vp, C.c_uint32, C.c_uint64, C.c_uint64, vp, C.c_uint64, vp, vp]
     lib.wb_diff2_recombine.argtypes = [vp, vp, sz, C.c_uint32, vp, sz, C.POINTER(sz)]
@@ -341,3 +342,8 @@ def wb_route_account(plan: Plan, trainer_node: Sequence[int], rollout_node: Sequ
                                  node_gbs, C.byref(st), ing.ctypes.data, req.ctypes.data, n_nodes),
            "wb_route_account")
     return {n: getattr(st, n) for n, _ in st._fields_}, ing, req
+
+
+def wb_wait_probe(limit_ms: int, stream: int = 0) -> int:
+    """Returns the raw status: WB_ERR_INTERNAL (11) means the bounded wait gave up as designed."""
+    return load().wb_wait_probe(limit_ms, stream)

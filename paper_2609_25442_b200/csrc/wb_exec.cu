@@ -255,14 +255,25 @@ __device__ __forceinline__ bool mbar_try(uint32_t addr, uint32_t parity) {
       : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
   return ok != 0;
 }
-// Wait for the phase with the given parity to complete; gives up after kWaitLimitNs.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Wait for the phase with the given parity to complete; gives up after `limit_ns`.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
   const uint32_t addr = smem_u32(bar);
   if (mbar_try(addr, parity)) return true;
   const uint64_t t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try(addr, parity)) return true;
-    if ((it & 255u) == 0 && global_ns() - t0 > kWaitLimitNs) return false;
+    if ((it & 255u) == 0 && global_ns() - t0 > limit_ns) return false;
+  }
+}
+
+// Self-test of the bounded wait: one thread waits on a barrier that nothing ever signals.  The
+// wait must give up after limit_ns, record its code and let the kernel end normally.
+__global__ void wb_wait_probe_kernel(uint64_t limit_ns, uint32_t* __restrict__ err) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(&bar, 0, limit_ns)) atomicMax(err, 0x7Du);   // "timed out", distinct from the executor's codes
   }
 }
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
@@ -995,6 +1006,24 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
   }
   plan->bound = true;
   return WB_OK;
+}
+
+extern "C" wb_status wb_wait_probe(uint32_t limit_ms, void* cuda_stream) {
+  if (limit_ms == 0 || limit_ms > 2000) return WB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t* d_err = nullptr;
+  uint32_t err = 0;
+  if (cudaMalloc(&d_err, sizeof(uint32_t)) != cudaSuccess) return WB_ERR_OOM;
+  cudaError_t e = cudaMemsetAsync(d_err, 0, sizeof(uint32_t), stream);
+  if (e == cudaSuccess) {
+    wb_wait_probe_kernel<<<1, 32, 0, stream>>>((uint64_t)limit_ms * 1000000ull, d_err);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&err, d_err, sizeof(uint32_t), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  cudaFree(d_err);
+  if (e != cudaSuccess) return WB_ERR_CUDA;
+  return err == 0x7Du ? WB_ERR_INTERNAL : WB_OK;
 }
 
 extern "C" wb_status wb_plan_check(const wb_plan* plan) {

@@ -314,3 +314,20 @@ def test_static_schedule_gives_the_same_result(device, name, scale):
     torch.cuda.synchronize()
     case.plan.check()
     assert_dst_equals(case, want)
+
+
+def test_bounded_wait_gives_up_and_the_context_survives(device):
+    """Every wait inside the kernels has a time limit.  A wait on a barrier that nothing signals runs
+    out, reports through the error word, and the kernel ends normally: later work still runs."""
+    import time
+    t0 = time.perf_counter()
+    status = wb.wb_wait_probe(50, torch.cuda.current_stream().cuda_stream)
+    dt = time.perf_counter() - t0
+    assert status == 11                      # WB_ERR_INTERNAL: the wait gave up as designed
+    assert 0.04 < dt < 1.5
+    case = DeviceCase(make_workload("cfg1"), device)     # the context is still usable
+    want = oracle_for(case)
+    case.plan.remap()
+    torch.cuda.synchronize()
+    case.plan.check()
+    assert_dst_equals(case, want)
