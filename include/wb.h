@@ -56,7 +56,8 @@ typedef enum {
   WB_ERR_CUDA = 9,             /* a CUDA runtime call failed                                 */
   WB_ERR_NOT_BOUND = 10,       /* execution requested before wb_plan_bind                    */
   WB_ERR_INTERNAL = 11,        /* a plan invariant does not hold (wb_plan_verify)            */
-  WB_ERR_STATIC_LIMIT = 12     /* the plan's tile table exceeds WB_STATIC_SCRATCH_BYTES       */
+  WB_ERR_STATIC_LIMIT = 12,    /* the plan's tile table exceeds WB_STATIC_SCRATCH_BYTES       */
+  WB_ERR_REPLICA_MISMATCH = 13 /* two trainer replicas of a checkpoint region differ          */
 } wb_status;
 
 typedef enum { WB_F32 = 0, WB_BF16 = 1 } wb_dtype;
@@ -232,6 +233,13 @@ wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bucket, void*
  * recorded an error (the kernels bound every internal wait; a wait that ran out sets a
  * sticky error word instead of hanging).  OK, NOT_BOUND, CUDA, or INTERNAL. */
 wb_status wb_plan_check(const wb_plan* plan);
+
+/* wb_plan_check_replicas (device, synchronous): the plan reads a replicated checkpoint region from
+ * one trainer replica only (Section 3.2: "the trainer workers collectively send only one copy"),
+ * which presumes the replicas are bit-identical.  This debug pass compares every pair of replicas
+ * the source layout declares, element by element, on the bound tensors.  *n_mismatches (host, may
+ * be NULL) receives the number of differing elements.  OK, REPLICA_MISMATCH, NOT_BOUND, CUDA. */
+wb_status wb_plan_check_replicas(const wb_plan* plan, uint64_t* n_mismatches, void* cuda_stream);
 
 /* wb_wait_probe: self-test of the kernels' bounded waits.  Launches one thread that waits on a
  * barrier nothing ever signals, with a limit of limit_ms (1..2000) milliseconds, and synchronises.

@@ -25,7 +25,7 @@ STATUS_NAMES = {
     0: "WB_OK", 1: "WB_ERR_INVALID_ARG", 2: "WB_ERR_DTYPE", 3: "WB_ERR_SHAPE_MISMATCH",
     4: "WB_ERR_OUT_OF_RANGE", 5: "WB_ERR_DST_OVERLAP", 6: "WB_ERR_UNCOVERED",
     7: "WB_ERR_BUCKET_TOO_SMALL", 8: "WB_ERR_OOM", 9: "WB_ERR_CUDA", 10: "WB_ERR_NOT_BOUND",
-    11: "WB_ERR_INTERNAL", 12: "WB_ERR_STATIC_LIMIT",
+    11: "WB_ERR_INTERNAL", 12: "WB_ERR_STATIC_LIMIT", 13: "WB_ERR_REPLICA_MISMATCH",
 }
 
 
@@ -79,7 +79,7 @@ EXPORTS = [
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
     "wb_remap_host", "wb_remap_static", "wb_plan_check",
-    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -120,6 +120,7 @@ def load() -> C.CDLL:
     lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
     lib.wb_wait_probe.argtypes = [C.c_uint32, vp]
+    lib.wb_plan_check_replicas.argtypes = [vp, C.POINTER(C.c_uint64), vp]
     lib.wb_route_account.argtypes = [vp, vp, sz, vp, sz, C.c_double, C.c_double, vp, vp, vp, sz]
     lib.wb_diff2_nonzeros.argtypes = [vp, C.c_uint32, C.c_uint64, C.c_uint64, vp, C.c_uint64, vp, vp]
     lib.wb_diff2_recombine.argtypes = [vp, vp, sz, C.c_uint32, vp, sz, C.POINTER(sz)]
@@ -229,6 +230,14 @@ class Plan:
 
     def check(self) -> None:
         _check(_lib.wb_plan_check(self.handle), "wb_plan_check")
+
+    def check_replicas(self, stream: int = 0) -> int:
+        """Number of elements in which trainer replicas differ (0 = consistent)."""
+        n = C.c_uint64()
+        st = _lib.wb_plan_check_replicas(self.handle, C.byref(n), stream)
+        if st not in (WB_OK, 13):
+            raise WbError(st, "wb_plan_check_replicas")
+        return n.value
 
     def remap(self, stream: int = 0) -> None:
         _check(_lib.wb_remap(self.handle, stream), "wb_remap")

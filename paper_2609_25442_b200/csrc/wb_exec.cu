@@ -952,7 +952,8 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
       bytes += up256(T->tiles.size() * sizeof(DTile)) + up256(T->extras.size() * sizeof(DDst)) +
                up256(T->cta_begin.size() * sizeof(uint32_t)) + 256;
     const size_t err_off = up256(bytes);
-    bytes = up256(err_off + 256);
+    const size_t cmp_off = err_off + 256;
+    bytes = up256(cmp_off + plan->replica_pairs.size() * sizeof(DCompare) + 256);
     std::vector<char> host(bytes, 0);
     if (!plan->d_arena || plan->arena_bytes != bytes) {
       wbi::release_device_tables(plan);
@@ -962,6 +963,22 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
     if (cudaGetDevice(&plan->device) != cudaSuccess) return WB_ERR_CUDA;
     char* dbase = static_cast<char*>(plan->d_arena);
     plan->d_err = reinterpret_cast<uint32_t*>(dbase + err_off);
+    plan->d_mismatch = reinterpret_cast<unsigned long long*>(dbase + err_off + 64);
+    plan->d_compare = reinterpret_cast<DCompare*>(dbase + cmp_off);
+    {
+      DCompare* hc = reinterpret_cast<DCompare*>(host.data() + cmp_off);
+      for (size_t k = 0; k < plan->replica_pairs.size(); ++k) {
+        const ReplicaPair& rp = plan->replica_pairs[k];
+        const NSlice& a = plan->src.slices[rp.slice_a];
+        const NSlice& b = plan->src.slices[rp.slice_b];
+        DCompare c{};
+        c.a = (uint64_t)(uintptr_t)plan->src_base[a.tensor] + a.elem(rp.rect.r0, rp.rect.c0) * es;
+        c.b = (uint64_t)(uintptr_t)plan->src_base[b.tensor] + b.elem(rp.rect.r0, rp.rect.c0) * es;
+        c.nr = (uint32_t)rp.rect.nr; c.nc = (uint32_t)rp.rect.nc;
+        c.a_sr = (uint32_t)a.sr(); c.a_sc = (uint32_t)a.sc(); c.b_sr = (uint32_t)b.sr(); c.b_sc = (uint32_t)b.sc();
+        hc[k] = c;
+      }
+    }
     size_t off = 0;
     for (size_t ti = 0; ti < tabs.size(); ++ti) {
       TileTable* T = tabs[ti];
@@ -1006,6 +1023,45 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
   }
   plan->bound = true;
   return WB_OK;
+}
+
+// Replica consistency: the planner reads a replicated region from one holder only, which is valid
+// because replicas carry the same bits.  This debug pass compares every replica pair element by
+// element and counts the differences.
+template <typename T>
+__global__ void wb_compare_kernel(const DCompare* __restrict__ ops, uint32_t n_ops,
+                                  unsigned long long* __restrict__ mismatches) {
+  unsigned long long bad = 0;
+  for (uint32_t k = blockIdx.x; k < n_ops; k += gridDim.x) {
+    const DCompare c = ops[k];
+    const T* a = reinterpret_cast<const T*>(c.a);
+    const T* b = reinterpret_cast<const T*>(c.b);
+    const unsigned long long n = (unsigned long long)c.nr * c.nc;
+    for (unsigned long long e = threadIdx.x; e < n; e += blockDim.x) {
+      const unsigned long long i = e / c.nc, j = e - i * c.nc;
+      if (a[i * c.a_sr + j * c.a_sc] != b[i * c.b_sr + j * c.b_sc]) ++bad;
+    }
+  }
+  if (bad) atomicAdd(mismatches, bad);
+}
+
+extern "C" wb_status wb_plan_check_replicas(const wb_plan* plan, uint64_t* n_mismatches, void* cuda_stream) {
+  if (!plan) return WB_ERR_INVALID_ARG;
+  if (!plan->bound) return WB_ERR_NOT_BOUND;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  unsigned long long bad = 0;
+  const uint32_t n = (uint32_t)plan->replica_pairs.size();
+  if (n) {
+    if (cudaMemsetAsync(plan->d_mismatch, 0, sizeof(unsigned long long), stream) != cudaSuccess) return WB_ERR_CUDA;
+    const uint32_t grid = n < 148u * 8 ? n : 148u * 8;
+    if (esize(plan->src.dtype) == 4) wb_compare_kernel<uint32_t><<<grid, 256, 0, stream>>>(plan->d_compare, n, plan->d_mismatch);
+    else wb_compare_kernel<uint16_t><<<grid, 256, 0, stream>>>(plan->d_compare, n, plan->d_mismatch);
+    if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaMemcpyAsync(&bad, plan->d_mismatch, sizeof(bad), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return WB_ERR_CUDA;
+  }
+  if (n_mismatches) *n_mismatches = bad;
+  return bad ? WB_ERR_REPLICA_MISMATCH : WB_OK;
 }
 
 extern "C" wb_status wb_wait_probe(uint32_t limit_ms, void* cuda_stream) {

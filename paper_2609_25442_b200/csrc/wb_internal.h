@@ -128,6 +128,18 @@ struct Slab {
   uint32_t sender, receiver;       // virtual ranks
 };
 
+// Two source slices that hold the same checkpoint rectangle (replicas).
+struct ReplicaPair { uint32_t slice_a, slice_b; Rect rect; };
+
+// Device form of a replica pair: element (i, j) of the rectangle at a + (i*a_sr + j*a_sc)*es etc.
+struct alignas(16) DCompare {
+  uint64_t a, b;
+  uint32_t nr, nc;
+  uint32_t a_sr, a_sc, b_sr, b_sc;
+  uint32_t pad[2];
+};
+static_assert(sizeof(DCompare) == 48, "");
+
 struct Payload {
   uint32_t slab;
   Rect rect;
@@ -155,6 +167,7 @@ struct wb_plan {
   std::vector<wbi::Slab> slabs;
   std::vector<uint32_t> slab_dsts;
   std::vector<wbi::Round> rounds;
+  std::vector<wbi::ReplicaPair> replica_pairs;
   wbi::TileTable remap;
   std::vector<uint64_t> egress, ingress;
   wb_plan_stats_t stats{};
@@ -166,6 +179,8 @@ struct wb_plan {
   std::vector<void*> dst_base;
   void* d_arena = nullptr;              // one device allocation holding every table
   uint32_t* d_err = nullptr;            // sticky device error word (inside the arena)
+  wbi::DCompare* d_compare = nullptr;   // replica pairs (inside the arena)
+  unsigned long long* d_mismatch = nullptr;
   // wb_remap_host pipeline state (created on first use; streams and events are CUDA handles)
   std::vector<wbi::HostGroup> host_groups;
   void* h2d_stream = nullptr;

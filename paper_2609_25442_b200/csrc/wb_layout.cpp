@@ -23,6 +23,7 @@ extern "C" const char* wb_status_str(wb_status s) {
     case WB_ERR_NOT_BOUND: return "plan not bound to device memory";
     case WB_ERR_INTERNAL: return "plan invariant violated";
     case WB_ERR_STATIC_LIMIT: return "tile table larger than the static scratch array";
+    case WB_ERR_REPLICA_MISMATCH: return "trainer replicas of a checkpoint region differ";
   }
   return "unknown status";
 }

@@ -289,6 +289,7 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
     struct Hit { uint32_t dslice; Rect rect; };
     std::vector<Piece> pieces;
     std::vector<Rect> owned, frags, tmp;
+    std::vector<uint32_t> owned_by;
     std::vector<uint32_t> order;
     std::vector<Hit> hits;
     std::vector<uint64_t> covered;
@@ -316,6 +317,7 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
       });
       pieces.clear();
       owned.clear();
+      owned_by.clear();
       uint64_t held_area = 0, slice_area = 0;
       for (size_t g0 = 0; g0 < order.size();) {
         size_t g1 = g0 + 1;
@@ -327,10 +329,15 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
         }
         const uint32_t m = (uint32_t)(g1 - g0);
         slice_area += gr.area() * m;
+        // replicas are assumed identical; remember which pairs a consistency check must compare
+        for (uint32_t k = 1; k < m; ++k) P->replica_pairs.push_back(ReplicaPair{order[g0], order[g0 + k], gr});
         // keep only what no earlier group already owns
         frags.assign(1, gr);
-        for (const Rect& o : owned) {
-          if (!intersect(gr, o, nullptr)) continue;
+        for (size_t oi = 0; oi < owned.size(); ++oi) {
+          const Rect& o = owned[oi];
+          Rect both;
+          if (!intersect(gr, o, &both)) continue;
+          P->replica_pairs.push_back(ReplicaPair{owned_by[oi], order[g0], both});
           tmp.clear();
           for (const Rect& f : frags) subtract(f, o, &tmp);
           frags.swap(tmp);
@@ -338,6 +345,7 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
         }
         for (const Rect& f : frags) {
           owned.push_back(f);
+          owned_by.push_back(order[g0]);
           held_area += f.area();
           if (m == 1 || (P->opts.flags & WB_PLAN_NO_REPLICA_SPLIT)) {
             pieces.push_back(Piece{f, order[g0]});

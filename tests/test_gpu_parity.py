@@ -94,7 +94,7 @@ def test_pack_unpack_matches_oracle(device, name, scale, budget):
     assert_dst_equals(case, want)
 
 
-@pytest.mark.parametrize("seed", range(48))
+@pytest.mark.parametrize("seed", range(160))
 def test_fuzz_layouts(device, seed):
     src_dt, dst_dt = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][seed % 4]
     shapes, tl, rl = fuzz_case(9000 + seed, src_dt, dst_dt, max_dim=[40, 150, 300][seed % 3])
@@ -331,3 +331,17 @@ def test_bounded_wait_gives_up_and_the_context_survives(device):
     torch.cuda.synchronize()
     case.plan.check()
     assert_dst_equals(case, want)
+
+
+def test_replica_consistency_check(device):
+    """The plan reads a replicated region from one replica; wb_plan_check_replicas verifies the
+    assumption behind that on the bound tensors."""
+    wl = make_workload("cfg1")                    # norms live on both TP ranks
+    case = DeviceCase(wl, device)
+    assert case.plan.check_replicas() == 0
+    k = wl.trainer.index("t2.final.flat")          # TP rank 1's copy of final_norm starts this shard
+    case.src.tensors[k][3] += 1.0
+    case.src.tensors[k][200] += 1.0
+    assert case.plan.check_replicas() == 2
+    wl4 = make_workload("cfg4", "small")           # no replicas at all
+    assert DeviceCase(wl4, device).plan.check_replicas() == 0

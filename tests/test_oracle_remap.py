@@ -239,7 +239,7 @@ def test_checkpoint_view_recovers_the_seeded_checkpoint(name, scale):
 
 
 # ---- fuzz: random affine source maps against a dictionary join --------------------------------------
-@pytest.mark.parametrize("seed", range(60))
+@pytest.mark.parametrize("seed", range(200))
 def test_fuzz_against_dictionary_join(seed):
     src_dt, dst_dt = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][seed % 4]
     shapes, tl, rl = fuzz_case(1000 + seed, src_dt, dst_dt)

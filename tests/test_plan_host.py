@@ -106,7 +106,7 @@ def test_plan_tables_reproduce_oracle(name, scale):
         assert st["bucket_bytes_max"] <= 1 << 20
 
 
-@pytest.mark.parametrize("seed", range(40))
+@pytest.mark.parametrize("seed", range(240))
 def test_fuzz_plans(seed):
     src_dt, dst_dt = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][seed % 4]
     shapes, tl, rl = fuzz_case(5000 + seed, src_dt, dst_dt, max_dim=70)
