@@ -171,47 +171,6 @@ __device__ __forceinline__ void copy_run(const char* __restrict__ s, char* __res
   }
 }
 
-// Rows whose every run starts 16-byte aligned on both sides: one flat vector index space.
-template <int ES, int ED>
-__device__ __forceinline__ void copy_rows_aligned(const char* __restrict__ s, char* __restrict__ d,
-                                                  uint32_t nr, uint32_t nc, uint32_t sp, uint32_t dp,
-                                                  uint32_t t, uint32_t nth) {
-  using UN = Unit<ES, ED>;
-  using E = Elem<ES, ED>;
-  constexpr int NV = UN::NV;
-  constexpr int U = Unroll<ES, ED>::U;
-  const uint32_t vpr = nc / NV;
-  const uint32_t total = nr * vpr;
-  const size_t sps = (size_t)sp * ES, dps = (size_t)dp * ED;
-  for (uint32_t v0 = t; v0 < total; v0 += nth * U) {
-    UN r[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const uint32_t v = v0 + u * nth;
-      if (v < total) {
-        const uint32_t row = v / vpr, cv = v - row * vpr;
-        r[u].load(s + row * sps + (size_t)cv * (NV * ES));
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const uint32_t v = v0 + u * nth;
-      if (v < total) {
-        const uint32_t row = v / vpr, cv = v - row * vpr;
-        st16(d + row * dps + (size_t)cv * 16, r[u].out());
-      }
-    }
-  }
-  const uint32_t rem = nc - vpr * NV;   // ragged row ends
-  if (rem) {
-    const uint32_t cnt = nr * rem;
-    for (uint32_t e = t; e < cnt; e += nth) {
-      const uint32_t row = e / rem, c = vpr * NV + (e - row * rem);
-      E::store(d + row * dps + (size_t)c * ED, E::load(s + row * sps + (size_t)c * ES));
-    }
-  }
-}
-
 struct TileRegs {
   uint4 a, b, c;
 };
@@ -321,8 +280,14 @@ template <int ES, int ED> struct Rings {      // worker ring: staged chunks and 
   static constexpr size_t kDyn = kDirect + (size_t)kSlots * kSlotBytes;
 };
 constexpr int kWorkerWarps = kWorkers / 32;
+#ifndef WB_STAGED_MIN_ROW_BYTES
+#define WB_STAGED_MIN_ROW_BYTES 1024
+#endif
+constexpr size_t kStagedMinRowBytes = WB_STAGED_MIN_ROW_BYTES;   // shorter rows take the warp-level path
 
-enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_TRANS = 3 };
+enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3 };
+constexpr uint32_t kBatchTileBytes = 32768;    // tiles moving less than this are batched, one warp per tile
+constexpr uint32_t kBatchMaxTiles = 120;
 
 // What the producer tells the workers about one ring slot.
 struct ChunkDesc {
@@ -475,21 +440,21 @@ template <int ES> __device__ __forceinline__ uint32_t pack_pair16(uint32_t lo, u
 //            ends of a whole run use element stores.
 // The patch pitch is odd in 32-bit words, so lanes hit distinct banks in both phases.
 template <int ES, int ED>
-__device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratch, uint32_t scratch_bytes,
-                                               uint32_t warp, uint32_t lane) {
+__device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch, uint32_t patch_bytes,
+                                               uint32_t warp, uint32_t nw, uint32_t lane) {
+  // patch: this warp's private part of the ring slot; warp / nw: its share of the tile's blocks
   using E = Elem<ES, ED>;
   constexpr uint32_t NV = 16 / ED;
   constexpr uint32_t PER_WORD = 4 / ED;                     // destination elements per 32-bit word
   constexpr int UA = 16;                                    // rows per batch of loads
   // rows per block: as many as the warp's share of the slot allows next to the NV-1 halo rows
   // (multiple of 8, at most 64); no halo is needed when every run starts on a 16-byte boundary
-  const uint32_t share = scratch_bytes / kWorkerWarps / 4;  // words
+  const uint32_t share = patch_bytes / 4;                    // words
   const bool aligned = (((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0;
   const uint32_t halo = aligned ? 0u : NV - 1, room = aligned ? 0u : 8u;
   const uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD - room) & ~7u);
   const uint32_t pitch_w = (rb + room) / PER_WORD + 1;      // odd: (rb+room)/PER_WORD is even
-  uint32_t* T = reinterpret_cast<uint32_t*>(scratch) + warp * (32 * pitch_w);
-  const uint32_t tbase = smem_u32(T);
+  const uint32_t tbase = smem_u32(patch);
   const uint32_t nbi = (f.nr + rb - 1) / rb, nbj = (f.nc + 31) / 32;
   const uint32_t nb = nbi * nbj;
   const size_t sps = (size_t)f.ssr * ES;
@@ -529,48 +494,42 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
           asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 4), "r"((uint32_t)cast_raw<ES, ED>(v[u])));
     }
   };
-  // phase B: the 16-byte windows of every destination run that start inside the block's rows
+  // phase B: lane j writes destination run j -- the 16-byte windows that start inside the block's rows
   auto phase_b = [&](const Block& k) {
     __syncwarp();
-    const uint32_t smax = k.ni / NV + 2;                          // windows per run, upper bound
-    for (uint32_t task = lane; task < k.nj * smax; task += 32) {
-      const uint32_t w = task / k.nj, j = task - w * k.nj;        // consecutive lanes: consecutive runs
-      char* run = f.d + (size_t)(k.j0 + j) * f.dsc * ED;          // element (j, 0) of the run
+    if (lane < k.nj) {
+      char* run = f.d + (size_t)(k.j0 + lane) * f.dsc * ED;       // element (j, 0) of the run
       const uint32_t a = (uint32_t)(((uintptr_t)run / ED + k.i0) & (NV - 1));   // offset of row i0 in its window
-      const uint32_t trow = tbase + j * pitch_w * 4;
-      if (w == 0) {
-        // rows before the first window that starts here: the previous block's window covers them,
-        // except at the very start of the run
-        const uint32_t lead = a ? NV - a : 0;
-        if (k.i0 == 0)
-          for (uint32_t e = 0; e < min(lead, k.ni); ++e)
-            E::store(run + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
-        continue;
-      }
-      const uint32_t e0 = (a ? NV - a : 0) + (w - 1) * NV;         // first row (relative to i0) of the window
-      if (e0 >= k.ni) continue;
-      char* out = run + (size_t)(k.i0 + e0) * ED;                 // 16-byte aligned
-      if (e0 + NV <= k.nl) {
-        uint4 x;
-        if constexpr (ED == 4) {
-          x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
-          x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
-        } else {
-          const uint32_t p = trow + (e0 >> 1) * 4;
-          const uint32_t w0 = lds_raw<4>(p), w1 = lds_raw<4>(p + 4), w2 = lds_raw<4>(p + 8), w3 = lds_raw<4>(p + 12);
-          if (e0 & 1) {
-            const uint32_t w4 = lds_raw<4>(p + 16);
-            x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
-                           __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
+      const uint32_t lead = a ? NV - a : 0;                        // rows before the first window that starts here
+      const uint32_t trow = tbase + lane * pitch_w * 4;
+      // those rows belong to the previous block's last window, except at the very start of the run
+      if (k.i0 == 0)
+        for (uint32_t e = 0; e < min(lead, k.ni); ++e)
+          E::store(run + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
+      char* out = run + (size_t)(k.i0 + lead) * ED;               // 16-byte aligned
+      for (uint32_t e0 = lead; e0 < k.ni; e0 += NV, out += 16) {
+        if (e0 + NV <= k.nl) {
+          uint4 x;
+          if constexpr (ED == 4) {
+            x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
+            x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
           } else {
-            x = make_uint4(w0, w1, w2, w3);
+            const uint32_t p = trow + (e0 >> 1) * 4;
+            const uint32_t w0 = lds_raw<4>(p), w1 = lds_raw<4>(p + 4), w2 = lds_raw<4>(p + 8), w3 = lds_raw<4>(p + 12);
+            if (e0 & 1) {
+              const uint32_t w4 = lds_raw<4>(p + 16);
+              x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
+                             __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
+            } else {
+              x = make_uint4(w0, w1, w2, w3);
+            }
           }
+          st16(out, x);
+        } else {
+          // the run ends inside this window
+          for (uint32_t e = e0; e < k.nl; ++e)
+            E::store(run + (size_t)(k.i0 + e) * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
         }
-        st16(out, x);
-      } else {
-        // the run ends inside this window
-        for (uint32_t e = e0; e < k.nl; ++e)
-          E::store(run + (size_t)(k.i0 + e) * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
       }
     }
     __syncwarp();
@@ -584,7 +543,7 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
     uint32_t b2 = b, r2 = r0 + UA;
     Block blk2 = blk;
     const bool same = r2 < blk.nl;
-    if (!same) { b2 = b + kWorkerWarps; r2 = 0; }
+    if (!same) { b2 = b + nw; r2 = 0; }
     const bool more = same || b2 < nb;
     if (!same && more) blk2 = block_of(b2);
     if (more) issue(blk2, r2, nxt);
@@ -601,47 +560,115 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* scratc
   }
 }
 
-// Cooperative execution of one tile by the worker warps (thread t of nth).
+// Workers: ROWS tile with short rows (dst[i*dsr + j] = cast(src[i*ssr + j]), nc small).  The tile is
+// a flat sequence of nr*nc elements; every warp takes batches of 256 consecutive elements on its
+// own.  Lane l loads elements l, l+32, ... of the batch (coalesced inside each row; row and column
+// advance incrementally, no division per element), eight loads in flight, one batch ahead.  If the
+// destination rows are contiguous (dsr == nc) the cast values go through a 512-byte private patch
+// and leave as 16-byte vectors; otherwise each value is stored to its own row.
 template <int ES, int ED>
-__device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __restrict__ extras, uint64_t dst_add,
-                                          uint32_t t) {
+__device__ __forceinline__ void warp_small_rows(const TileFields& f, char* patch_mem, uint32_t warp, uint32_t nw,
+                                                uint32_t lane) {
   using E = Elem<ES, ED>;
-  constexpr uint32_t nth = kWorkers;
-  const char* s = f.s;
-  char* d = f.d;
-  const uint32_t nr = f.nr, nc = f.nc, ssr = f.ssr, ssc = f.ssc, dsr = f.dsr, dsc = f.dsc;
-  if (f.kind == KIND_ROWS && f.n_extra == 0) {
-    if (nr == 1) {
-      copy_run<ES, ED>(s, d, nc, t, nth);
-    } else {
-      const bool aligned = (((uintptr_t)d & 15u) == 0) && ((((size_t)dsr * ED) & 15u) == 0) &&
-                           (((uintptr_t)s & (Unit<ES, ED>::SRC_ALIGN - 1)) == 0) &&
-                           ((((size_t)ssr * ES) & (Unit<ES, ED>::SRC_ALIGN - 1)) == 0);
-      if (aligned) {
-        copy_rows_aligned<ES, ED>(s, d, nr, nc, ssr, dsr, t, nth);
-      } else if (nc >= 128) {
-        const uint32_t lane = t & 31, warp = t >> 5;
-        for (uint32_t row = warp; row < nr; row += nth / 32)
-          copy_run<ES, ED>(s + (size_t)row * ssr * ES, d + (size_t)row * dsr * ED, nc, lane, 32);
+  constexpr uint32_t NV = 16 / ED;
+  constexpr int U = 8;
+  constexpr uint32_t B = 32 * U;
+  const uint32_t nc = f.nc, cnt = f.nr * f.nc;
+  const bool packed = f.dsr == nc;
+  // packed: elements before the first 16-byte boundary of the destination are stored one by one
+  uint32_t head = 0;
+  if (packed) {
+    head = (uint32_t)((16u - ((uintptr_t)f.d & 15u)) & 15u) / ED;
+    if (head > cnt) head = cnt;
+    if (warp == 0 && lane < head) {
+      const uint32_t i = lane / nc, j = lane - i * nc;
+      E::store(f.d + (size_t)lane * ED, E::load(f.s + ((size_t)i * f.ssr + j) * ES));
+    }
+  }
+  const uint32_t n_batches = (cnt - head + B - 1) / B;
+  if (warp >= n_batches) return;
+  const uint32_t q32 = 32 / nc, r32 = 32 % nc;
+  const uint32_t patch = smem_u32(patch_mem);               // B * ED bytes of this warp's part of the slot
+  // loads of batch b: raw source elements
+  auto issue = [&](uint32_t b, uint32_t (&raw)[U]) {
+    const uint32_t e0 = head + b * B + lane;
+    uint32_t i = e0 / nc, j = e0 - i * nc;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      raw[u] = 0;
+      if (e0 + 32u * u < cnt) {
+        const char* p = f.s + ((size_t)i * f.ssr + j) * ES;
+        if constexpr (ES == 4) raw[u] = __ldcs(reinterpret_cast<const uint32_t*>(p));
+        else raw[u] = __ldcs(reinterpret_cast<const uint16_t*>(p));
+      }
+      i += q32; j += r32;
+      if (j >= nc) { j -= nc; ++i; }
+    }
+  };
+  auto consume = [&](uint32_t b, const uint32_t (&raw)[U]) {
+    const uint32_t e0 = head + b * B;                       // first element of the batch
+    const uint32_t n = min(B, cnt - e0);
+    if (!packed) {
+      uint32_t i = (e0 + lane) / nc, j = (e0 + lane) - i * nc;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        if (lane + 32u * u < n) E::store(f.d + ((size_t)i * f.dsr + j) * ED, cast_raw<ES, ED>(raw[u]));
+        i += q32; j += r32;
+        if (j >= nc) { j -= nc; ++i; }
+      }
+      return;
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t at = patch + (lane + 32u * u) * ED;
+      if constexpr (ED == 2) asm volatile("st.shared.u16 [%0], %1;" ::"r"(at), "h"((uint16_t)cast_raw<ES, ED>(raw[u])));
+      else asm volatile("st.shared.u32 [%0], %1;" ::"r"(at), "r"((uint32_t)cast_raw<ES, ED>(raw[u])));
+    }
+    __syncwarp();
+    char* out = f.d + (size_t)e0 * ED;                      // 16-byte aligned
+    for (uint32_t v = lane; v * NV < n; v += 32) {
+      if ((v + 1) * NV <= n) {
+        uint4 x;
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x.x), "=r"(x.y), "=r"(x.z), "=r"(x.w) : "r"(patch + v * 16));
+        st16(out + (size_t)v * 16, x);
       } else {
-        const uint32_t cnt = nr * nc;
-        for (uint32_t e = t; e < cnt; e += nth) {
-          const uint32_t i = e / nc, j = e - i * nc;
-          E::store(d + ((size_t)i * dsr + j) * ED, E::load(s + ((size_t)i * ssr + j) * ES));
-        }
+        for (uint32_t e = v * NV; e < n; ++e)
+          E::store(out + (size_t)e * ED, (typename E::V)lds_raw<ED>(patch + e * ED));
       }
     }
-  } else {
-    // element-wise: arbitrary strides, any number of destinations
-    const uint32_t cnt = nr * nc;
-    for (uint32_t e = t; e < cnt; e += nth) {
-      const uint32_t i = e / nc, j = e - i * nc;
-      const typename E::V v = E::load(s + ((size_t)i * ssr + (size_t)j * ssc) * ES);
-      E::store(d + ((size_t)i * dsr + (size_t)j * dsc) * ED, v);
-      for (uint32_t x = 0; x < f.n_extra; ++x) {
-        const DDst o = extras[f.extra + x];
-        E::store(reinterpret_cast<char*>(o.dst + dst_add) + ((size_t)i * o.sr + (size_t)j * o.sc) * ED, v);
-      }
+    __syncwarp();
+  };
+  uint32_t b = warp;
+  auto step = [&](uint32_t (&cr)[U], uint32_t (&nx)[U]) -> bool {
+    const uint32_t b2 = b + nw;
+    const bool more = b2 < n_batches;
+    if (more) issue(b2, nx);
+    consume(b, cr);
+    b = b2;
+    return more;
+  };
+  uint32_t ra[U], rb2[U];
+  issue(b, ra);
+  for (;;) {
+    if (!step(ra, rb2)) break;
+    if (!step(rb2, ra)) break;
+  }
+}
+
+// Element-wise execution of a tile by nth cooperating threads (this one is t): arbitrary strides, any
+// number of destinations.  Only rare shapes come here (strided vectors, fan-out to replicas).
+template <int ES, int ED>
+__device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __restrict__ extras, uint64_t dst_add,
+                                          uint32_t t, uint32_t nth) {
+  using E = Elem<ES, ED>;
+  const uint64_t cnt = (uint64_t)f.nr * f.nc;
+  for (uint64_t e = t; e < cnt; e += nth) {
+    const uint32_t i = (uint32_t)(e / f.nc), j = (uint32_t)(e - (uint64_t)i * f.nc);
+    const typename E::V v = E::load(f.s + ((size_t)i * f.ssr + (size_t)j * f.ssc) * ES);
+    E::store(f.d + ((size_t)i * f.dsr + (size_t)j * f.dsc) * ED, v);
+    for (uint32_t x = 0; x < f.n_extra; ++x) {
+      const DDst o = extras[f.extra + x];
+      E::store(reinterpret_cast<char*>(o.dst + dst_add) + ((size_t)i * o.sr + (size_t)j * o.sc) * ED, v);
     }
   }
 }
@@ -704,11 +731,27 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
       if (d.mode == MODE_ROWS) {
         staged_rows<ES, ED>(d, stage, tr);
       } else {
-        const TileFields f = decode(load_tile(tiles + d.tile), src_add, dst_add);
-        if (d.mode == MODE_TRANS)
-          warp_transpose<ES, ED>(f, const_cast<char*>(stage), kSlotBytes, tr >> 5, t & 31);
-        else
-          coop_tile<ES, ED>(f, extras, dst_add, t);
+        // queued tiles: one big tile shared by all worker warps, or a run of small tiles with one
+        // warp per tile
+        const bool run = d.mode == MODE_BATCH;
+        const uint32_t warp = tr >> 5, lane = t & 31;
+        const uint32_t w = run ? 0u : warp, nw = run ? 1u : (uint32_t)kWorkerWarps;
+        // every warp owns one fixed part of the slot as scratch, whatever kind of tile it runs
+        constexpr uint32_t kPatchBytes = ((uint32_t)kSlotBytes / kWorkerWarps) & ~15u;
+        char* patch = const_cast<char*>(stage) + warp * kPatchBytes;
+        for (uint32_t k = d.tile + (run ? warp : 0u); k < d.tile + d.nr; k += run ? (uint32_t)kWorkerWarps : 1u) {
+          const TileFields f = decode(load_tile(tiles + k), src_add, dst_add);
+          if (f.n_extra == 0 && f.kind == KIND_TRANS) {
+            warp_transpose<ES, ED>(f, patch, kPatchBytes, w, nw, lane);
+          } else if (f.n_extra == 0 && f.kind == KIND_ROWS && (f.nr == 1 || (size_t)f.nc * ES >= kStagedMinRowBytes)) {
+            for (uint32_t row = w; row < f.nr; row += nw)
+              copy_run<ES, ED>(f.s + (size_t)row * f.ssr * ES, f.d + (size_t)row * f.dsr * ED, f.nc, lane, 32);
+          } else if (f.n_extra == 0 && f.kind == KIND_ROWS && f.nr * (uint64_t)f.nc < (1ull << 31)) {
+            warp_small_rows<ES, ED>(f, patch, w, nw, lane);
+          } else {
+            coop_tile<ES, ED>(f, extras, dst_add, w * 32 + lane, nw * 32);
+          }
+        }
       }
       __syncwarp();
       if ((t & 31) == 0) mbar_arrive(&slot_empty[slot]);
@@ -729,12 +772,13 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     if (!ok) { if (lane == 0) atomicMax(err, ERR_WAIT_SLOT_EMPTY); failed = true; }
     return ok != 0;
   };
-  auto push_simple = [&](uint32_t mode, uint32_t tile) {
+  auto push_simple = [&](uint32_t mode, uint32_t tile, uint32_t count = 1) {
     if (!acquire_slot()) return;
     const uint32_t slot = n_w % kSlots;
     if (lane == 0) {
       desc[slot].mode = mode;
       desc[slot].tile = tile;
+      desc[slot].nr = count;
       mbar_arrive(&slot_full[slot]);    // release: the descriptor is visible to whoever sees the phase
     }
     ++n_w;
@@ -808,11 +852,23 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     return true;
   };
 
+  uint32_t run0 = 0, run_n = 0;         // pending run of small tiles [run0, run0 + run_n)
+  auto flush_run = [&]() {
+    if (run_n) push_simple(MODE_BATCH, run0, run_n);
+    run_n = 0;
+  };
   while (!failed && next_batch()) {
   TileRegs nxt = load_tile(tiles + bk);
   for (uint32_t k = bk; k < bend && !failed; ++k) {
     const TileFields f = decode(nxt, src_add, dst_add);
     if (k + 1 < bend) nxt = load_tile(tiles + k + 1);
+    // small tiles are handed over in runs and executed one warp per tile
+    if ((uint64_t)f.nr * f.nc * (ES + ED * (1 + f.n_extra)) < kBatchTileBytes && !direct_ok<ES, ED>(f)) {
+      if (run_n == 0) run0 = k;
+      if (++run_n == kBatchMaxTiles) flush_run();
+      continue;
+    }
+    flush_run();
     if (direct_ok<ES, ED>(f)) {
       if (lane == 0) {
         for (uint32_t i = 0; i < f.nr && !failed; ++i) {
@@ -831,7 +887,7 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
         }
       }
       failed = __shfl_sync(0xFFFFFFFFu, (uint32_t)failed, 0) != 0;
-    } else if (f.kind == KIND_ROWS && f.n_extra == 0 && (size_t)f.nc * ES >= 128) {
+    } else if (f.kind == KIND_ROWS && f.n_extra == 0 && (size_t)f.nc * ES >= kStagedMinRowBytes) {
       const uint32_t row_bytes = f.nc * ES + 16;                 // worst-case aligned superset of a row
       if (row_bytes <= (uint32_t)kSlotBytes) {
         const uint32_t pitch = roundup16(row_bytes);
@@ -846,12 +902,11 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
             push_staged(MODE_ROWS, f.s + ((size_t)r * f.ssr + c) * ES, f.d + ((size_t)r * f.dsr + c) * ED, 1,
                         min(piece, f.nc - c), 0, 0, (uint32_t)kSlotBytes);
       }
-    } else if (f.kind == KIND_TRANS && f.n_extra == 0) {
-      push_simple(MODE_TRANS, k);         // no staging: the workers use the slot as scratch
     } else {
-      push_simple(MODE_COOP, k);
+      push_simple(MODE_COOP, k);          // transposes, short rows, fan-out: the workers share the tile
     }
   }
+  flush_run();          // runs do not cross scheduling batches: tile indices must stay consecutive
   }
   if (lane == 0) {
     while (!failed && n_store < n_load) store_oldest();
