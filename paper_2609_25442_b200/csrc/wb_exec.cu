@@ -286,7 +286,10 @@ constexpr int kWorkerWarps = kWorkers / 32;
 constexpr size_t kStagedMinRowBytes = WB_STAGED_MIN_ROW_BYTES;   // shorter rows take the warp-level path
 
 enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3 };
-constexpr uint32_t kBatchTileBytes = 32768;    // tiles moving less than this are batched, one warp per tile
+#ifndef WB_BATCH_TILE_BYTES
+#define WB_BATCH_TILE_BYTES 8192
+#endif
+constexpr uint32_t kBatchTileBytes = WB_BATCH_TILE_BYTES;   // tiles moving less than this are batched, one warp per tile
 constexpr uint32_t kBatchMaxTiles = 120;
 
 // What the producer tells the workers about one ring slot.
