@@ -1,18 +1,27 @@
 // Device side of the weight-remap library: binding a plan to device memory and the
 // persistent tile-walking kernel behind wb_remap / wb_pack / wb_unpack (sm_100a).
 //
-// One launch executes a whole tile table.  Each thread block owns a contiguous range of
-// tiles (balanced by bytes at plan time) and walks it; tiles are independent, so there is
-// no inter-block communication and nothing a block ever waits on.
+// One persistent launch (one thread block per SM) executes a whole tile table.  Blocks draw
+// batches of consecutive tiles from a counter in device memory (or walk the byte-balanced range
+// the planner computed, under WB_PLAN_STATIC_SCHEDULE); tiles are independent, so blocks never
+// wait on each other.  Inside a block warp 0 is the producer and the other warps are workers:
+//
+//   direct   same element size, long rows, source and destination congruent mod 16 bytes:
+//            lane 0 of the producer moves them by itself with bulk copies global -> shared ->
+//            global through a small ring; the data never touches registers.
+//   staged   other ROWS tiles with rows of at least kStagedMinRowBytes: the producer warp bulk-
+//            loads the rows into a ring slot, the workers realign, cast and store 16 bytes at a time.
+//   queued   everything else is handed to the workers by tile index, either one tile shared by all
+//            worker warps or a run of small tiles, one warp per tile.
 //
 // Tile kinds
 //   ROWS   nr runs of nc contiguous elements on both sides (nr == 1: one long run).
-//          16-byte vector loads and stores with the cast done in registers; unaligned
-//          heads/tails are peeled per run; rows whose pitches keep every run 16-byte
-//          aligned are flattened into one vector index space.
 //   TRANS  source contiguous along j, destination contiguous along i: each warp transposes
 //          32-column blocks through a private shared-memory patch.
-//   ELEM   anything else (strided vectors, fan-out): one element per thread.
+//   ELEM   anything else (strided vectors, fan-out to several destinations): element loop.
+//
+// Every wait in the kernel is bounded (see mbar_wait); a wait that runs out sets the plan's error
+// word, which wb_plan_check reports.
 #include <cuda_runtime.h>
 
 #include <algorithm>
