@@ -48,7 +48,16 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--grid-ctas", type=int, default=0)
-    ap.add_argument("--path", default="remap", choices=["remap", "pack_unpack", "extract"])
+    ap.add_argument("--path", default="remap",
+                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "extract"],
+                    help="remap: fused launch; pack_unpack: wb_pack + wb_unpack per round on one stream; "
+                         "rounds: wb_transfer_rounds (depth-2 buckets, two streams); rounds_serial: its "
+                         "unpipelined baseline; extract: source-map extraction kernel")
+    ap.add_argument("--budget-mib", type=int, default=0, help="bucket budget per round (0: the 4 GiB default)")
+    ap.add_argument("--budget-sweep", default="",
+                    help="comma-separated bucket budgets in MiB: time the pipelined and the serial rounds "
+                         "path for each and add the list to the JSON line (the buffer-size sensitivity "
+                         "experiment of the paper's Appendix D, on the kernels alone)")
     ap.add_argument("--static-schedule", action="store_true",
                     help="fixed per-block tile ranges instead of run-time batches")
     return ap.parse_args()
@@ -278,6 +287,7 @@ def main():
     tl = wb.Layout(wl.trainer.tensors, wl.trainer.slices)
     rl = wb.Layout(wl.rollout.tensors, wl.rollout.slices)
     plan = wb.Plan(tl, rl, tile_bytes=args.tile_bytes, grid_ctas=args.grid_ctas,
+                   bucket_budget_bytes=args.budget_mib << 20,
                    flags=wb.WB_PLAN_STATIC_SCHEDULE if args.static_schedule else 0)
     plan_s = time.perf_counter() - t0
     stats = plan.stats()
@@ -291,7 +301,7 @@ def main():
 
     n_rounds = plan.num_rounds()
     buckets = None
-    if args.path == "pack_unpack":
+    if args.path != "remap":
         buckets = [torch.empty(max(plan.bucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
                    for _ in range(2)]
 
@@ -299,6 +309,10 @@ def main():
         if args.path == "remap":
             plan.remap(stream)
             return 1
+        if args.path in ("rounds", "rounds_serial"):
+            plan.transfer_rounds(buckets[0].data_ptr(), buckets[1].data_ptr(),
+                                 wb.WB_ROUNDS_SERIAL if args.path == "rounds_serial" else 0, stream)
+            return 2 * n_rounds
         for r in range(n_rounds):
             b = buckets[r % 2].data_ptr()
             plan.pack(r, b, stream)
@@ -346,6 +360,32 @@ def main():
                 "traffic_source": "ncu on the large scale of this layout, scaled by bytes moved",
                 "peak_source": peak_src, "kernel": "wb_exec_kernel", "best_ms": float(min(per_step)),
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # ---- bucket budget sweep (rounds path) ---------------------------------------------------------
+    sweep = None
+    if args.budget_sweep and rank == 0 and world == 1:
+        sweep = []
+        del buckets
+        for mib in [int(x) for x in args.budget_sweep.split(",") if x]:
+            p2 = wb.Plan(tl, rl, tile_bytes=args.tile_bytes, grid_ctas=args.grid_ctas, bucket_budget_bytes=mib << 20)
+            bind(p2, src, dst)
+            nr = p2.num_rounds()
+            nb = max(p2.bucket_bytes(r) for r in range(nr))
+            bk = [torch.empty(nb, dtype=torch.uint8, device=dev) for _ in range(2)]
+            row = {"budget_mib": mib, "rounds": nr, "bucket_bytes": nb}
+            for key, flags in (("pipelined_ms", 0), ("serial_ms", wb.WB_ROUNDS_SERIAL)):
+                for _ in range(3):
+                    p2.transfer_rounds(bk[0].data_ptr(), bk[1].data_ptr(), flags, stream)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(args.steps):
+                    p2.transfer_rounds(bk[0].data_ptr(), bk[1].data_ptr(), flags, stream)
+                b.record()
+                torch.cuda.synchronize()
+                row[key] = a.elapsed_time(b) / args.steps
+            p2.check()
+            sweep.append(row)
+            del bk, p2
 
     # ---- end to end through the host-buffer entry point -------------------------------------------
     e2e = None
@@ -399,6 +439,8 @@ def main():
                           "multi_gpu": "independent replicas, no collective"},
                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                "gpu_launches": launches, "pct_of_8TBs_nominal": 100.0 * value / world / 8000.0}
+        if sweep is not None:
+            out["budget_sweep"] = sweep
         print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()

@@ -247,6 +247,22 @@ wb_status wb_plan_check_replicas(const wb_plan* plan, uint64_t* n_mismatches, vo
  * did not have to, CUDA / OOM on runtime errors.  The context stays usable afterwards. */
 wb_status wb_wait_probe(uint32_t limit_ms, void* cuda_stream);
 
+/* wb_transfer_rounds: every round of the two-pass path, pipelined (Section 3.2: "overlapping
+ * consecutive rounds"; Section 4: a depth-2 buffer system lets adjacent rounds proceed in
+ * parallel).  Round r packs into bucket r mod 2 on one internal stream and is assembled from it on
+ * a second internal stream; pack(r) waits until unpack(r-2) has released that bucket, unpack(r)
+ * waits for pack(r).  Equivalent to wb_pack + wb_unpack for rounds 0..R-1 in order; the rollout
+ * tensors end up as after wb_remap.  Work starts after what `cuda_stream` already holds and
+ * `cuda_stream` completes after the last assembly.  Returns without synchronising.
+ * bucket0 / bucket1: DEVICE, distinct, each >= max over rounds of wb_plan_bucket_bytes, 16-byte
+ * aligned, caller-owned.  flags: WB_ROUNDS_SERIAL runs pack(0), unpack(0), pack(1), ... on
+ * `cuda_stream` alone through bucket0 (bucket1 may be NULL) - the unpipelined baseline.
+ * Creates two streams and a few events on first use; not reentrant per plan (shares them with
+ * wb_remap_host).  Errors: INVALID_ARG, NOT_BOUND, CUDA, OOM. */
+#define WB_ROUNDS_SERIAL 1u
+wb_status wb_transfer_rounds(const wb_plan* plan, void* bucket0, void* bucket1, uint32_t flags,
+                             void* cuda_stream);
+
 /* wb_remap_host: the same transfer for callers whose weights are in HOST memory.  The remap
  * is cut into groups of consecutive tiles; for each group the trainer bytes it reads are copied
  * host -> bound device regions on an internal copy stream, its tiles run on `cuda_stream`, and the

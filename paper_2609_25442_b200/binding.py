@@ -78,7 +78,7 @@ EXPORTS = [
     "wb_layout_describe", "wb_layout_free", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
-    "wb_remap_host", "wb_remap_static", "wb_plan_check",
+    "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_transfer_rounds",
     "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
@@ -117,6 +117,7 @@ def load() -> C.CDLL:
     lib.wb_pack.argtypes = [vp, sz, vp, vp]
     lib.wb_unpack.argtypes = [vp, sz, vp, vp]
     lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
+    lib.wb_transfer_rounds.argtypes = [vp, vp, vp, C.c_uint32, vp]
     lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
     lib.wb_wait_probe.argtypes = [C.c_uint32, vp]
@@ -248,12 +249,16 @@ class Plan:
     def unpack(self, rnd: int, bucket_ptr: int, stream: int = 0) -> None:
         _check(_lib.wb_unpack(self.handle, rnd, bucket_ptr, stream), "wb_unpack")
 
+    def transfer_rounds(self, bucket0_ptr: int, bucket1_ptr: int, flags: int = 0, stream: int = 0) -> None:
+        _check(_lib.wb_transfer_rounds(self.handle, bucket0_ptr, bucket1_ptr, flags, stream), "wb_transfer_rounds")
+
     def remap_host(self, host_src_ptrs: Sequence[int], host_dst_ptrs: Sequence[int], stream: int = 0) -> None:
         a, b = _ptr_array(host_src_ptrs), _ptr_array(host_dst_ptrs)
         _check(_lib.wb_remap_host(self.handle, a, len(host_src_ptrs), b, len(host_dst_ptrs), stream),
                "wb_remap_host")
 
 
+WB_ROUNDS_SERIAL = 1
 WB_STATIC_SCRATCH_BYTES = 4 << 20
 WB_STATIC_SYNC_CHECK = 1
 

@@ -1178,6 +1178,79 @@ extern "C" wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bu
                       esize(plan->dst.dtype), esize(plan->dst.dtype), static_cast<cudaStream_t>(cuda_stream));
 }
 
+// Internal streams and events shared by the multi-stream entry points (created on first use,
+// destroyed with the device tables).
+static wb_status ensure_pipeline(wb_plan* plan, size_t n_events) {
+  if (!plan->h2d_stream) {
+    cudaStream_t a, b;
+    if (cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaStreamCreateWithFlags(&b, cudaStreamNonBlocking) != cudaSuccess) { cudaStreamDestroy(a); return WB_ERR_CUDA; }
+    plan->h2d_stream = a;
+    plan->d2h_stream = b;
+  }
+  while (plan->host_events.size() < n_events) {
+    cudaEvent_t e;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return WB_ERR_CUDA;
+    plan->host_events.push_back(e);
+  }
+  return WB_OK;
+}
+
+// wb_transfer_rounds: all rounds of the two-pass path with two buckets in flight (Section 3.2:
+// consecutive rounds overlap; Section 4: a depth-2 buffer system).  Packing runs on one internal
+// stream and assembly on another; pack(r) waits for unpack(r-2), which frees bucket r mod 2, and
+// unpack(r) waits for pack(r).  On one GPU the two persistent kernels compete for the same SMs, so
+// what overlaps is the tail of one launch with the head of the next.
+extern "C" wb_status wb_transfer_rounds(const wb_plan* plan_c, void* bucket0, void* bucket1, uint32_t flags,
+                                        void* cuda_stream) {
+  if (!plan_c || !bucket0 || ((uintptr_t)bucket0 & 15u) || (flags & ~WB_ROUNDS_SERIAL)) return WB_ERR_INVALID_ARG;
+  const bool serial = flags & WB_ROUNDS_SERIAL;
+  if (!serial && (!bucket1 || ((uintptr_t)bucket1 & 15u) || bucket1 == bucket0)) return WB_ERR_INVALID_ARG;
+  if (!plan_c->bound) return WB_ERR_NOT_BOUND;
+  wb_plan* plan = const_cast<wb_plan*>(plan_c);     // lazily built pipeline state, not the plan itself
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const uint32_t es = esize(plan->src.dtype), ed = esize(plan->dst.dtype);
+  const size_t R = plan->rounds.size();
+  if (R == 0) return WB_OK;
+  if (serial) {
+    for (size_t r = 0; r < R; ++r) {
+      wb_status st = launch_table(plan, plan->rounds[r].pack, 0, (uint64_t)(uintptr_t)bucket0, es, ed, stream);
+      if (st == WB_OK) st = launch_table(plan, plan->rounds[r].unpack, (uint64_t)(uintptr_t)bucket0, 0, ed, ed, stream);
+      if (st != WB_OK) return st;
+    }
+    return WB_OK;
+  }
+  try {
+    wb_status st = ensure_pipeline(plan, 2 * R + 1);
+    if (st != WB_OK) return st;
+    cudaStream_t ps = static_cast<cudaStream_t>(plan->h2d_stream), us = static_cast<cudaStream_t>(plan->d2h_stream);
+    auto packed = [&](size_t r) { return static_cast<cudaEvent_t>(plan->host_events[2 * r]); };
+    auto unpacked = [&](size_t r) { return static_cast<cudaEvent_t>(plan->host_events[2 * r + 1]); };
+    cudaEvent_t start = static_cast<cudaEvent_t>(plan->host_events[2 * R]);
+    // both internal streams start after whatever the caller already queued on its stream
+    if (cudaEventRecord(start, stream) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaStreamWaitEvent(ps, start, 0) != cudaSuccess) return WB_ERR_CUDA;
+    if (cudaStreamWaitEvent(us, start, 0) != cudaSuccess) return WB_ERR_CUDA;
+    for (size_t r = 0; r < R; ++r) {
+      const uint64_t bucket = (uint64_t)(uintptr_t)((r & 1) ? bucket1 : bucket0);
+      if (r >= 2 && cudaStreamWaitEvent(ps, unpacked(r - 2), 0) != cudaSuccess) return WB_ERR_CUDA;
+      st = launch_table(plan, plan->rounds[r].pack, 0, bucket, es, ed, ps);
+      if (st != WB_OK) return st;
+      if (cudaEventRecord(packed(r), ps) != cudaSuccess) return WB_ERR_CUDA;
+      if (cudaStreamWaitEvent(us, packed(r), 0) != cudaSuccess) return WB_ERR_CUDA;
+      st = launch_table(plan, plan->rounds[r].unpack, bucket, 0, ed, ed, us);
+      if (st != WB_OK) return st;
+      if (cudaEventRecord(unpacked(r), us) != cudaSuccess) return WB_ERR_CUDA;
+    }
+    // the caller's stream completes when the last assembly has (the assembly stream is in order
+    // and its last kernel waited for the last pack)
+    if (cudaStreamWaitEvent(stream, unpacked(R - 1), 0) != cudaSuccess) return WB_ERR_CUDA;
+  } catch (const std::bad_alloc&) {
+    return WB_ERR_OOM;
+  }
+  return WB_OK;
+}
+
 // wb_remap_host pipelines the transfer over PCIe: the remap table is cut into groups of
 // consecutive tiles; group g's source spans go host -> device on one copy stream, its tiles run
 // on the caller's stream, its destination spans go device -> host on a second copy stream, so
@@ -1249,18 +1322,7 @@ extern "C" wb_status wb_remap_host(const wb_plan* plan_c, const void* const* hos
   try {
     if (plan->host_groups.empty()) build_host_groups(plan);
     const size_t G = plan->host_groups.size();
-    if (!plan->h2d_stream) {
-      cudaStream_t a, b;
-      if (cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking) != cudaSuccess) return WB_ERR_CUDA;
-      if (cudaStreamCreateWithFlags(&b, cudaStreamNonBlocking) != cudaSuccess) { cudaStreamDestroy(a); return WB_ERR_CUDA; }
-      plan->h2d_stream = a;
-      plan->d2h_stream = b;
-    }
-    while (plan->host_events.size() < 2 * G + 2) {
-      cudaEvent_t e;
-      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return WB_ERR_CUDA;
-      plan->host_events.push_back(e);
-    }
+    { wb_status pst = ensure_pipeline(plan, 2 * G + 2); if (pst != WB_OK) return pst; }
     cudaStream_t up = static_cast<cudaStream_t>(plan->h2d_stream), down = static_cast<cudaStream_t>(plan->d2h_stream);
     auto ev = [&](size_t i) { return static_cast<cudaEvent_t>(plan->host_events[i]); };
     // the copy streams start after whatever the caller already queued on its stream

@@ -94,6 +94,43 @@ def test_pack_unpack_matches_oracle(device, name, scale, budget):
     assert_dst_equals(case, want)
 
 
+@pytest.mark.parametrize("name,scale,budget", [
+    ("cfg1", "full", 0), ("cfg1b", "full", 1 << 20), ("cfg3", "small", 1 << 20), ("cfg4", "small", 1 << 19),
+    ("cfg5", "small", 1 << 18), ("cfg2", "medium", 16 << 20), ("cfg3", "medium", 32 << 20),
+    ("cfg5", "medium", 16 << 20)])
+def test_pipelined_rounds_match_oracle(device, name, scale, budget):
+    """Depth-2 bucket pipeline (Section 3.2 / Section 4): all rounds through two buckets on two
+    internal streams give the same rollout tensors as the fused remap, on the caller's stream."""
+    wl = make_workload(name, scale)
+    case = DeviceCase(wl, device, bucket_budget_bytes=budget)
+    want = oracle_for(case)
+    n_rounds = case.plan.num_rounds()
+    if budget:
+        assert n_rounds > 2                     # the second use of a bucket is exercised
+    nb = max(case.plan.bucket_bytes(r) for r in range(n_rounds))
+    buckets = [torch.full((nb + 64,), 0x5A, dtype=torch.uint8, device=device) for _ in range(2)]
+    side = torch.cuda.Stream(device=device)
+    for flags, stream in [(0, None), (wb.WB_ROUNDS_SERIAL, None), (0, side), (0, side)]:
+        case.reset_dst()
+        torch.cuda.synchronize()
+        sp = 0 if stream is None else stream.cuda_stream
+        case.plan.transfer_rounds(buckets[0].data_ptr(), buckets[1].data_ptr(), flags, sp)
+        if stream is not None:
+            # back to back on the same stream: the second transfer is ordered after the first
+            case.plan.transfer_rounds(buckets[0].data_ptr(), buckets[1].data_ptr(), flags, sp)
+            stream.synchronize()                # the caller's stream alone covers all internal work
+        else:
+            torch.cuda.synchronize()
+        assert_dst_equals(case, want)
+        case.plan.check()
+        for b in buckets:
+            assert bool((b[nb:] == 0x5A).all())
+    with pytest.raises(wb.WbError):
+        case.plan.transfer_rounds(buckets[0].data_ptr(), buckets[0].data_ptr())     # one bucket twice
+    with pytest.raises(wb.WbError):
+        case.plan.transfer_rounds(buckets[0].data_ptr() + 2, buckets[1].data_ptr())  # misaligned
+
+
 @pytest.mark.parametrize("seed", range(160))
 def test_fuzz_layouts(device, seed):
     src_dt, dst_dt = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][seed % 4]

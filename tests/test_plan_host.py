@@ -274,6 +274,12 @@ def test_error_bucket_too_small_and_unbound_execution():
     plan = build(wl.trainer, wl.rollout)
     _expect("WB_ERR_NOT_BOUND", lambda: plan.remap())
     _expect("WB_ERR_INVALID_ARG", lambda: plan.pack(99, 16))
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.transfer_rounds(256, 512))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds(256, 256))       # one bucket given twice
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds(256, 0))         # second bucket missing
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds(258, 512))       # not 16-byte aligned
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds(256, 512, flags=8))
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.transfer_rounds(256, 0, flags=wb.WB_ROUNDS_SERIAL))
     _expect("WB_ERR_INVALID_ARG", lambda: plan.bind([0] * plan.n_src, [0] * plan.n_dst))
     lib = wb.load()
     assert lib.wb_remap(None, None) == 1
