@@ -28,92 +28,242 @@ template <> __device__ __forceinline__ long long field_at<WB_ID_BF16>(const void
   return (long long)__float2ll_rn(__uint_as_float(bits));
 }
 
-// A warp task is a strip of kStrip = 32*kV columns marched down up to kRowsPerTask rows.  Lane l
-// owns columns c0 + l + 32 k (k < kV), so each of its kV loads per row is a fully coalesced warp
-// access and all kV are in flight together.  The two values to the left of a column come from
-// lanes l-1 and l-2 by shuffle (from the previous k for lanes 0 and 1; from memory at the strip's
-// left edge), and the horizontal second difference h(i,j) = A(i,j) - 2 A(i,j-1) + A(i,j-2) of the
-// two rows above stays in registers, so diff2(i,j) = h(i,j) - 2 h(i-1,j) + h(i-2,j) costs one
-// global load per element (plus two halo rows per task).  Non-zeros are rare: a warp vote skips
-// the compaction for almost every row.
+// A warp task is a strip of kStrip = 32 * kQ * kG columns marched down up to kRowsPerTask rows.
+// In each of the kG groups a lane owns kQ = 4 adjacent columns, c0 + 128 g + 4 l + {0..3}, which it
+// fetches with one or two vector loads, so only its leftmost two columns need values from another
+// lane (one rotating shuffle per group hands lane l-1's last two columns to lane l; lane 0 takes
+// the strip's left halo in group 0 and what the rotation brought round from lane 31 after that).
+//
+// diff2 is separable.  The kernel applies the vertical second difference first,
+//   v(i,j) = A(i,j) - 2 A(i-1,j) + A(i-2,j),      diff2(i,j) = v(i,j) - 2 v(i,j-1) + v(i,j-2),
+// because v needs no other lane (the two rows above stay in registers) and vanishes wherever three
+// consecutive rows belong to one slice-copy operation: a warp vote then skips the horizontal step
+// for almost every row.  A field with a single row (a flat shard) has v = A and goes straight to
+// the horizontal step.  The loads of the next row visit (the next row, or the first row of the
+// warp's next task) are issued before the current row is consumed.
 constexpr int kRowsPerTask = 64;
-constexpr int kV = 8;
+constexpr int kQ = 4;
+constexpr int kG = 2;
+constexpr int kV = kQ * kG;
 constexpr int kStrip = 32 * kV;
 
-template <int KIND>
-__device__ __forceinline__ void row_h(const void* field, unsigned long long row_base, unsigned long long cols,
-                                      unsigned long long c0, unsigned lane, long long h[kV]) {
+template <int KIND> struct FieldElem;
+template <> struct FieldElem<WB_ID_I64> { static constexpr int kBytes = 8; };
+template <> struct FieldElem<WB_ID_U16> { static constexpr int kBytes = 2; };
+template <> struct FieldElem<WB_ID_F32> { static constexpr int kBytes = 4; };
+template <> struct FieldElem<WB_ID_BF16> { static constexpr int kBytes = 2; };
+
+__device__ __forceinline__ long long bf16_bits_to_ll(unsigned int b) {
+  return (long long)__float2ll_rn(__uint_as_float(b << 16));
+}
+
+// Four adjacent elements starting at element index idx, the address known to be aligned for the
+// vector access of the kind.
+template <int KIND> __device__ __forceinline__ void load_quad(const void* f, unsigned long long idx, long long x[kQ]);
+template <> __device__ __forceinline__ void load_quad<WB_ID_I64>(const void* f, unsigned long long idx, long long x[kQ]) {
+  const longlong2* p = reinterpret_cast<const longlong2*>(static_cast<const long long*>(f) + idx);
+  const longlong2 a = __ldg(p), b = __ldg(p + 1);
+  x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+}
+template <> __device__ __forceinline__ void load_quad<WB_ID_U16>(const void* f, unsigned long long idx, long long x[kQ]) {
+  const uint2 a = __ldg(reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(f) + idx));
+  x[0] = a.x & 0xFFFFu; x[1] = a.x >> 16; x[2] = a.y & 0xFFFFu; x[3] = a.y >> 16;
+}
+template <> __device__ __forceinline__ void load_quad<WB_ID_F32>(const void* f, unsigned long long idx, long long x[kQ]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(f) + idx));
+  x[0] = __float2ll_rn(a.x); x[1] = __float2ll_rn(a.y); x[2] = __float2ll_rn(a.z); x[3] = __float2ll_rn(a.w);
+}
+template <> __device__ __forceinline__ void load_quad<WB_ID_BF16>(const void* f, unsigned long long idx, long long x[kQ]) {
+  const uint2 a = __ldg(reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(f) + idx));
+  x[0] = bf16_bits_to_ll(a.x & 0xFFFFu); x[1] = bf16_bits_to_ll(a.x >> 16);
+  x[2] = bf16_bits_to_ll(a.y & 0xFFFFu); x[3] = bf16_bits_to_ll(a.y >> 16);
+}
+
+// One row of a strip as a lane holds it: its kV elements and (lane 0) the two elements left of
+// the strip.
+struct RowRegs {
   long long a[kV];
+  long long e1, e2;                                            // A[c0-1], A[c0-2]
+};
+
+template <int KIND>
+__device__ __forceinline__ void row_load(const void* field, unsigned long long row_base, unsigned long long cols,
+                                         unsigned long long c0, unsigned lane, RowRegs& r) {
+  // vector accesses need the quad's first element on a multiple of the vector size; every quad of
+  // a row starts at a column that is a multiple of 4, so one test covers the row
+  constexpr unsigned long long kVecElems = FieldElem<KIND>::kBytes == 8 ? 2 : 4;
+  const unsigned long long first = (unsigned long long)(reinterpret_cast<uintptr_t>(field) / FieldElem<KIND>::kBytes) + row_base;
+  const bool vec = first % kVecElems == 0;
 #pragma unroll
-  for (int k = 0; k < kV; ++k) {
-    const unsigned long long c = c0 + lane + 32u * k;
-    a[k] = c < cols ? field_at<KIND>(field, row_base + c) : 0;
-  }
-  // halo: the two columns left of the strip (read by lanes 0 and 1, both end up needing them)
-  long long e1 = 0, e2 = 0;                                  // A[c0-1], A[c0-2]
-  if (lane < 2) {
-    if (c0 >= 1) e1 = field_at<KIND>(field, row_base + c0 - 1);
-    if (c0 >= 2) e2 = field_at<KIND>(field, row_base + c0 - 2);
-  }
-  long long prev30 = e2, prev31 = e1;                          // "lanes 30 / 31 of k-1"; uniform per warp below
-  prev30 = __shfl_sync(0xFFFFFFFFu, prev30, 0);
-  prev31 = __shfl_sync(0xFFFFFFFFu, prev31, 0);
+  for (int g = 0; g < kG; ++g) {
+    const unsigned long long c = c0 + 128u * g + 4u * lane;
+    if (vec && c + kQ <= cols) {
+      load_quad<KIND>(field, row_base + c, &r.a[kQ * g]);
+    } else {
 #pragma unroll
-  for (int k = 0; k < kV; ++k) {
-    long long l1 = __shfl_up_sync(0xFFFFFFFFu, a[k], 1), l2 = __shfl_up_sync(0xFFFFFFFFu, a[k], 2);
-    if (lane == 0) { l1 = prev31; l2 = prev30; }
-    if (lane == 1) l2 = prev31;
-    h[k] = a[k] - 2 * l1 + l2;
-    prev30 = __shfl_sync(0xFFFFFFFFu, a[k], 30);
-    prev31 = __shfl_sync(0xFFFFFFFFu, a[k], 31);
+      for (int q = 0; q < kQ; ++q) r.a[kQ * g + q] = c + q < cols ? field_at<KIND>(field, row_base + c + q) : 0;
+    }
+  }
+  r.e1 = r.e2 = 0;
+  if (lane == 0) {
+    if (c0 >= 1) r.e1 = field_at<KIND>(field, row_base + c0 - 1);
+    if (c0 >= 2) r.e2 = field_at<KIND>(field, row_base + c0 - 2);
   }
 }
 
-template <int KIND>
-__global__ void __launch_bounds__(256)
-wb_diff2_kernel(const void* __restrict__ field, unsigned long long rows, unsigned long long cols,
-                wb_diff2_entry* __restrict__ out, unsigned long long cap, unsigned long long* __restrict__ count) {
-  const unsigned lane = threadIdx.x & 31;
-  const unsigned long long strips = (cols + kStrip - 1) / kStrip, blocks = (rows + kRowsPerTask - 1) / kRowsPerTask;
-  const unsigned long long n_tasks = strips * blocks;
-  const unsigned long long warp0 = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const unsigned long long n_warps = ((unsigned long long)gridDim.x * blockDim.x) >> 5;
-  for (unsigned long long task = warp0; task < n_tasks; task += n_warps) {
-    const unsigned long long rb = task / strips, cs = task - rb * strips;   // neighbouring warps: neighbouring strips
-    const unsigned long long i0 = rb * kRowsPerTask;
-    const unsigned long long i1 = i0 + kRowsPerTask < rows ? i0 + kRowsPerTask : rows;
-    const unsigned long long c0 = cs * kStrip;
-    long long hm1[kV], hm2[kV];
+// Horizontal second difference of one row of values v (with halo ve1 = v[c0-1], ve2 = v[c0-2] in
+// lane 0), and compaction of its non-zero entries.
+__device__ __forceinline__ void emit_row(const long long v[kV], long long ve1, long long ve2, unsigned long long row,
+                                         unsigned long long c0, unsigned long long cols, unsigned lane,
+                                         wb_diff2_entry* __restrict__ out, unsigned long long cap,
+                                         unsigned long long* __restrict__ count) {
+  const unsigned from = (lane + 31u) & 31u;
+  long long carry1 = ve1, carry2 = ve2;                        // lane 0: the two values left of the group
 #pragma unroll
-    for (int k = 0; k < kV; ++k) hm1[k] = hm2[k] = 0;
-    if (i0 >= 2) row_h<KIND>(field, (i0 - 2) * cols, cols, c0, lane, hm2);
-    if (i0 >= 1) row_h<KIND>(field, (i0 - 1) * cols, cols, c0, lane, hm1);
-    for (unsigned long long i = i0; i < i1; ++i) {
-      long long h[kV], d[kV];
-      row_h<KIND>(field, i * cols, cols, c0, lane, h);
-      long long any = 0;
+  for (int g = 0; g < kG; ++g) {
+    const long long* x = &v[kQ * g];
+    long long l1 = __shfl_sync(0xFFFFFFFFu, x[3], from), l2 = __shfl_sync(0xFFFFFFFFu, x[2], from);
+    if (lane == 0) {                                           // received lane 31's pair: the next group's halo
+      const long long n1 = l1, n2 = l2;
+      l1 = carry1; l2 = carry2;
+      carry1 = n1; carry2 = n2;
+    }
+    long long d[kQ];
+    d[0] = x[0] - 2 * l1 + l2;
+    d[1] = x[1] - 2 * x[0] + l1;
+    d[2] = x[2] - 2 * x[1] + x[0];
+    d[3] = x[3] - 2 * x[2] + x[1];
+    const unsigned long long c = c0 + 128u * g + 4u * lane;
+    int n = 0;
 #pragma unroll
-      for (int k = 0; k < kV; ++k) {
-        d[k] = (c0 + lane + 32u * k < cols) ? h[k] - 2 * hm1[k] + hm2[k] : 0;
-        hm2[k] = hm1[k];
-        hm1[k] = h[k];
-        any |= d[k];
+    for (int q = 0; q < kQ; ++q) {
+      if (c + q >= cols) d[q] = 0;
+      n += d[q] != 0;
+    }
+    if (!__any_sync(0xFFFFFFFFu, n != 0)) continue;
+    // exclusive prefix of the lanes' counts, one atomic for the warp
+    int incl = n;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= (unsigned)o) incl += t;
+    }
+    const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    unsigned long long slot0 = 0;
+    if (lane == 0) slot0 = atomicAdd(count, (unsigned long long)total);
+    slot0 = __shfl_sync(0xFFFFFFFFu, slot0, 0);
+    unsigned long long slot = slot0 + (unsigned)(incl - n);
+#pragma unroll
+    for (int q = 0; q < kQ; ++q)
+      if (d[q] != 0) {
+        if (slot < cap) out[slot] = wb_diff2_entry{row, c + q, d[q]};
+        ++slot;
       }
-      if (__any_sync(0xFFFFFFFFu, any != 0)) {
+  }
+}
+
+// The sequence of row visits of a warp: for each of its tasks the two rows above the task, which
+// only prime the registers (rows -2 and -1 of the field read as zeros), then the task's own rows.
+struct Visit {
+  unsigned long long task;
+  int row, i0, i1;                                             // fields with several rows: rows, cols < 2^31
+  unsigned c0;
+};
+
+__device__ __forceinline__ void visit_begin(Visit& v, unsigned long long task, unsigned strips, unsigned rows,
+                                            unsigned rows_per_task) {
+  const unsigned long long rb = task / strips;                 // neighbouring warps: neighbouring strips
+  v.task = task;
+  v.i0 = (int)((unsigned)rb * rows_per_task);
+  v.i1 = (unsigned)v.i0 + rows_per_task < rows ? (int)((unsigned)v.i0 + rows_per_task) : (int)rows;
+  v.c0 = (unsigned)(task - rb * strips) * kStrip;
+  v.row = v.i0 - 2;
+}
+
+template <int KIND>
+__device__ __forceinline__ void visit_load(const void* field, const Visit& v, unsigned long long cols, unsigned lane,
+                                           RowRegs& r) {
+  if (v.row >= 0) {
+    row_load<KIND>(field, (unsigned long long)v.row * cols, cols, v.c0, lane, r);
+  } else {
+#pragma unroll
+    for (int k = 0; k < kV; ++k) r.a[k] = 0;
+    r.e1 = r.e2 = 0;
+  }
+}
+
+// The rows a warp holds live in a ring of register sets addressed by the position in an unrolled
+// loop (current row, the row being fetched and the two rows above), so advancing a row moves no registers.
+template <int KIND>
+__global__ void __launch_bounds__(256, 2)
+wb_diff2_kernel(const void* __restrict__ field, unsigned long long rows, unsigned long long cols,
+                unsigned long long rows_per_task, wb_diff2_entry* __restrict__ out, unsigned long long cap,
+                unsigned long long* __restrict__ count) {
+  constexpr int kRing = 4;
+  const unsigned lane = threadIdx.x & 31;
+  const unsigned strips = (unsigned)((cols + kStrip - 1) / kStrip);
+  const unsigned long long n_tasks = (unsigned long long)strips * ((rows + rows_per_task - 1) / rows_per_task);
+  const unsigned long long warp0 = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const unsigned n_warps = (gridDim.x * blockDim.x) >> 5;
+  if (warp0 >= n_tasks) return;
+  Visit v, w;
+  visit_begin(v, warp0, strips, (unsigned)rows, (unsigned)rows_per_task);
+  RowRegs R[kRing];
+  visit_load<KIND>(field, v, cols, lane, R[0]);
+  for (;;) {
+#pragma unroll
+    for (int s = 0; s < kRing; ++s) {
+      const RowRegs& cur = R[s];
+      w = v;                                                   // the visit after this one
+      bool more = true;
+      if (++w.row == w.i1) {
+        more = w.task + n_warps < n_tasks;
+        if (more) visit_begin(w, w.task + n_warps, strips, (unsigned)rows, (unsigned)rows_per_task);
+      }
+      if (more) visit_load<KIND>(field, w, cols, lane, R[(s + 1) % kRing]);
+      if (v.row >= v.i0) {
+        const RowRegs& p1 = R[(s + kRing - 1) % kRing];
+        const RowRegs& p2 = R[(s + kRing - 2) % kRing];
+        long long vv[kV];
+        bool nz = false;
 #pragma unroll
         for (int k = 0; k < kV; ++k) {
-          const unsigned mask = __ballot_sync(0xFFFFFFFFu, d[k] != 0);
-          if (!mask) continue;
-          unsigned long long slot0 = 0;
-          if (lane == 0) slot0 = atomicAdd(count, (unsigned long long)__popc(mask));
-          slot0 = __shfl_sync(0xFFFFFFFFu, slot0, 0);
-          if (d[k] != 0) {
-            const unsigned long long slot = slot0 + __popc(mask & ((1u << lane) - 1));
-            if (slot < cap) out[slot] = wb_diff2_entry{i, c0 + lane + 32u * k, d[k]};
-          }
+          vv[k] = cur.a[k] - 2 * p1.a[k] + p2.a[k];
+          nz |= vv[k] != 0;
         }
+        const long long ve1 = cur.e1 - 2 * p1.e1 + p2.e1, ve2 = cur.e2 - 2 * p1.e2 + p2.e2;
+        nz |= (ve1 | ve2) != 0;
+        if (__any_sync(0xFFFFFFFFu, nz))
+          emit_row(vv, ve1, ve2, (unsigned long long)v.row, v.c0, cols, lane, out, cap, count);
       }
+      if (!more) return;
+      v = w;
     }
+  }
+}
+
+// A field with one row (a flat shard): diff2 is the second difference along the row, every task is
+// one strip, and a warp alternates between two register sets so that the next strip is in flight
+// while the current one is consumed.
+template <int KIND>
+__global__ void __launch_bounds__(256, 3)
+wb_diff2_row_kernel(const void* __restrict__ field, unsigned long long cols, wb_diff2_entry* __restrict__ out,
+                    unsigned long long cap, unsigned long long* __restrict__ count) {
+  const unsigned lane = threadIdx.x & 31;
+  const unsigned long long stride = (((unsigned long long)gridDim.x * blockDim.x) >> 5) * kStrip;
+  unsigned long long c0 = ((((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5)) * kStrip;
+  if (c0 >= cols) return;
+  RowRegs r0, r1;
+  row_load<KIND>(field, 0, cols, c0, lane, r0);
+  for (;;) {
+    const unsigned long long c1 = c0 + stride;
+    if (c1 < cols) row_load<KIND>(field, 0, cols, c1, lane, r1);
+    emit_row(r0.a, r0.e1, r0.e2, 0, c0, cols, lane, out, cap, count);
+    if (c1 >= cols) return;
+    c0 = c1 + stride;
+    if (c0 < cols) row_load<KIND>(field, 0, cols, c0, lane, r0);
+    emit_row(r1.a, r1.e1, r1.e2, 0, c1, cols, lane, out, cap, count);
+    if (c0 >= cols) return;
   }
 }
 
@@ -124,16 +274,35 @@ extern "C" wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint
   if (!field || !count || (!out && cap) || id_kind > WB_ID_BF16) return WB_ERR_INVALID_ARG;
   if (rows == 0 || cols == 0) return WB_OK;
   if (rows > (1ull << 40) || cols > (1ull << 40) || rows * cols > (1ull << 48)) return WB_ERR_INVALID_ARG;
+  if (rows > 1 && (rows >= (1ull << 31) || cols >= (1ull << 31))) return WB_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const unsigned long long tasks = ((cols + kStrip - 1) / kStrip) * ((rows + kRowsPerTask - 1) / kRowsPerTask);
-  const unsigned long long want = (tasks + 7) / 8;                 // 8 warps per block
-  const unsigned grid = (unsigned)(want < 148ull * 8 ? want : 148ull * 8);
-  auto* cnt = reinterpret_cast<unsigned long long*>(count);
-  switch (id_kind) {
-    case WB_ID_I64: wb_diff2_kernel<WB_ID_I64><<<grid, 256, 0, stream>>>(field, rows, cols, out, cap, cnt); break;
-    case WB_ID_U16: wb_diff2_kernel<WB_ID_U16><<<grid, 256, 0, stream>>>(field, rows, cols, out, cap, cnt); break;
-    case WB_ID_F32: wb_diff2_kernel<WB_ID_F32><<<grid, 256, 0, stream>>>(field, rows, cols, out, cap, cnt); break;
-    default: wb_diff2_kernel<WB_ID_BF16><<<grid, 256, 0, stream>>>(field, rows, cols, out, cap, cnt); break;
+  // Tasks are dealt to warps round robin, so the rows per task are chosen to give every warp the
+  // same number of tasks (about kRowsPerTask rows each) instead of leaving a last, partly filled turn.
+  const unsigned long long strips = (cols + kStrip - 1) / kStrip;
+  const unsigned long long resident = 148ull * (rows == 1 ? 3 : 2);   // blocks the registers let an SM hold
+  const unsigned long long n_warps = resident * 8;                      // 8 warps per block
+  unsigned long long rows_per_task = rows < (unsigned long long)kRowsPerTask ? rows : kRowsPerTask;
+  if (strips * ((rows + rows_per_task - 1) / rows_per_task) > n_warps) {
+    unsigned long long turns = (strips * rows + n_warps * kRowsPerTask / 2) / (n_warps * kRowsPerTask);
+    if (turns == 0) turns = 1;
+    const unsigned long long row_blocks = (turns * n_warps) / strips;   // tasks <= turns * n_warps
+    if (row_blocks >= 1) rows_per_task = (rows + row_blocks - 1) / row_blocks;
   }
+  const unsigned long long tasks = strips * ((rows + rows_per_task - 1) / rows_per_task);
+  const unsigned long long want = (tasks + 7) / 8;
+  const unsigned grid = (unsigned)(want < resident ? want : resident);
+  auto* cnt = reinterpret_cast<unsigned long long*>(count);
+#define WB_DIFF2_LAUNCH(KIND)                                                                         \
+  do {                                                                                               \
+    if (rows == 1) wb_diff2_row_kernel<KIND><<<grid, 256, 0, stream>>>(field, cols, out, cap, cnt);   \
+    else wb_diff2_kernel<KIND><<<grid, 256, 0, stream>>>(field, rows, cols, rows_per_task, out, cap, cnt);   \
+  } while (0)
+  switch (id_kind) {
+    case WB_ID_I64: WB_DIFF2_LAUNCH(WB_ID_I64); break;
+    case WB_ID_U16: WB_DIFF2_LAUNCH(WB_ID_U16); break;
+    case WB_ID_F32: WB_DIFF2_LAUNCH(WB_ID_F32); break;
+    default: WB_DIFF2_LAUNCH(WB_ID_BF16); break;
+  }
+#undef WB_DIFF2_LAUNCH
   return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
 }

@@ -137,3 +137,20 @@ def test_scan_rejects_fields_no_slice_copy_produces():
     with pytest.raises(wb.WbError) as e:
         wb.wb_scan_slices(far, 8, 8, base, one, one, 0)
     assert e.value.name == "WB_ERR_OUT_OF_RANGE"
+
+
+def test_diff2_kernel_entry_point_checks_its_arguments_on_the_host():
+    """Size limits are refused before anything is launched (no GPU needed to see them)."""
+    lib = wb.load()
+    import ctypes as C
+    lib.wb_diff2_nonzeros.argtypes = [C.c_void_p, C.c_uint32, C.c_uint64, C.c_uint64, C.c_void_p, C.c_uint64,
+                                      C.c_void_p, C.c_void_p]
+    dummy = C.c_uint64(0)
+    p = C.addressof(dummy)
+    INVALID = 1
+    assert lib.wb_diff2_nonzeros(None, 0, 4, 4, p, 1, p, None) == INVALID
+    assert lib.wb_diff2_nonzeros(p, 9, 4, 4, p, 1, p, None) == INVALID              # unknown field kind
+    assert lib.wb_diff2_nonzeros(p, 0, 1 << 31, 2, p, 1, p, None) == INVALID        # several rows: < 2^31 rows
+    assert lib.wb_diff2_nonzeros(p, 0, 2, 1 << 31, p, 1, p, None) == INVALID
+    assert lib.wb_diff2_nonzeros(p, 0, 1, (1 << 48) + 1, p, 1, p, None) == INVALID
+    assert lib.wb_diff2_nonzeros(p, 0, 0, 4, p, 1, p, None) == 0                    # empty field: nothing to do

@@ -51,6 +51,55 @@ def test_diff2_kernel_matches_the_definition(shape):
     assert n == len(want) and np.array_equal(got, want)
 
 
+def _piecewise_affine(shape, rng, n_rect=8):
+    a = np.zeros(shape, np.int64)
+    for _ in range(n_rect):
+        i0, j0 = rng.integers(0, shape[0]), rng.integers(0, shape[1])
+        ni, nj = rng.integers(1, shape[0] - i0 + 1), rng.integers(1, shape[1] - j0 + 1)
+        a[i0:i0 + ni, j0:j0 + nj] = (int(rng.integers(1, 1 << 40)) + np.arange(ni)[:, None] * int(rng.integers(1, 1 << 20))
+                                     + np.arange(nj)[None, :])
+    return a
+
+
+def test_diff2_kernel_on_a_field_of_many_row_blocks():
+    """More (strip, row block) tasks than resident warps: the rows per task are rebalanced, warps walk
+    several tasks each, and rectangle edges fall on every position relative to the task seams."""
+    rng = np.random.default_rng(77)
+    a = _piecewise_affine((40000, 1100), rng, n_rect=24)
+    for i in (0, 1, 2, 63, 64, 65, 84, 85, 86, 169, 170, 39999):        # isolated entries around likely seams
+        a[i, rng.integers(0, 1100)] += int(rng.integers(1, 1 << 30))
+    want = oracle_entries(a)
+    got, n = gpu_entries(torch.from_numpy(a).to(DEV), wb.WB_ID_I64, cap=1 << 18)
+    assert n == len(want) and np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("shape", [(1, 4099), (1, 4096), (9, 514), (9, 515), (130, 260)])
+@pytest.mark.parametrize("skew", [1, 2, 3])
+def test_diff2_kernel_at_any_alignment_of_the_field(shape, skew):
+    """Fields that start `skew` elements into an allocation: rows whose first element is not on the
+    boundary the vector loads want take the element-wise loads, with the same result."""
+    rng = np.random.default_rng(shape[0] * 7 + shape[1] + skew)
+    a = _piecewise_affine(shape, rng)
+    n = a.size
+    want = oracle_entries(a)
+    buf = torch.zeros(n + 8, dtype=torch.int64, device=DEV)
+    buf[skew:skew + n] = torch.from_numpy(a.reshape(-1)).to(DEV)
+    got, cnt = gpu_entries(buf[skew:skew + n].view(*shape), wb.WB_ID_I64)
+    assert cnt == len(want) and np.array_equal(got, want)
+    # 16-bit chunks of the same field, as raw bits
+    c16 = id_chunk(a, 0, 16)
+    b16 = torch.zeros(n + 8, dtype=torch.int16, device=DEV)
+    b16[skew:skew + n] = torch.from_numpy(c16.astype(np.uint16).view(np.int16).reshape(-1)).to(DEV)
+    got16, _ = gpu_entries(b16[skew:skew + n].view(*shape), wb.WB_ID_U16, 1 << 17)
+    assert np.array_equal(got16, oracle_entries(c16))
+    # 24-bit chunks held in fp32
+    c24 = id_chunk(a, 0, 24)
+    b32 = torch.zeros(n + 8, dtype=torch.float32, device=DEV)
+    b32[skew:skew + n] = torch.from_numpy(c24.astype(np.float32).reshape(-1)).to(DEV)
+    got32, _ = gpu_entries(b32[skew:skew + n].view(*shape), wb.WB_ID_F32, 1 << 17)
+    assert np.array_equal(got32, oracle_entries(c24))
+
+
 def test_diff2_kernel_reads_chunks_in_the_parameter_dtypes():
     rng = np.random.default_rng(5)
     ids = rng.integers(1, 1 << 34, size=(61, 517)).astype(np.int64)
