@@ -248,6 +248,19 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+
+// Per-thread asynchronous 16-byte copy global -> shared (both 16-byte aligned), and the arrival that
+// signals an mbarrier once all earlier copies of the calling thread have landed (the pending count
+// is raised by the instruction itself, so the barrier's initial count is not involved).
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+template <int OFF> __device__ __forceinline__ void cp_async16_at(uint32_t smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0+%2], [%1+%2], 16;" ::"r"(smem_dst), "l"(gsrc), "n"(OFF) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.shared.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
@@ -294,7 +307,21 @@ constexpr int kWorkerWarps = kWorkers / 32;
 #endif
 constexpr size_t kStagedMinRowBytes = WB_STAGED_MIN_ROW_BYTES;   // shorter rows take the warp-level path
 
-enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3 };
+enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3, MODE_TRANS = 4 };
+// Staged transposition: a chunk is up to kTransPiece - 16 bytes of consecutive source columns (the
+// 16-byte aligned superset of a row piece is one 16-byte asynchronous copy per lane of the producer
+// warp - bulk copies this small are limited by their issue rate) by as many source rows as fit a slot.  Row r of the chunk lands at r * kTransPitch + 16 * ((r / NV) & 7) in the slot
+// (NV = destination elements per 16 bytes): the pitch is a multiple of 128 bytes, so lanes that
+// read the same column NV rows apart - neighbouring 16-byte windows of one destination run - hit
+// different banks.  kTransHalo rows past the chunk's own rows complete its last window.
+constexpr uint32_t kTransPiece = 512;                      // bytes one warp instruction copies per row (aligned superset)
+constexpr uint32_t kTransPitch = kTransPiece + 128;
+constexpr uint32_t kTransHalo = 8;
+#ifndef WB_TRANS_MIN_PIECE
+#define WB_TRANS_MIN_PIECE 256
+#endif
+constexpr uint32_t kTransMinPiece = WB_TRANS_MIN_PIECE;   // narrower tiles stay with the warp-level transposition
+constexpr uint32_t kTransMinRows = 16;
 #ifndef WB_BATCH_TILE_BYTES
 #define WB_BATCH_TILE_BYTES 8192
 #endif
@@ -304,10 +331,10 @@ constexpr uint32_t kBatchMaxTiles = 120;
 // What the producer tells the workers about one ring slot.
 struct ChunkDesc {
   uint32_t mode;
-  uint32_t tile;      // MODE_COOP: index of the tile to run
+  uint32_t tile;      // MODE_COOP / MODE_BATCH: index of the (first) tile to run; MODE_TRANS: the chunk's own rows
   uint32_t nr, nc;    // staged chunk: rows in the stage, elements per row
   uint32_t pitch;     // bytes between rows in the stage
-  uint32_t pad;
+  uint32_t pad;       // MODE_TRANS: 1 if the chunk holds the first rows of its destination runs
   uint64_t src;       // global address of the chunk's first source element (alignment arithmetic only)
   uint64_t dst;       // global address of the chunk's first destination element
   uint64_t sps;       // source row pitch in bytes
@@ -433,6 +460,24 @@ template <int ES, int ED> __device__ __forceinline__ typename Elem<ES, ED>::V ca
   else if constexpr (ES == 4) return f32_to_bf16(raw);
   else return raw << 16;
 }
+// Shared-memory word accesses at a compile-time offset from a 32-bit shared-space address, and a
+// loop over compile-time indices (so that unrolled code uses immediate offsets).
+template <int OFF> __device__ __forceinline__ uint32_t lds32_at(uint32_t base) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(base), "n"(OFF));
+  return v;
+}
+template <int OFF> __device__ __forceinline__ void sts32_at(uint32_t base, uint32_t v) {
+  asm volatile("st.shared.u32 [%0+%1], %2;" ::"r"(base), "n"(OFF), "r"(v));
+}
+template <int I> struct Idx { static constexpr int value = I; };
+template <int I, int N, typename F> __device__ __forceinline__ void static_for(F&& fn) {
+  if constexpr (I < N) {
+    fn(Idx<I>{});
+    static_for<I + 1, N>(fn);
+  }
+}
+
 // two consecutive 2-byte destination elements packed in one word
 template <int ES> __device__ __forceinline__ uint32_t pack_pair16(uint32_t lo, uint32_t hi) {
   if constexpr (ES == 4) return f32x2_to_bf16x2(lo, hi);
@@ -445,8 +490,8 @@ template <int ES> __device__ __forceinline__ uint32_t pack_pair16(uint32_t lo, u
 //            load instruction, 16 loads in flight per lane, one batch ahead), casts, and writes
 //            each value into its private patch of the ring slot, laid out as destination rows:
 //            T[lane][row].
-//   phase B  lane = destination run.  A run may start at any 2-/4-byte alignment in global memory;
-//            it is written in 16-byte aligned windows.  A block owns the windows that START in its
+//   phase B  A run may start at any 2-/4-byte alignment in global memory; it is written in 16-byte
+//            aligned windows, neighbouring lanes taking neighbouring windows of a run.  A block owns the windows that START in its
 //            rows and reads up to NV-1 rows past its end to complete the last one, so neighbouring
 //            blocks never share a window and almost every store is a full vector; only the two
 //            ends of a whole run use element stores.
@@ -463,7 +508,9 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
   // (multiple of 8, at most 64); no halo is needed when every run starts on a 16-byte boundary
   const uint32_t share = patch_bytes / 4;                    // words
   const bool aligned = (((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0;
-  const uint32_t halo = aligned ? 0u : NV - 1, room = aligned ? 0u : 8u;
+  // rows read past a block's end to complete its last window: NV-1 are needed; with 2-byte
+  // destinations 8 are read, which keeps the row count of a whole block a multiple of UA
+  const uint32_t halo = aligned ? 0u : (ED == 2 ? 8u : NV - 1), room = aligned ? 0u : 8u;
   const uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD - room) & ~7u);
   const uint32_t pitch_w = (rb + room) / PER_WORD + 1;      // odd: (rb+room)/PER_WORD is even
   const uint32_t tbase = smem_u32(patch);
@@ -472,15 +519,28 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
   const size_t sps = (size_t)f.ssr * ES;
   if (warp >= nb) return;
 
-  struct Block { uint32_t i0, j0, ni, nj, nl; };      // nl: rows loaded = own rows + halo
+  // nl: rows loaded = own rows + halo.  full: every lane has a column and every batch all its rows,
+  // so loads and shared-memory writes need no predicates; whole: in addition the block has all its
+  // rows and halo and does not begin a run, so every window it owns is a full vector.
+  struct Block { uint32_t i0, j0, ni, nj, nl; bool full, whole; };
   auto block_of = [&](uint32_t b) {
     const uint32_t bi = b / nbj, bj = b - bi * nbj;
     const uint32_t i0 = bi * rb, ni = min(rb, f.nr - i0);
-    return Block{i0, bj * 32, ni, min(32u, f.nc - bj * 32), min(ni + halo, f.nr - i0)};
+    const uint32_t nj = min(32u, f.nc - bj * 32), nl = min(ni + halo, f.nr - i0);
+    const bool full = nj == 32 && nl % UA == 0;
+    return Block{i0, bj * 32, ni, nj, nl, full, full && nl == rb + halo && (aligned || i0 != 0)};
   };
   // phase A, loads: UA rows of this lane's column into registers
   auto issue = [&](const Block& k, uint32_t r0, uint32_t (&dst)[UA]) {
     const char* src = f.s + ((size_t)(k.i0 + r0) * f.ssr + k.j0 + lane) * ES;
+    if (k.full) {
+#pragma unroll
+      for (int u = 0; u < UA; ++u, src += sps) {
+        if constexpr (ES == 4) dst[u] = __ldcs(reinterpret_cast<const uint32_t*>(src));
+        else dst[u] = __ldcs(reinterpret_cast<const uint16_t*>(src));
+      }
+      return;
+    }
 #pragma unroll
     for (int u = 0; u < UA; ++u) {
       dst[u] = 0;
@@ -494,6 +554,20 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
   auto consume = [&](const Block& k, uint32_t r0, const uint32_t (&v)[UA]) {
     if (lane >= k.nj) return;
     const uint32_t trow = tbase + lane * pitch_w * 4;
+    if (k.full) {
+      const uint32_t at = trow + r0 * ED;
+      if constexpr (ED == 2)
+        static_for<0, UA / 2>([&](auto uc) {
+          constexpr int u = decltype(uc)::value * 2;
+          sts32_at<u * 2>(at, pack_pair16<ES>(v[u], v[u + 1]));
+        });
+      else
+        static_for<0, UA>([&](auto uc) {
+          constexpr int u = decltype(uc)::value;
+          sts32_at<u * 4>(at, (uint32_t)cast_raw<ES, ED>(v[u]));
+        });
+      return;
+    }
     if constexpr (ED == 2) {
 #pragma unroll
       for (int u = 0; u < UA; u += 2)
@@ -506,58 +580,109 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
           asm volatile("st.shared.u32 [%0], %1;" ::"r"(trow + (r0 + u) * 4), "r"((uint32_t)cast_raw<ES, ED>(v[u])));
     }
   };
-  // phase B: lane j writes destination run j -- the 16-byte windows that start inside the block's rows
+  // phase B: the block's 16-byte windows (those that start inside its rows), numbered run by run,
+  // are dealt to the lanes in order, so neighbouring lanes write neighbouring windows of one
+  // destination run and a store instruction touches a few whole lines instead of 32 scattered
+  // 16-byte pieces.
   auto phase_b = [&](const Block& k) {
     __syncwarp();
-    if (lane < k.nj) {
-      char* run = f.d + (size_t)(k.j0 + lane) * f.dsc * ED;       // element (j, 0) of the run
+    if (k.whole) {
+      // lane = destination run; rb / NV full windows, the first one `lead` rows into the block
+      char* run = f.d + (size_t)(k.j0 + lane) * f.dsc * ED;
+      const uint32_t a = (uint32_t)(((uintptr_t)run / ED + k.i0) & (NV - 1));
+      const uint32_t lead = a ? NV - a : 0;
+      char* out = run + (size_t)(k.i0 + lead) * ED;
+      const uint32_t trow = tbase + lane * pitch_w * 4;
+      if constexpr (ED == 4) {
+        uint32_t p = trow + lead * 4;
+        for (uint32_t w = 0; w < rb / NV; ++w, p += 16, out += 16)
+          st16(out, make_uint4(lds32_at<0>(p), lds32_at<4>(p), lds32_at<8>(p), lds32_at<12>(p)));
+      } else if (aligned) {
+        uint32_t p = trow;
+        for (uint32_t w = 0; w < rb / NV; ++w, p += 16, out += 16)
+          st16(out, make_uint4(lds32_at<0>(p), lds32_at<4>(p), lds32_at<8>(p), lds32_at<12>(p)));
+      } else {
+        uint32_t p = trow + (lead >> 1) * 4;
+        const uint32_t sh = (lead & 1u) * 16u;                     // odd lead: windows straddle the words
+        for (uint32_t w = 0; w < rb / NV; ++w, p += 16, out += 16) {
+          const uint32_t w0 = lds32_at<0>(p), w1 = lds32_at<4>(p), w2 = lds32_at<8>(p), w3 = lds32_at<12>(p),
+                         w4 = lds32_at<16>(p);
+          st16(out, make_uint4(__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh),
+                               __funnelshift_r(w2, w3, sh), __funnelshift_r(w3, w4, sh)));
+        }
+      }
+      __syncwarp();
+      return;
+    }
+    const uint32_t wins = (k.ni + NV - 1) / NV;                    // windows per run, at most
+    const uint32_t total = k.nj * wins;
+    for (uint32_t idx = lane; idx < total; idx += 32) {
+      const uint32_t j = idx / wins, w = idx - j * wins;
+      char* run = f.d + (size_t)(k.j0 + j) * f.dsc * ED;            // element (j, 0) of the run
       const uint32_t a = (uint32_t)(((uintptr_t)run / ED + k.i0) & (NV - 1));   // offset of row i0 in its window
       const uint32_t lead = a ? NV - a : 0;                        // rows before the first window that starts here
-      const uint32_t trow = tbase + lane * pitch_w * 4;
+      const uint32_t trow = tbase + j * pitch_w * 4;
       // those rows belong to the previous block's last window, except at the very start of the run
-      if (k.i0 == 0)
+      if (w == 0 && k.i0 == 0)
         for (uint32_t e = 0; e < min(lead, k.ni); ++e)
           E::store(run + (size_t)e * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
-      char* out = run + (size_t)(k.i0 + lead) * ED;               // 16-byte aligned
-      for (uint32_t e0 = lead; e0 < k.ni; e0 += NV, out += 16) {
-        if (e0 + NV <= k.nl) {
-          uint4 x;
-          if constexpr (ED == 4) {
-            x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
-            x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
-          } else {
-            const uint32_t p = trow + (e0 >> 1) * 4;
-            const uint32_t w0 = lds_raw<4>(p), w1 = lds_raw<4>(p + 4), w2 = lds_raw<4>(p + 8), w3 = lds_raw<4>(p + 12);
-            if (e0 & 1) {
-              const uint32_t w4 = lds_raw<4>(p + 16);
-              x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
-                             __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
-            } else {
-              x = make_uint4(w0, w1, w2, w3);
-            }
-          }
-          st16(out, x);
+      const uint32_t e0 = lead + w * NV;
+      if (e0 >= k.ni) continue;
+      char* out = run + (size_t)(k.i0 + e0) * ED;                  // 16-byte aligned
+      if (e0 + NV <= k.nl) {
+        uint4 x;
+        if constexpr (ED == 4) {
+          x.x = lds_raw<4>(trow + (e0 + 0) * 4); x.y = lds_raw<4>(trow + (e0 + 1) * 4);
+          x.z = lds_raw<4>(trow + (e0 + 2) * 4); x.w = lds_raw<4>(trow + (e0 + 3) * 4);
         } else {
-          // the run ends inside this window
-          for (uint32_t e = e0; e < k.nl; ++e)
-            E::store(run + (size_t)(k.i0 + e) * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
+          const uint32_t p = trow + (e0 >> 1) * 4;
+          const uint32_t w0 = lds_raw<4>(p), w1 = lds_raw<4>(p + 4), w2 = lds_raw<4>(p + 8), w3 = lds_raw<4>(p + 12);
+          if (e0 & 1) {
+            const uint32_t w4 = lds_raw<4>(p + 16);
+            x = make_uint4(__funnelshift_r(w0, w1, 16), __funnelshift_r(w1, w2, 16),
+                           __funnelshift_r(w2, w3, 16), __funnelshift_r(w3, w4, 16));
+          } else {
+            x = make_uint4(w0, w1, w2, w3);
+          }
         }
+        st16(out, x);
+      } else {
+        // the run ends inside this window
+        for (uint32_t e = e0; e < k.nl; ++e)
+          E::store(run + (size_t)(k.i0 + e) * ED, (typename E::V)lds_raw<ED>(trow + e * ED));
       }
     }
     __syncwarp();
   };
 
+  // The rows of a block are short pieces (128 bytes) a row pitch apart, and a lane holds only two
+  // batches of loads, which is not enough memory parallelism to cover DRAM latency.  So the warp asks
+  // for the block after next to be brought into L2 ahead of time (lane = row; every sector of the
+  // piece): that costs no registers, and the loads then hit L2.
+  auto prefetch = [&](uint32_t pb) {
+#ifndef WB_NO_TRANS_PREFETCH
+    if (pb >= nb) return;
+    const Block k = block_of(pb);
+    for (uint32_t r = lane; r < k.nl; r += 32) {
+      const char* row = f.s + ((size_t)(k.i0 + r) * f.ssr + k.j0) * ES;
+      const uint32_t bytes = k.nj * ES;                             // one request per 32-byte sector
+      for (uint32_t o = 0; o < bytes; o += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + o));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(row + bytes - 1));
+    }
+#endif
+  };
   // The warp's batches in order; the loads of batch q+1 are issued before batch q is consumed, so
   // they are in flight during the shared-memory writes and during phase B.
   uint32_t b = warp, r0 = 0;
   Block blk = block_of(b);
+  prefetch(b + nw);
   auto step = [&](uint32_t (&cur)[UA], uint32_t (&nxt)[UA]) -> bool {
     uint32_t b2 = b, r2 = r0 + UA;
     Block blk2 = blk;
     const bool same = r2 < blk.nl;
     if (!same) { b2 = b + nw; r2 = 0; }
     const bool more = same || b2 < nb;
-    if (!same && more) blk2 = block_of(b2);
+    if (!same && more) { blk2 = block_of(b2); prefetch(b2 + nw); }
     if (more) issue(blk2, r2, nxt);
     consume(blk, r0, cur);
     if (!same) phase_b(blk);
@@ -685,6 +810,60 @@ __device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __res
   }
 }
 
+// Workers: a staged transposition chunk (rows of the source in shared memory, see kTransPitch)
+// -> destination runs, dst[j*dps + i] = cast(chunk[i][j]).  A run may start at any 2-/4-byte
+// alignment in global memory; it is written in 16-byte aligned windows.  The chunk owns the windows
+// that START in its own rows and uses the halo rows to complete the last one, so neighbouring
+// chunks never share a window; only the two ends of a whole run use element stores.  Windows are
+// numbered run by run and dealt to the threads in order: neighbouring lanes write neighbouring
+// windows of one run (whole lines per store instruction) and read different banks.
+template <int ES, int ED>
+__device__ __forceinline__ void staged_trans(const ChunkDesc& d, const char* stage, uint32_t t) {
+  using E = Elem<ES, ED>;
+  constexpr uint32_t NV = 16 / ED;
+  const uint32_t own = d.tile, nl = d.nr;
+  const uint32_t wins = (own + NV - 1) / NV;                   // windows per run, at most
+  const uint32_t total = d.nc * wins;
+  const uint32_t lead0 = (uint32_t)d.src & 15u, dlead = (uint32_t)d.sps & 15u;
+  const uint32_t sbase = smem_u32(stage);
+  constexpr uint32_t kSwzShift = ED == 2 ? 1 : 2;               // ((i / NV) & 7) << 4 == (i << shift) & 0x70
+  auto elem = [&](uint32_t i, uint32_t j) -> uint32_t {         // raw source element (i, j) of the chunk
+    return lds_raw<ES>(sbase + i * kTransPitch + ((i << kSwzShift) & 0x70u) + ((lead0 + i * dlead) & 15u) + j * ES);
+  };
+  const bool pow2 = (wins & (wins - 1)) == 0;
+  const uint32_t wshift = 31u - __clz(wins);
+  for (uint32_t idx = t; idx < total; idx += (uint32_t)kWorkers) {
+    const uint32_t j = pow2 ? idx >> wshift : idx / wins, w = idx - j * wins;
+    const uint64_t run = d.dst + (uint64_t)j * d.dps;           // destination element (j, first own row)
+    const uint32_t a = (uint32_t)(run / ED) & (NV - 1);
+    const uint32_t lead = a ? NV - a : 0;                       // rows before the first window that starts here
+    // those rows belong to the previous chunk's last window, except at the very start of the run
+    if (w == 0 && d.pad)
+      for (uint32_t e = 0; e < min(lead, own); ++e)
+        E::store(reinterpret_cast<char*>(run) + (size_t)e * ED, cast_raw<ES, ED>(elem(e, j)));
+    const uint32_t e0 = lead + w * NV;
+    if (e0 >= own) continue;
+    char* out = reinterpret_cast<char*>(run) + (size_t)e0 * ED;   // 16-byte aligned
+    if (e0 + NV <= nl) {
+      uint32_t v[NV];
+#pragma unroll
+      for (uint32_t k = 0; k < NV; ++k) v[k] = elem(e0 + k, j);
+      uint4 x;
+      if constexpr (ED == 2)
+        x = make_uint4(pack_pair16<ES>(v[0], v[1]), pack_pair16<ES>(v[2], v[3]), pack_pair16<ES>(v[4], v[5]),
+                       pack_pair16<ES>(v[6], v[7]));
+      else
+        x = make_uint4((uint32_t)cast_raw<ES, ED>(v[0]), (uint32_t)cast_raw<ES, ED>(v[1]),
+                       (uint32_t)cast_raw<ES, ED>(v[2]), (uint32_t)cast_raw<ES, ED>(v[3]));
+      st16(out, x);
+    } else {
+      // the run ends inside this window
+      for (uint32_t e = e0; e < nl; ++e)
+        E::store(out + (size_t)(e - e0) * ED, cast_raw<ES, ED>(elem(e, j)));
+    }
+  }
+}
+
 // Error codes written to the plan's device error word.
 enum : uint32_t { ERR_NONE = 0, ERR_WAIT_LOAD = 1, ERR_WAIT_SLOT_EMPTY = 2, ERR_WAIT_SLOT_FULL = 3 };
 
@@ -742,6 +921,10 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
       if (tr >= (uint32_t)kWorkers) tr -= kWorkers;
       if (d.mode == MODE_ROWS) {
         staged_rows<ES, ED>(d, stage, tr);
+      } else if (d.mode == MODE_TRANS) {
+#ifndef WB_TRANS_SKIP_WORK
+        staged_trans<ES, ED>(d, stage, tr);
+#endif
       } else {
         // queued tiles: one big tile shared by all worker warps, or a run of small tiles with one
         // warp per tile
@@ -818,6 +1001,38 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
       bulk_load(stage + (size_t)r * pitch, reinterpret_cast<const void*>(a & ~(uintptr_t)15),
                 roundup16((uint32_t)(a & 15u) + n * ES), &slot_full[slot]);
     }
+    ++n_w;
+  };
+  // stage a transposition chunk: R row pieces of n elements, one warp-wide asynchronous copy per row
+  auto push_trans = [&](const char* src, char* dst, uint32_t R, uint32_t n, uint64_t sps, uint64_t dps,
+                        uint32_t own, uint32_t first) {
+    if (!acquire_slot()) return;
+    const uint32_t slot = n_w % kSlots;
+    const uint32_t stage = smem_u32(wring + (size_t)slot * kSlotBytes);
+    if (lane == 0) {
+      ChunkDesc c;
+      c.mode = MODE_TRANS; c.tile = own; c.nr = R; c.nc = n; c.pitch = kTransPitch; c.pad = first;
+      c.src = (uint64_t)(uintptr_t)src; c.dst = (uint64_t)(uintptr_t)dst; c.sps = sps; c.dps = dps;
+      desc[slot] = c;
+    }
+    // Four lanes per row, eight rows per step: a lane copies every fourth 16-byte unit of its row
+    // (immediate offsets), so the address arithmetic is paid once per eight rows.  This loop is the
+    // producer's critical path: one warp feeds the whole block.
+    constexpr uint32_t kSwzShift = ED == 2 ? 1 : 2;               // ((r / NV) & 7) << 4 == (r << shift) & 0x70
+    const uint32_t nbytes = n * ES, q16 = (lane & 3u) * 16u;
+    for (uint32_t r = lane >> 2; r < R; r += 8) {
+      const uintptr_t a = (uintptr_t)src + (uint64_t)r * sps;
+      const uint32_t need = (uint32_t)(a & 15u) + nbytes;         // bytes of the aligned superset that are needed
+      const char* g = reinterpret_cast<const char*>(a & ~(uintptr_t)15) + q16;
+      const uint32_t sm = stage + r * kTransPitch + ((r << kSwzShift) & 0x70u) + q16;
+      static_for<0, (int)(kTransPiece / 64)>([&](auto kc) {
+        constexpr int off = decltype(kc)::value * 64;
+        if (q16 + (uint32_t)off < need) cp_async16_at<off>(sm, g);
+      });
+    }
+    cp_async_arrive(&slot_full[slot]);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&slot_full[slot]);   // after every lane's pending arrival is counted
     ++n_w;
   };
   // direct ring (lane 0): store the oldest loaded chunk; one store behind, its stage is free again
@@ -914,8 +1129,19 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
             push_staged(MODE_ROWS, f.s + ((size_t)r * f.ssr + c) * ES, f.d + ((size_t)r * f.dsr + c) * ED, 1,
                         min(piece, f.nc - c), 0, 0, (uint32_t)kSlotBytes);
       }
+    } else if (f.kind == KIND_TRANS && f.n_extra == 0 && (size_t)f.nc * ES >= kTransMinPiece && f.nr >= kTransMinRows) {
+      // staged transposition: chunks of kTransPiece bytes of columns x kOwn rows (+ halo), rows fastest
+      constexpr uint32_t kOwn = (((uint32_t)kSlotBytes / kTransPitch) - kTransHalo) & ~7u;
+      constexpr uint32_t kCols = (kTransPiece - 16) / ES;
+      // no halo when every destination run starts on a 16-byte boundary: windows never straddle chunks
+      const uint32_t halo = ((((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0 && kOwn % (16 / ED) == 0) ? 0u : kTransHalo;
+      for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += kCols)
+        for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += kOwn)
+          push_trans(f.s + ((size_t)i0 * f.ssr + j0) * ES, f.d + ((size_t)j0 * f.dsc + i0) * ED,
+                     min(kOwn + halo, f.nr - i0), min(kCols, f.nc - j0), (uint64_t)f.ssr * ES,
+                     (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0), i0 == 0 ? 1u : 0u);
     } else {
-      push_simple(MODE_COOP, k);          // transposes, short rows, fan-out: the workers share the tile
+      push_simple(MODE_COOP, k);          // narrow transposes, short rows, fan-out: the workers share the tile
     }
   }
   flush_run();          // runs do not cross scheduling batches: tile indices must stay consecutive

@@ -209,7 +209,9 @@ struct TileBuilder {
     }
     const uint32_t kind = trans ? KIND_TRANS : KIND_ELEM;
     // 2-D blocks, multiples of 64 on both axes where the extent allows
-    uint64_t tc = std::min<uint64_t>(nc, 512);
+    // 496 columns: a whole number of the executor's staged transposition chunks (124 four-byte or
+    // 248 two-byte source elements each)
+    uint64_t tc = std::min<uint64_t>(nc, trans ? 496 : 512);
     uint64_t tr = std::min<uint64_t>(nr, std::max<uint64_t>(64, roundup(T / tc, 64)));
     for (uint64_t i = 0; i < nr; i += tr)
       for (uint64_t j = 0; j < nc; j += tc)
