@@ -314,7 +314,10 @@ enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3, MO
 // (NV = destination elements per 16 bytes): the pitch is a multiple of 128 bytes, so lanes that
 // read the same column NV rows apart - neighbouring 16-byte windows of one destination run - hit
 // different banks.  kTransHalo rows past the chunk's own rows complete its last window.
-constexpr uint32_t kTransPiece = 512;                      // bytes one warp instruction copies per row (aligned superset)
+#ifndef WB_TRANS_PIECE
+#define WB_TRANS_PIECE 512
+#endif
+constexpr uint32_t kTransPiece = WB_TRANS_PIECE;                      // bytes one warp instruction copies per row (aligned superset)
 constexpr uint32_t kTransPitch = kTransPiece + 128;
 constexpr uint32_t kTransHalo = 8;
 #ifndef WB_TRANS_MIN_PIECE
@@ -1003,7 +1006,7 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     }
     ++n_w;
   };
-  // stage a transposition chunk: R row pieces of n elements, one warp-wide asynchronous copy per row
+  // stage a transposition chunk: R row pieces of n elements, four lanes per row
   auto push_trans = [&](const char* src, char* dst, uint32_t R, uint32_t n, uint64_t sps, uint64_t dps,
                         uint32_t own, uint32_t first) {
     if (!acquire_slot()) return;
