@@ -11,13 +11,16 @@
 //            global through a small ring; the data never touches registers.
 //   staged   other ROWS tiles with rows of at least kStagedMinRowBytes: the producer warp bulk-
 //            loads the rows into a ring slot, the workers realign, cast and store 16 bytes at a time.
+//   staged   transposing tiles: the producer warp copies chunks of source rows into a ring slot
+//   transp.  (per-lane asynchronous copies, bank-swizzled rows), the workers write 16-byte windows
+//            of the destination runs, neighbouring lanes on neighbouring windows of one run.
 //   queued   everything else is handed to the workers by tile index, either one tile shared by all
 //            worker warps or a run of small tiles, one warp per tile.
 //
 // Tile kinds
 //   ROWS   nr runs of nc contiguous elements on both sides (nr == 1: one long run).
-//   TRANS  source contiguous along j, destination contiguous along i: each warp transposes
-//          32-column blocks through a private shared-memory patch.
+//   TRANS  source contiguous along j, destination contiguous along i: staged transposition, or
+//          (narrow tiles) each warp transposes 32-column blocks through a private patch.
 //   ELEM   anything else (strided vectors, fan-out to several destinations): element loop.
 //
 // Every wait in the kernel is bounded (see mbar_wait); a wait that runs out sets the plan's error
