@@ -239,6 +239,46 @@ def test_unaligned_runs(device, src_off, dst_off, dts):
         assert (got[:dst_off] == (0xCDCD if dts[1] == WB_BF16 else 0xCDCDCDCD)).all()
 
 
+TRANS_SHAPES = [(16, 64), (17, 65), (15, 300), (40, 124), (41, 125), (63, 123), (64, 124), (65, 125), (71, 247),
+                (72, 248), (73, 249), (64, 496), (129, 497), (200, 1000), (333, 130), (1, 700), (700, 1), (8, 2048)]
+
+
+@pytest.mark.parametrize("dts", [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)])
+@pytest.mark.parametrize("skew", [(0, 0, 0), (1, 3, 0), (2, 5, 7), (4, 8, 4)])
+def test_transposition_shapes(device, dts, skew):
+    """dst[j, i] = cast(src[i, j]) for shapes on both sides of every block and chunk size of the
+    transposing paths, with the source starting `so` elements into its tensor, the destination `do`,
+    and the source rows `extra` elements longer than the part that is moved (so row starts fall on
+    every alignment).  The oracle is numpy's transpose of the seeded bits; the element before and
+    after every destination must keep the canary."""
+    so, do, extra = skew
+    for (R, C) in TRANS_SHAPES:
+        pitch = C + extra
+        tl, rl = Layout("t"), Layout("r")
+        tl.add_tensor("T", 0, dts[0], so + R * pitch)
+        # the source matrix is the left C columns of a wider [R, pitch] matrix, which is checkpoint tensor 0
+        tl.add_slice(0, so, pitch, 1, 0, R, pitch, 0, 0, R, pitch)
+        rl.add_tensor("R", 0, dts[1], do + R * C + 3)
+        rl.add_slice(0, do, 1, R, 0, R, pitch, 0, 0, R, C)        # checkpoint (i, j) -> local do + j*R + i
+        tl.freeze(); rl.freeze()
+        plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices))
+        src = RankArenas(tl.tensors, device, fill_byte=0)
+        dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+        bind(plan, src, dst)
+        rng = np.random.default_rng(R * 1000 + C)
+        bits = random_bits(rng, so + R * pitch, dts[0])
+        src.tensors[0].copy_(from_bits(bits).to(device))
+        plan.remap()
+        torch.cuda.synchronize()
+        plan.check()
+        got = to_bits(dst.tensors[0])
+        m = bits[so:].reshape(R, pitch)[:, :C]
+        want = cast_bits(np.ascontiguousarray(m.T).reshape(-1), dts[0], dts[1])
+        assert np.array_equal(got[do:do + R * C], want), (R, C)
+        canary = 0xCDCD if dts[1] == WB_BF16 else 0xCDCDCDCD
+        assert (got[:do] == canary).all() and (got[do + R * C:] == canary).all(), (R, C)
+
+
 def test_inverse_remap_restores_the_trainer(device):
     wl = make_workload("cfg1b")
     tl, rl = wl.trainer.swapped_dtype(WB_BF16), wl.rollout.swapped_dtype(WB_BF16)
