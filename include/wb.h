@@ -211,7 +211,10 @@ wb_status wb_plan_tiles(const wb_plan* plan, int which, size_t round, wb_tile_vi
  * src_base[i] / dst_base[i]: DEVICE address of trainer / rollout local tensor i, aligned to
  * its element size (16-byte alignment lets the kernels use their widest path).  Host
  * arrays of device pointers, copied.  May be called again to re-bind.  The bound regions
- * must not alias each other.  Errors: INVALID_ARG, OOM, CUDA. */
+ * must not alias each other.  The kernels fetch whole 16-byte units: they may READ (never write)
+ * the up to 15 bytes between a run's first / last element and the enclosing 16-byte boundaries,
+ * which always lie inside the same device allocation (allocations are at least 256-byte granular).
+ * Errors: INVALID_ARG, OOM, CUDA. */
 wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, size_t n_src,
                        void* const* dst_base, size_t n_dst);
 
