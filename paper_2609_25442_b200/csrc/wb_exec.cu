@@ -345,6 +345,7 @@ struct ChunkDesc {
   uint64_t dst;       // global address of the chunk's first destination element
   uint64_t sps;       // source row pitch in bytes
   uint64_t dps;       // destination pitch in bytes: between rows (ROWS) or between columns (TRANS)
+  uint4 raw[3];       // MODE_COOP: the tile's descriptor, so that the workers need not fetch it from global memory
 };
 
 __device__ __forceinline__ uint32_t roundup16(uint32_t x) { return (x + 15u) & ~15u; }
@@ -940,8 +941,13 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
         // every warp owns one fixed part of the slot as scratch, whatever kind of tile it runs
         constexpr uint32_t kPatchBytes = ((uint32_t)kSlotBytes / kWorkerWarps) & ~15u;
         char* patch = const_cast<char*>(stage) + warp * kPatchBytes;
-        for (uint32_t k = d.tile + (run ? warp : 0u); k < d.tile + d.nr; k += run ? (uint32_t)kWorkerWarps : 1u) {
-          const TileFields f = decode(load_tile(tiles + k), src_add, dst_add);
+        const uint32_t k0 = d.tile + (run ? warp : 0u), kend = d.tile + d.nr, kstep = run ? (uint32_t)kWorkerWarps : 1u;
+        TileRegs regs;
+        if (!run) { regs.a = d.raw[0]; regs.b = d.raw[1]; regs.c = d.raw[2]; }
+        else if (k0 < kend) regs = load_tile(tiles + k0);
+        for (uint32_t k = k0; k < kend; k += kstep) {
+          const TileFields f = decode(regs, src_add, dst_add);
+          if (k + kstep < kend) regs = load_tile(tiles + k + kstep);    // the next descriptor is on its way meanwhile
           if (f.n_extra == 0 && f.kind == KIND_TRANS) {
             warp_transpose<ES, ED>(f, patch, kPatchBytes, w, nw, lane);
           } else if (f.n_extra == 0 && f.kind == KIND_ROWS && (f.nr == 1 || (size_t)f.nc * ES >= kStagedMinRowBytes)) {
@@ -973,13 +979,14 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     if (!ok) { if (lane == 0) atomicMax(err, ERR_WAIT_SLOT_EMPTY); failed = true; }
     return ok != 0;
   };
-  auto push_simple = [&](uint32_t mode, uint32_t tile, uint32_t count = 1) {
+  auto push_simple = [&](uint32_t mode, uint32_t tile, uint32_t count = 1, const TileRegs* regs = nullptr) {
     if (!acquire_slot()) return;
     const uint32_t slot = n_w % kSlots;
     if (lane == 0) {
       desc[slot].mode = mode;
       desc[slot].tile = tile;
       desc[slot].nr = count;
+      if (regs) { desc[slot].raw[0] = regs->a; desc[slot].raw[1] = regs->b; desc[slot].raw[2] = regs->c; }
       mbar_arrive(&slot_full[slot]);    // release: the descriptor is visible to whoever sees the phase
     }
     ++n_w;
@@ -1093,7 +1100,8 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
   while (!failed && next_batch()) {
   TileRegs nxt = load_tile(tiles + bk);
   for (uint32_t k = bk; k < bend && !failed; ++k) {
-    const TileFields f = decode(nxt, src_add, dst_add);
+    const TileRegs cur = nxt;
+    const TileFields f = decode(cur, src_add, dst_add);
     if (k + 1 < bend) nxt = load_tile(tiles + k + 1);
     // small tiles are handed over in runs and executed one warp per tile
     if ((uint64_t)f.nr * f.nc * (ES + ED * (1 + f.n_extra)) < kBatchTileBytes && !direct_ok<ES, ED>(f)) {
@@ -1147,7 +1155,7 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
                      min(kOwn + halo, f.nr - i0), min(kCols, f.nc - j0), (uint64_t)f.ssr * ES,
                      (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0), i0 == 0 ? 1u : 0u);
     } else {
-      push_simple(MODE_COOP, k);          // narrow transposes, short rows, fan-out: the workers share the tile
+      push_simple(MODE_COOP, k, 1, &cur);   // narrow transposes, short rows, fan-out: the workers share the tile
     }
   }
   flush_run();          // runs do not cross scheduling batches: tile indices must stay consecutive
