@@ -475,11 +475,34 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
     {
       TileBuilder tb{&P->remap, es, ed, P->opts.tile_bytes};
       Ref src; std::vector<Ref> dsts;
+      // Tiles of one checkpoint tensor are emitted slab by slab; they are then ordered by the address
+      // of their strided side (rows a pitch apart: several slabs cut the same rows into column
+      // pieces), so that tiles which touch the same rows, lines and DRAM pages run close in time.
+      std::vector<std::pair<size_t, size_t>> ranges;     // [first, last) tile of each checkpoint tensor
+      uint32_t cur_ckpt = UINT32_MAX;
       for (const Slab& sl : P->slabs) {
+        if (sl.ckpt_index != cur_ckpt) {
+          if (!ranges.empty()) ranges.back().second = P->remap.tiles.size();
+          ranges.push_back({P->remap.tiles.size(), 0});
+          cur_ckpt = sl.ckpt_index;
+        }
         slab_refs(sl, sl.rect, &src, &dsts);
         tb.add(src, dsts, sl.rect.nr, sl.rect.nc);
       }
+      if (!ranges.empty()) ranges.back().second = P->remap.tiles.size();
       if (!tb.ok) return fail(WB_ERR_INVALID_ARG);
+#ifndef WB_NO_TILE_ORDER
+      for (auto& rg : ranges) {
+        auto key = [](const HTile& t) {
+          // 0: source rows strided, by source address; 1: destination strided, by destination address; 2: as emitted
+          if (t.kind == KIND_ROWS && t.nr > 1 && t.ssr > t.nc) return std::make_tuple(0, (int64_t)t.src_tensor, t.src_off);
+          if (t.kind == KIND_ROWS && t.nr > 1 && t.dsr > t.nc) return std::make_tuple(1, (int64_t)t.dst_tensor, t.dst_off);
+          return std::make_tuple(2, (int64_t)0, (uint64_t)0);
+        };
+        std::stable_sort(P->remap.tiles.begin() + rg.first, P->remap.tiles.begin() + rg.second,
+                         [&](const HTile& a, const HTile& b) { return key(a) < key(b); });
+      }
+#endif
       assign_ctas(&P->remap, P->grid);
     }
 
