@@ -209,10 +209,18 @@ struct TileBuilder {
     }
     const uint32_t kind = trans ? KIND_TRANS : KIND_ELEM;
     // 2-D blocks, multiples of 64 on both axes where the extent allows
-    // 496 columns: a whole number of the executor's staged transposition chunks (124 four-byte or
-    // 248 two-byte source elements each)
-    uint64_t tc = std::min<uint64_t>(nc, trans ? 496 : 512);
+    // transposed: one staged transposition chunk of the executor wide (496 source bytes) and as tall
+    // as the tile size allows, so that a tile writes long pieces of few destination runs and the
+    // element stores at the two ends of a run piece are rare
+    uint64_t tc = std::min<uint64_t>(nc, trans ? 496 / es : 512);
     uint64_t tr = std::min<uint64_t>(nr, std::max<uint64_t>(64, roundup(T / tc, 64)));
+    if (trans) {
+      // rows fastest: consecutive tiles continue the same destination runs
+      for (uint64_t j = 0; j < nc; j += tc)
+        for (uint64_t i = 0; i < nr; i += tr)
+          emit(src, dsts.data(), n_dst, i, j, std::min(tr, nr - i), std::min(tc, nc - j), kind);
+      return;
+    }
     for (uint64_t i = 0; i < nr; i += tr)
       for (uint64_t j = 0; j < nc; j += tc)
         emit(src, dsts.data(), n_dst, i, j, std::min(tr, nr - i), std::min(tc, nc - j), kind);
