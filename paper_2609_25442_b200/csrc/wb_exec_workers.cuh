@@ -38,7 +38,7 @@ template <int ES, int ED> struct Rings {      // worker ring: staged chunks and 
 };
 constexpr int kWorkerWarps = kWorkers / 32;
 #ifndef WB_STAGED_MIN_ROW_BYTES
-#define WB_STAGED_MIN_ROW_BYTES 1024
+#define WB_STAGED_MIN_ROW_BYTES 512
 #endif
 constexpr size_t kStagedMinRowBytes = WB_STAGED_MIN_ROW_BYTES;   // shorter rows take the warp-level path
 
@@ -56,7 +56,7 @@ constexpr uint32_t kTransPiece = WB_TRANS_PIECE;                      // bytes o
 constexpr uint32_t kTransPitch = kTransPiece + 128;
 constexpr uint32_t kTransHalo = 8;
 #ifndef WB_TRANS_MIN_PIECE
-#define WB_TRANS_MIN_PIECE 256
+#define WB_TRANS_MIN_PIECE 128
 #endif
 constexpr uint32_t kTransMinPiece = WB_TRANS_MIN_PIECE;   // narrower tiles stay with the warp-level transposition
 constexpr uint32_t kTransMinRows = 16;
