@@ -38,7 +38,7 @@ template <int ES, int ED> struct Rings {      // worker ring: staged chunks and 
 };
 constexpr int kWorkerWarps = kWorkers / 32;
 #ifndef WB_STAGED_MIN_ROW_BYTES
-#define WB_STAGED_MIN_ROW_BYTES 512
+#define WB_STAGED_MIN_ROW_BYTES 1024
 #endif
 constexpr size_t kStagedMinRowBytes = WB_STAGED_MIN_ROW_BYTES;   // shorter rows take the warp-level path
 
