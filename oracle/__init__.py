@@ -17,6 +17,12 @@ Pins (see tests marked "not gpu"):
                           remap identity.
   remap.checkpoint_view   equality with the seeded checkpoint tensors the trainer
                           buffers were loaded from.
+  quant.e4m3_encode / e4m3_decode / quantize / dequantize
+                          (Section 5 sketches pre-transfer quantisation and fixes no rule: the
+                          rule is a reading of ours, parity unpinned by the paper) format definition
+                          in exact rationals, torch's CPU float8_e4m3fn table and cast inside the
+                          finite range, brute-force nearest-even over all codes incl. every
+                          midpoint, saturation and NaN table, scale rule and round-trip bound.
   The order of payloads inside a transfer bucket and the rule that picks which trainer
   replica supplies a replicated element are planner choices the paper does not fix:
   parity unpinned by the paper, checked only against the directory the library reports
