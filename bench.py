@@ -49,10 +49,11 @@ def parse_args():
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--grid-ctas", type=int, default=0)
     ap.add_argument("--path", default="remap",
-                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "extract"],
+                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "rounds_fp8", "extract"],
                     help="remap: fused launch; pack_unpack: wb_pack + wb_unpack per round on one stream; "
                          "rounds: wb_transfer_rounds (depth-2 buckets, two streams); rounds_serial: its "
-                         "unpipelined baseline; extract: source-map extraction kernel")
+                         "unpipelined baseline; rounds_fp8: amax pass, then per round pack, quantise the bucket to FP8, "
+                         "dequantise, unpack; extract: source-map extraction kernel")
     ap.add_argument("--budget-mib", type=int, default=0, help="bucket budget per round (0: the 4 GiB default)")
     ap.add_argument("--budget-sweep", default="",
                     help="comma-separated bucket budgets in MiB: time the pipelined and the serial rounds "
@@ -305,10 +306,24 @@ def main():
         buckets = [torch.empty(max(plan.bucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
                    for _ in range(2)]
 
+    amax = qbucket = None
+    if args.path == "rounds_fp8":
+        amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
+        qbucket = torch.empty(max(plan.qbucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
+
     def step():
         if args.path == "remap":
             plan.remap(stream)
             return 1
+        if args.path == "rounds_fp8":
+            plan.absmax(amax.data_ptr(), stream)
+            for r in range(n_rounds):
+                b = buckets[r % 2].data_ptr()
+                plan.pack(r, b, stream)
+                plan.bucket_quantize(r, b, qbucket.data_ptr(), amax.data_ptr(), stream)
+                plan.bucket_dequantize(r, qbucket.data_ptr(), b, amax.data_ptr(), stream)
+                plan.unpack(r, b, stream)
+            return 1 + 4 * n_rounds
         if args.path in ("rounds", "rounds_serial"):
             plan.transfer_rounds(buckets[0].data_ptr(), buckets[1].data_ptr(),
                                  wb.WB_ROUNDS_SERIAL if args.path == "rounds_serial" else 0, stream)
@@ -360,6 +375,31 @@ def main():
                 "traffic_source": "ncu on the large scale of this layout, scaled by bytes moved",
                 "peak_source": peak_src, "kernel": "wb_exec_kernel", "best_ms": float(min(per_step)),
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # ---- FP8 path: each of the three extra kernels on its own, over all rounds ----------------------
+    fp8 = None
+    if args.path == "rounds_fp8" and rank == 0:
+        def timed(fn, reps=5):
+            fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+        es_, ed_ = (4 if wl.src_dtype == 0 else 2), (4 if wl.dst_dtype == 0 else 2)
+        elems = stats["dst_bytes_written"] // ed_          # one bucket element per rollout element written once
+        bucket_elems = sum(plan.qbucket_bytes(r) for r in range(n_rounds))
+        t_a = timed(lambda: plan.absmax(amax.data_ptr(), stream))
+        t_q = timed(lambda: [plan.bucket_quantize(r, buckets[0].data_ptr(), qbucket.data_ptr(), amax.data_ptr(), stream)
+                             for r in range(n_rounds)])
+        t_d = timed(lambda: [plan.bucket_dequantize(r, qbucket.data_ptr(), buckets[0].data_ptr(), amax.data_ptr(), stream)
+                             for r in range(n_rounds)])
+        fp8 = {"absmax_ms": t_a, "absmax_gbs": stats["src_bytes_read"] / t_a / 1e6,
+               "quantize_ms": t_q, "quantize_gbs": bucket_elems * (ed_ + 1) / t_q / 1e6,
+               "dequantize_ms": t_d, "dequantize_gbs": bucket_elems * (ed_ + 1) / t_d / 1e6,
+               "bucket_elements": bucket_elems, "wire_bytes_fp8": bucket_elems, "wire_bytes_unquantised": bucket_elems * ed_}
 
     # ---- bucket budget sweep (rounds path) ---------------------------------------------------------
     sweep = None
@@ -441,6 +481,8 @@ def main():
                "gpu_launches": launches, "pct_of_8TBs_nominal": 100.0 * value / world / 8000.0}
         if sweep is not None:
             out["budget_sweep"] = sweep
+        if fp8 is not None:
+            out["fp8"] = fp8
         print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()

@@ -266,6 +266,33 @@ wb_status wb_wait_probe(uint32_t limit_ms, void* cuda_stream);
 wb_status wb_transfer_rounds(const wb_plan* plan, void* bucket0, void* bucket1, uint32_t flags,
                              void* cuda_stream);
 
+/* ---- FP8 quantisation of a round's bucket (device; asynchronous on `cuda_stream`) -----------------
+ * Section 5 ("Parameter precision mismatch") sketches it: trainer tensors are quantised before the
+ * transfer, which needs the full tensor gathered first; "in each transfer round, the trainers would
+ * gather the sharded tensors to be quantized" before the write.  The paper fixes no rule.  The one
+ * built: FP8 E4M3 (largest finite value 448), one scale per checkpoint tensor, s = amax / 448 in
+ * fp32 (s = 1 if amax = 0), amax = the tensor's largest magnitude in the destination dtype;
+ * q = e4m3(x / s), fp32 division, round to nearest even, saturating, NaN -> 0x7F;
+ * x' = cast_dst(value(q) * s).  Checkpoint tensors are numbered 0 .. wb_plan_num_ckpts-1 in ascending
+ * order of their ids (wb_plan_ckpt_ids).
+ * wb_absmax: the gather, as a maximum: one pass over the de-duplicated trainer regions of the bound
+ *   tensors; amax (DEVICE, wb_plan_num_ckpts floats) is zeroed and then filled.  A tensor that holds a
+ *   NaN gets a NaN amax (magnitudes are compared as sign-cleared bit patterns).
+ * wb_bucket_quantize: `bucket` (DEVICE, as written by wb_pack for `round`) -> `qbucket` (DEVICE,
+ *   wb_plan_qbucket_bytes(round) bytes, one byte per element at the same element offset; padding is
+ *   never written).  wb_bucket_dequantize: the inverse, into a bucket wb_unpack can consume.
+ *   Both buffers 16-byte aligned, caller-owned.  Work lists are built and uploaded on first use
+ *   (one device allocation, released with the plan's device tables).
+ * Errors: INVALID_ARG, NOT_BOUND, OOM, CUDA. */
+size_t wb_plan_num_ckpts(const wb_plan* plan);
+wb_status wb_plan_ckpt_ids(const wb_plan* plan, uint64_t* out /* host */, size_t cap);
+size_t wb_plan_qbucket_bytes(const wb_plan* plan, size_t round);   /* 0 if round is invalid */
+wb_status wb_absmax(const wb_plan* plan, float* amax, void* cuda_stream);
+wb_status wb_bucket_quantize(const wb_plan* plan, size_t round, const void* bucket, void* qbucket,
+                             const float* amax, void* cuda_stream);
+wb_status wb_bucket_dequantize(const wb_plan* plan, size_t round, const void* qbucket, void* bucket,
+                               const float* amax, void* cuda_stream);
+
 /* wb_remap_host: the same transfer for callers whose weights are in HOST memory.  The remap
  * is cut into groups of consecutive tiles; for each group the trainer bytes it reads are copied
  * host -> bound device regions on an internal copy stream, its tiles run on `cuda_stream`, and the

@@ -79,6 +79,8 @@ EXPORTS = [
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
     "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_transfer_rounds",
+    "wb_plan_num_ckpts", "wb_plan_ckpt_ids", "wb_plan_qbucket_bytes", "wb_absmax", "wb_bucket_quantize",
+    "wb_bucket_dequantize",
     "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
@@ -118,6 +120,14 @@ def load() -> C.CDLL:
     lib.wb_unpack.argtypes = [vp, sz, vp, vp]
     lib.wb_remap_host.argtypes = [vp, vp, sz, vp, sz, vp]
     lib.wb_transfer_rounds.argtypes = [vp, vp, vp, C.c_uint32, vp]
+    lib.wb_plan_num_ckpts.argtypes = [vp]
+    lib.wb_plan_num_ckpts.restype = sz
+    lib.wb_plan_ckpt_ids.argtypes = [vp, vp, sz]
+    lib.wb_plan_qbucket_bytes.argtypes = [vp, sz]
+    lib.wb_plan_qbucket_bytes.restype = sz
+    lib.wb_absmax.argtypes = [vp, vp, vp]
+    lib.wb_bucket_quantize.argtypes = [vp, sz, vp, vp, vp, vp]
+    lib.wb_bucket_dequantize.argtypes = [vp, sz, vp, vp, vp, vp]
     lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
     lib.wb_wait_probe.argtypes = [C.c_uint32, vp]
@@ -251,6 +261,29 @@ class Plan:
 
     def transfer_rounds(self, bucket0_ptr: int, bucket1_ptr: int, flags: int = 0, stream: int = 0) -> None:
         _check(_lib.wb_transfer_rounds(self.handle, bucket0_ptr, bucket1_ptr, flags, stream), "wb_transfer_rounds")
+
+    # ---- FP8 quantisation of buckets ----------------------------------------------------------
+    def num_ckpts(self) -> int:
+        return int(_lib.wb_plan_num_ckpts(self.handle))
+
+    def ckpt_ids(self) -> np.ndarray:
+        out = np.zeros(self.num_ckpts(), np.uint64)
+        _check(_lib.wb_plan_ckpt_ids(self.handle, out.ctypes.data, out.size), "wb_plan_ckpt_ids")
+        return out
+
+    def qbucket_bytes(self, rnd: int) -> int:
+        return int(_lib.wb_plan_qbucket_bytes(self.handle, rnd))
+
+    def absmax(self, amax_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_absmax(self.handle, amax_ptr, stream), "wb_absmax")
+
+    def bucket_quantize(self, rnd: int, bucket_ptr: int, qbucket_ptr: int, amax_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_bucket_quantize(self.handle, rnd, bucket_ptr, qbucket_ptr, amax_ptr, stream),
+               "wb_bucket_quantize")
+
+    def bucket_dequantize(self, rnd: int, qbucket_ptr: int, bucket_ptr: int, amax_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_bucket_dequantize(self.handle, rnd, qbucket_ptr, bucket_ptr, amax_ptr, stream),
+               "wb_bucket_dequantize")
 
     def remap_host(self, host_src_ptrs: Sequence[int], host_dst_ptrs: Sequence[int], stream: int = 0) -> None:
         a, b = _ptr_array(host_src_ptrs), _ptr_array(host_dst_ptrs)

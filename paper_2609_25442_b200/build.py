@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwb.so")
-SOURCES = ["wb_layout.cpp", "wb_plan.cpp", "wb_exec.cu", "wb_extract.cu", "wb_scan.cpp"]
+SOURCES = ["wb_layout.cpp", "wb_plan.cpp", "wb_exec.cu", "wb_extract.cu", "wb_scan.cpp", "wb_quant.cu"]
 
 
 def _nvcc() -> str:

@@ -91,6 +91,7 @@ inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
 namespace wbi {
 void release_device_tables(wb_plan* plan) {
+  release_quant_tables(plan);
   if (plan->d_arena) {
     cudaFree(plan->d_arena);
     plan->d_arena = nullptr;
@@ -115,6 +116,7 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
     if (!src_base[i] || ((uintptr_t)src_base[i] % es)) return WB_ERR_INVALID_ARG;
   for (size_t i = 0; i < n_dst; ++i)
     if (!dst_base[i] || ((uintptr_t)dst_base[i] % ed)) return WB_ERR_INVALID_ARG;
+  wbi::release_quant_tables(plan);      // they hold addresses of the previous binding
   try {
     plan->src_base.assign(src_base, src_base + n_src);
     plan->dst_base.assign(dst_base, dst_base + n_dst);

@@ -187,9 +187,12 @@ struct wb_plan {
   void* d2h_stream = nullptr;
   std::vector<void*> host_events;
   size_t arena_bytes = 0;
+  void* quant_tables = nullptr;         // work lists of the FP8 bucket quantisation (wb_quant.cu), built on first use
 };
 
 namespace wbi {
 // implemented in wb_exec.cu
 void release_device_tables(wb_plan* plan);
+// implemented in wb_quant.cu
+void release_quant_tables(wb_plan* plan);
 }

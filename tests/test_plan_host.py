@@ -280,6 +280,14 @@ def test_error_bucket_too_small_and_unbound_execution():
     _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds(258, 512))       # not 16-byte aligned
     _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds(256, 512, flags=8))
     _expect("WB_ERR_NOT_BOUND", lambda: plan.transfer_rounds(256, 0, flags=wb.WB_ROUNDS_SERIAL))
+    # FP8 bucket quantisation: host-side queries work on any plan, device calls need a binding
+    assert plan.num_ckpts() == len(wl.ckpt) and plan.ckpt_ids().tolist() == list(range(len(wl.ckpt)))
+    assert plan.qbucket_bytes(0) * 2 == plan.bucket_bytes(0) and plan.qbucket_bytes(99) == 0
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.absmax(256))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.absmax(0))
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.bucket_quantize(0, 256, 512, 1024))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.bucket_quantize(0, 258, 512, 1024))     # not 16-byte aligned
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.bucket_dequantize(99, 256, 512, 1024))  # no such round
     _expect("WB_ERR_INVALID_ARG", lambda: plan.bind([0] * plan.n_src, [0] * plan.n_dst))
     lib = wb.load()
     assert lib.wb_remap(None, None) == 1
