@@ -270,10 +270,10 @@ wb_status wb_transfer_rounds(const wb_plan* plan, void* bucket0, void* bucket1, 
  * Section 5 ("Parameter precision mismatch") sketches it: trainer tensors are quantised before the
  * transfer, which needs the full tensor gathered first; "in each transfer round, the trainers would
  * gather the sharded tensors to be quantized" before the write.  The paper fixes no rule.  The one
- * built: FP8 E4M3 (largest finite value 448), one scale per checkpoint tensor, s = amax / 448 in
- * fp32 (s = 1 if amax = 0), amax = the tensor's largest magnitude in the destination dtype;
- * q = e4m3(x / s), fp32 division, round to nearest even, saturating, NaN -> 0x7F;
- * x' = cast_dst(value(q) * s).  Checkpoint tensors are numbered 0 .. wb_plan_num_ckpts-1 in ascending
+ * built: FP8 E4M3 (largest finite value 448), one scale per checkpoint tensor, s = amax / 448 and
+ * r = 448 / amax in fp32 (s = r = 1 if amax = 0), amax = the tensor's largest magnitude in the
+ * destination dtype; q = e4m3(x * r), fp32 multiplication, round to nearest even, saturating,
+ * NaN -> 0x7F; x' = cast_dst(value(q) * s).  Checkpoint tensors are numbered 0 .. wb_plan_num_ckpts-1 in ascending
  * order of their ids (wb_plan_ckpt_ids).
  * wb_absmax: the gather, as a maximum: one pass over the de-duplicated trainer regions of the bound
  *   tensors; amax (DEVICE, wb_plan_num_ckpts floats) is zeroed and then filled.  A tensor that holds a

@@ -8,10 +8,12 @@ the arithmetic below):
 
   format   FP8 E4M3 (4 exponent bits, bias 7, 3 mantissa bits, no infinities, largest finite
            value 448, NaN = S.1111.111).
-  scale    one per checkpoint tensor: s = amax / 448 in fp32, amax the largest magnitude of the
-           tensor's elements in the destination dtype (the "gather"); s = 1 if amax = 0.
-  encode   q = e4m3(x / s): fp32 division, round to nearest with ties to even, magnitudes beyond
-           the largest finite value saturate to it, NaN -> 0x7F.
+  scale    one per checkpoint tensor: s = amax / 448 and its counterpart r = 448 / amax, both one
+           fp32 division, amax the largest magnitude of the tensor's elements in the destination
+           dtype (the "gather"); s = r = 1 if amax = 0.
+  encode   q = e4m3(x * r): fp32 multiplication with the reciprocal scale (the convention of FP8
+           training libraries: one division per tensor, none per element), round to nearest with
+           ties to even, magnitudes beyond the largest finite value saturate to it, NaN -> 0x7F.
   decode   x' = cast_dst(value(q) * s): fp32 multiplication, then the destination dtype's rounding.
 
 The quantised object is the bucket payload (checkpoint format, destination dtype), so for an
@@ -94,9 +96,18 @@ def scale_of(amax: np.uint32) -> np.float32:
         return np.float32(a / np.float32(E4M3_MAX))
 
 
-def quantize(bits: np.ndarray, dtype: int, scale: np.float32) -> np.ndarray:
+def rscale_of(amax: np.uint32) -> np.float32:
+    """The reciprocal scale 448 / amax (fp32 division; 1 for an all-zero tensor)."""
+    a = np.array([amax], np.uint32).view(np.float32)[0]
+    if a == 0:
+        return np.float32(1.0)
     with np.errstate(invalid="ignore", divide="ignore", over="ignore"):
-        y = to_f32(bits, dtype) / np.float32(scale)
+        return np.float32(np.float32(E4M3_MAX) / a)
+
+
+def quantize(bits: np.ndarray, dtype: int, rscale: np.float32) -> np.ndarray:
+    with np.errstate(invalid="ignore", over="ignore"):
+        y = to_f32(bits, dtype) * np.float32(rscale)
     return e4m3_encode(y)
 
 

@@ -1,9 +1,9 @@
 // FP8 quantisation of transfer buckets (Section 5 of the paper, "Parameter precision mismatch":
 // trainer tensors are quantised before the transfer, which needs the full tensor gathered first).
 // The paper fixes no rule; the one built here: FP8 E4M3, one scale per checkpoint tensor,
-// s = amax / 448 with amax the tensor's largest magnitude in the destination dtype (the gather
-// becomes a maximum over every trainer shard of the tensor), q = e4m3(x / s) with round to nearest
-// even and saturation, x' = cast(value(q) * s).
+// s = amax / 448 and r = 448 / amax with amax the tensor's largest magnitude in the destination dtype
+// (the gather becomes a maximum over every trainer shard of the tensor), q = e4m3(x * r) with round
+// to nearest even and saturation, x' = cast(value(q) * s).
 //
 //   wb_absmax            one pass over the de-duplicated trainer regions -> amax per checkpoint tensor
 //   wb_bucket_quantize   a packed round's bucket (destination dtype) -> FP8 bucket, same element offsets
@@ -66,6 +66,10 @@ __device__ __forceinline__ uint32_t f32x2_to_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float scale_of(const float* __restrict__ amax, uint32_t ckpt) {
   const float a = __ldg(amax + ckpt);
   return a == 0.f ? 1.f : __fdiv_rn(a, 448.f);
+}
+__device__ __forceinline__ float rscale_of(const float* __restrict__ amax, uint32_t ckpt) {
+  const float a = __ldg(amax + ckpt);
+  return a == 0.f ? 1.f : __fdiv_rn(448.f, a);
 }
 
 // Sign-cleared fp32 pattern of one source element / of the elements packed in a 32-bit word.
@@ -135,7 +139,7 @@ wb_quantize_kernel(const QuantItem* __restrict__ items, uint32_t n_items, const 
                    uint8_t* __restrict__ q, const float* __restrict__ amax) {
   for (uint32_t k = blockIdx.x; k < n_items; k += gridDim.x) {
     const QuantItem it = items[k];
-    const float s = scale_of(amax, it.ckpt);
+    const float r = rscale_of(amax, it.ckpt);
     const char* x = bucket + it.off * ED;
     uint8_t* out = q + it.off;
     const uint32_t body = it.n & ~7u;
@@ -157,7 +161,7 @@ wb_quantize_kernel(const QuantItem* __restrict__ items, uint32_t n_items, const 
       }
       uint32_t c[4];
 #pragma unroll
-      for (int p = 0; p < 4; ++p) c[p] = f32x2_to_e4m3x2(__fdiv_rn(f[2 * p], s), __fdiv_rn(f[2 * p + 1], s));
+      for (int p = 0; p < 4; ++p) c[p] = f32x2_to_e4m3x2(__fmul_rn(f[2 * p], r), __fmul_rn(f[2 * p + 1], r));
       // two-byte buckets start payloads on multiples of 8 elements, four-byte buckets on multiples of 4
       if (ED == 2) {
         __stcs(reinterpret_cast<uint2*>(out + e), make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16)));
@@ -170,7 +174,7 @@ wb_quantize_kernel(const QuantItem* __restrict__ items, uint32_t n_items, const 
       float f;
       if (ED == 2) f = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(x)[e] << 16);
       else f = reinterpret_cast<const float*>(x)[e];
-      out[e] = (uint8_t)(f32x2_to_e4m3x2(__fdiv_rn(f, s), 0.f) & 0xFFu);
+      out[e] = (uint8_t)(f32x2_to_e4m3x2(__fmul_rn(f, r), 0.f) & 0xFFu);
     }
   }
 }

@@ -42,6 +42,7 @@ def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id)
     want_amax = np.array([quant.amax_bits(views[int(t)].reshape(-1), wl_dst_dtype) for t in ids], np.uint32)
     assert np.array_equal(got_amax, want_amax)
     scales = {int(t): quant.scale_of(want_amax[k]) for k, t in enumerate(ids)}
+    rscales = {int(t): quant.rscale_of(want_amax[k]) for k, t in enumerate(ids)}
     ed = 2 if wl_dst_dtype == WB_BF16 else 4
     for r in range(plan.num_rounds()):
         nb = plan.bucket_bytes(r)
@@ -61,7 +62,7 @@ def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id)
             r0, c0, nr, nc = (int(e[k]) for k in ("r0", "c0", "nr", "nc"))
             rect = views[t][r0:r0 + nr, c0:c0 + nc].reshape(-1)
             off = int(e["bucket_off"]) // ed
-            codes = quant.quantize(rect, wl_dst_dtype, scales[t])
+            codes = quant.quantize(rect, wl_dst_dtype, rscales[t])
             assert np.array_equal(q[off:off + nr * nc], codes), (r, t)
             back = quant.dequantize(codes, wl_dst_dtype, scales[t])
             assert same_bits(b2[off:off + nr * nc], back, wl_dst_dtype), (r, t)
@@ -72,7 +73,7 @@ def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id)
         plan.unpack(r, bucket2.data_ptr())
     torch.cuda.synchronize()
     plan.check()
-    return {t: quant.dequantize(quant.quantize(v.reshape(-1), wl_dst_dtype, scales[t]), wl_dst_dtype,
+    return {t: quant.dequantize(quant.quantize(v.reshape(-1), wl_dst_dtype, rscales[t]), wl_dst_dtype,
                                 scales[t]).reshape(v.shape) for t, v in views.items()}
 
 

@@ -81,8 +81,10 @@ def test_scale_and_round_trip(dtype):
     assert np.array([amax], np.uint32).view(np.float32)[0] == np.abs(vals).max()
     s = quant.scale_of(amax)
     assert s == np.float32(np.abs(vals).max() / np.float32(448))
-    q = quant.quantize(bits, dtype, s)
-    assert q.max() & 0x7F <= 0x7E                            # nothing overflows: |x / s| <= 448 (1 + 2^-23)
+    r = quant.rscale_of(amax)
+    assert r == np.float32(np.float32(448) / np.abs(vals).max())
+    q = quant.quantize(bits, dtype, r)
+    assert (q & 0x7F).max() <= 0x7E                          # nothing overflows: |x * r| <= 448 (1 + 2^-23)
     assert (q[np.argmax(np.abs(vals))] & 0x7F) == 0x7E       # the largest element lands on the largest code
     back = quant.to_f32(quant.dequantize(q, dtype, s), dtype)
     # E4M3 keeps 4 significant bits: relative error <= 2^-4 for normal codes, absolute <= s * 2^-10 below
@@ -94,10 +96,11 @@ def test_scale_and_round_trip(dtype):
 def test_degenerate_scales():
     assert quant.scale_of(np.uint32(0)) == np.float32(1.0)                       # all-zero tensor
     zeros = np.zeros(8, np.uint16)
-    assert quant.quantize(zeros, BF16, quant.scale_of(quant.amax_bits(zeros, BF16))).tolist() == [0] * 8
+    assert quant.rscale_of(np.uint32(0)) == np.float32(1.0)
+    assert quant.quantize(zeros, BF16, quant.rscale_of(quant.amax_bits(zeros, BF16))).tolist() == [0] * 8
     nan_bits = np.array([0x3F80, 0x7FC0, 0xBF80], np.uint16)                      # 1, NaN, -1 in bf16
     amax = quant.amax_bits(nan_bits, BF16)
     assert amax > 0x7F800000                                                      # the NaN wins the maximum
-    q = quant.quantize(nan_bits, BF16, quant.scale_of(amax))
+    q = quant.quantize(nan_bits, BF16, quant.rscale_of(amax))
     assert q.tolist() == [0x7F, 0x7F, 0x7F]                                       # no scale: everything is NaN
     assert quant.amax_bits(np.zeros(0, np.uint16), BF16) == 0
