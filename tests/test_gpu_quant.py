@@ -133,3 +133,28 @@ def test_special_tensors(dts):
     for k in range(len(vals)):
         got = to_bits(dst.tensors[k])
         assert same_bits(got, want[k].reshape(-1), ddt), k
+
+
+def test_rebinding_rebuilds_the_work_lists():
+    """The amax work list holds device addresses: binding the plan to other tensors must rebuild it."""
+    wl = make_workload("cfg1b")
+    dev = torch.device(DEV)
+    case = DeviceCase(wl, dev)
+    plan = case.plan
+    amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
+    plan.absmax(amax.data_ptr())
+    torch.cuda.synchronize()
+    first = amax.clone()
+    # a second set of trainer tensors with every value doubled (exact in fp32)
+    src2 = RankArenas(wl.trainer.tensors, dev, fill_byte=0)
+    for a, b in zip(src2.tensors, case.src.tensors):
+        a.copy_(b * 2)
+    bind(plan, src2, case.dst)
+    plan.absmax(amax.data_ptr())
+    torch.cuda.synchronize()
+    assert torch.equal(amax, first * 2) and bool((first > 0).all())
+    # and the old tensors may be gone by now
+    case.src = None
+    plan.absmax(amax.data_ptr())
+    torch.cuda.synchronize()
+    assert torch.equal(amax, first * 2)
