@@ -212,7 +212,12 @@ struct TileBuilder {
     // transposed: one staged transposition chunk of the executor wide (496 source bytes) and as tall
     // as the tile size allows, so that a tile writes long pieces of few destination runs and the
     // element stores at the two ends of a run piece are rare
-    uint64_t tc = std::min<uint64_t>(nc, trans ? 496 / es : 512);
+#ifndef WB_TRANS_NARROW_MIN_BYTES
+#define WB_TRANS_NARROW_MIN_BYTES (1u << 20)
+#endif
+    // (small slabs keep four chunks per tile: there the number of tiles matters more)
+    const bool narrow = nr * nc * (uint64_t)(es + ed) >= WB_TRANS_NARROW_MIN_BYTES;
+    uint64_t tc = std::min<uint64_t>(nc, trans ? (narrow ? 496 / es : 496) : 512);
     uint64_t tr = std::min<uint64_t>(nr, std::max<uint64_t>(64, roundup(T / tc, 64)));
     if (trans) {
       // rows fastest: consecutive tiles continue the same destination runs
