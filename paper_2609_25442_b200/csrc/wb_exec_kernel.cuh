@@ -58,9 +58,7 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
       if (d.mode == MODE_ROWS) {
         staged_rows<ES, ED>(d, stage, tr);
       } else if (d.mode == MODE_TRANS) {
-#ifndef WB_TRANS_SKIP_WORK
         staged_trans<ES, ED>(d, stage, tr);
-#endif
       } else {
         // queued tiles: one big tile shared by all worker warps, or a run of small tiles with one
         // warp per tile

@@ -396,19 +396,17 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
 
   // The rows of a block are short pieces (128 bytes) a row pitch apart, and a lane holds only two
   // batches of loads, which is not enough memory parallelism to cover DRAM latency.  So the warp asks
-  // for the block after next to be brought into L2 ahead of time (lane = row; every sector of the
-  // piece): that costs no registers, and the loads then hit L2.
+  // for the block after next to be brought into L2 ahead of time (lane = row; the first and the last
+  // byte of the piece - a request per sector was measured to cost more than it brings): that costs
+  // no registers, and the loads then hit L2.
   auto prefetch = [&](uint32_t pb) {
-#ifndef WB_NO_TRANS_PREFETCH
     if (pb >= nb) return;
     const Block k = block_of(pb);
     for (uint32_t r = lane; r < k.nl; r += 32) {
       const char* row = f.s + ((size_t)(k.i0 + r) * f.ssr + k.j0) * ES;
-      const uint32_t bytes = k.nj * ES;                             // one request per 32-byte sector
-      for (uint32_t o = 0; o < bytes; o += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + o));
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(row + bytes - 1));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(row + (size_t)(k.nj - 1) * ES));
     }
-#endif
   };
   // The warp's batches in order; the loads of batch q+1 are issued before batch q is consumed, so
   // they are in flight during the shared-memory writes and during phase B.

@@ -504,7 +504,6 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
       }
       if (!ranges.empty()) ranges.back().second = P->remap.tiles.size();
       if (!tb.ok) return fail(WB_ERR_INVALID_ARG);
-#ifndef WB_NO_TILE_ORDER
       for (auto& rg : ranges) {
         auto key = [](const HTile& t) {
           // 0: source rows strided, by source address; 1: destination strided, by destination address; 2: as emitted
@@ -515,7 +514,6 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
         std::stable_sort(P->remap.tiles.begin() + rg.first, P->remap.tiles.begin() + rg.second,
                          [&](const HTile& a, const HTile& b) { return key(a) < key(b); });
       }
-#endif
       assign_ctas(&P->remap, P->grid);
     }
 
