@@ -219,6 +219,8 @@ wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, size_t n_src,
                        void* const* dst_base, size_t n_dst);
 
 /* ---- execution (device; asynchronous on `cuda_stream`, a cudaStream_t or NULL) -----------
+ * Each of wb_remap / wb_pack / wb_unpack is a single kernel launch on `cuda_stream` and can be captured
+ * into a CUDA graph once it has been called outside capture (the first call sets a kernel attribute).
  * wb_remap: the fused path, trainer tensors -> rollout tensors in one persistent launch:
  * dst[x] = cast(src[y]) for every corresponding pair (Section 3.1), fp32 -> bf16 by
  * round-to-nearest-even, same dtype = bit copy.

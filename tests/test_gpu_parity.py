@@ -422,3 +422,24 @@ def test_replica_consistency_check(device):
     assert case.plan.check_replicas() == 2
     wl4 = make_workload("cfg4", "small")           # no replicas at all
     assert DeviceCase(wl4, device).plan.check_replicas() == 0
+
+
+def test_remap_in_a_cuda_graph(device):
+    """wb_remap is one kernel launch on the caller's stream, so it can be captured into a CUDA graph and
+    replayed (after one ordinary call, which sets the kernel's shared-memory attribute)."""
+    case = DeviceCase(make_workload("cfg1b"), device)
+    want = oracle_for(case)
+    case.plan.remap()                                   # outside capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream(device=device)
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            case.plan.remap(torch.cuda.current_stream().cuda_stream)
+    for _ in range(3):
+        case.reset_dst()
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        assert_dst_equals(case, want)
+    case.plan.check()
