@@ -54,6 +54,8 @@ def parse_args():
                          "rounds: wb_transfer_rounds (depth-2 buckets, two streams); rounds_serial: its "
                          "unpipelined baseline; rounds_fp8: amax pass, then per round pack, quantise the bucket to FP8, "
                          "dequantise, unpack; extract: source-map extraction kernel")
+    ap.add_argument("--cuda-graph", action="store_true",
+                    help="remap path: replay the launch from a captured CUDA graph (for the launch-bound tiny model)")
     ap.add_argument("--budget-mib", type=int, default=0, help="bucket budget per round (0: the 4 GiB default)")
     ap.add_argument("--budget-sweep", default="",
                     help="comma-separated bucket budgets in MiB: time the pipelined and the serial rounds "
@@ -311,9 +313,23 @@ def main():
         amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
         qbucket = torch.empty(max(plan.qbucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
 
+    graph = None
+    if args.cuda_graph and args.path == "remap":
+        plan.remap(stream)                               # the first call sets the kernel attribute
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        cap = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(cap):
+            with torch.cuda.graph(graph, stream=cap):
+                plan.remap(torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+
     def step():
         if args.path == "remap":
-            plan.remap(stream)
+            if graph is not None:
+                graph.replay()
+            else:
+                plan.remap(stream)
             return 1
         if args.path == "rounds_fp8":
             plan.absmax(amax.data_ptr(), stream)
@@ -476,6 +492,7 @@ def main():
                           "grid_ctas": stats["grid_ctas"], "tile_bytes": stats["tile_bytes"],
                           "plan_build_s": plan_s, "replicas_per_gpu": 1,
                           "schedule": "static" if args.static_schedule else "dynamic",
+                          "cuda_graph": bool(graph is not None),
                           "multi_gpu": "independent replicas, no collective"},
                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                "gpu_launches": launches, "pct_of_8TBs_nominal": 100.0 * value / world / 8000.0}
