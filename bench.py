@@ -154,7 +154,25 @@ def oracle_sample(wl, fetch_src, budget_elems=60_000_000):
 
     t_t, t_s, t_used = restrict(wl.trainer)
     r_t, r_s, _ = restrict(wl.rollout)
-    src = [fetch_src(k) for k in t_used]
+    if fetch_src is not None:
+        src = [fetch_src(k) for k in t_used]
+    else:
+        # seeded checkpoint values for the sampled tensors, put into the trainer buffers through the
+        # trainer's own slice list (so replicas agree, as after a real load_weights)
+        bits_dt = np.uint32 if wl.src_dtype == 0 else np.uint16
+        src = [np.zeros(int(t["numel"]), bits_dt) for t in t_t]
+        vals = {}
+        for sl in t_s:
+            c = int(sl["ckpt"])
+            if c not in vals:
+                rng = np.random.default_rng(wl.seed * 1000003 + c)
+                v = rng.standard_normal(wl.ckpt[c].numel, dtype=np.float32) * np.float32(0.02)
+                vals[c] = v.view(np.uint32) if wl.src_dtype == 0 else to_bits_np(torch.from_numpy(v).to(torch.bfloat16))
+            i = np.arange(int(sl["nr"]), dtype=np.int64)[:, None]
+            j = np.arange(int(sl["nc"]), dtype=np.int64)[None, :]
+            g = (int(sl["r0"]) + i) * int(sl["ckpt_cols"]) + int(sl["c0"]) + j
+            x = int(sl["local_off"]) + i * int(sl["stride_r"]) + j * int(sl["stride_c"])
+            src[int(sl["tensor"])][x] = vals[c][g]
     shapes = [(c.rows, c.cols) for c in wl.ckpt]
     t0 = time.perf_counter()
     res = remap_oracle(shapes, t_t, t_s, r_t, r_s, src)
@@ -179,23 +197,12 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     wl = make_workload(args.workload, args.scale)
-    rng = np.random.default_rng(wl.seed)
-    cache = {}
-
-    def fetch(k):   # seeded synthetic source bits, generated on the host for the sampled tensors only
-        if k not in cache:
-            n = int(wl.trainer.tensors[k]["numel"])
-            v = (rng.standard_normal(n, dtype=np.float32) * 0.02)
-            cache[k] = v.view(np.uint32) if wl.src_dtype == 0 else \
-                to_bits_np(torch.from_numpy(v).to(torch.bfloat16))
-        return cache[k]
-
     budget = 20_000_000
     times, moved, desc = [], 0, ""
     for _ in range(args.warmup):
-        oracle_sample(wl, fetch, budget)
+        oracle_sample(wl, None, budget)
     for _ in range(args.steps):
-        dt, moved, desc = oracle_sample(wl, fetch, budget)
+        dt, moved, desc = oracle_sample(wl, None, budget)
         times.append(dt)
     ms = 1e3 * sum(times) / max(len(times), 1)
     value = moved / (ms * 1e-3) / 1e9 if times else 0.0
