@@ -398,6 +398,28 @@ enum { WB_ID_I64 = 0,   /* field of int64                                       
  * 2^48; a field of several rows has rows, cols < 2^31.  Errors: INVALID_ARG, CUDA. */
 wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols,
                             wb_diff2_entry* out, uint64_t cap, uint64_t* count, void* cuda_stream);
+/* wb_diff2_nonzeros_batch: the same for many fields in ONE launch (a model has thousands of local
+ * tensors, most of them small; a launch per tensor is bound by launch latency - the per-tensor
+ * overhead Section 3.2 warns about).  `fields`: HOST array of n_fields descriptors (`field` DEVICE);
+ * every entry found in field k carries fields[k].tag.  `scratch`: DEVICE, 16-byte aligned, at least
+ * wb_diff2_batch_scratch_bytes(n_fields) bytes, must stay valid until the kernel has run.  `out`
+ * (DEVICE, `cap` entries, one list for all fields, no particular order) and *count (DEVICE uint64,
+ * zeroed by the caller) as above.  Fields with rows or cols = 0 are skipped.  Errors: INVALID_ARG,
+ * OOM, CUDA. */
+typedef struct wb_diff2_field {
+  const void* field;
+  uint64_t rows, cols;
+  uint32_t id_kind;
+  uint32_t tag;
+} wb_diff2_field;
+typedef struct wb_diff2_tagged_entry {
+  uint64_t row, col;
+  int64_t value;
+  uint32_t tag, reserved;
+} wb_diff2_tagged_entry;
+size_t wb_diff2_batch_scratch_bytes(size_t n_fields);
+wb_status wb_diff2_nonzeros_batch(const wb_diff2_field* fields, size_t n_fields, void* scratch, size_t scratch_bytes,
+                                  wb_diff2_tagged_entry* out, uint64_t cap, uint64_t* count, void* cuda_stream);
 /* wb_diff2_recombine (host): Algorithm 1, Recombine.  sum_k 2^(chunk_bits*k) * passes[k], merged
  * by position, zeros dropped, sorted by (row, col).  Writes up to cap entries, *n_out = total. */
 wb_status wb_diff2_recombine(const wb_diff2_entry* const* passes, const size_t* counts, size_t n_passes,

@@ -81,7 +81,7 @@ EXPORTS = [
     "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_transfer_rounds",
     "wb_plan_num_ckpts", "wb_plan_ckpt_ids", "wb_plan_qbucket_bytes", "wb_absmax", "wb_bucket_quantize",
     "wb_bucket_dequantize",
-    "wb_diff2_nonzeros", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_diff2_nonzeros", "wb_diff2_nonzeros_batch", "wb_diff2_batch_scratch_bytes", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -336,6 +336,29 @@ def wb_diff2_nonzeros(field_ptr: int, id_kind: int, rows: int, cols: int, out_pt
     load()
     _check(_lib.wb_diff2_nonzeros(field_ptr, id_kind, rows, cols, out_ptr, cap, count_ptr, stream),
            "wb_diff2_nonzeros")
+
+
+DIFF2_FIELD_DTYPE = np.dtype([("field", "<u8"), ("rows", "<u8"), ("cols", "<u8"), ("id_kind", "<u4"), ("tag", "<u4")])
+DIFF2_TAGGED_ENTRY_DTYPE = np.dtype([("row", "<u8"), ("col", "<u8"), ("value", "<i8"), ("tag", "<u4"), ("reserved", "<u4")])
+assert DIFF2_FIELD_DTYPE.itemsize == 32 and DIFF2_TAGGED_ENTRY_DTYPE.itemsize == 32
+
+
+def wb_diff2_batch_scratch_bytes(n_fields: int) -> int:
+    load()
+    _lib.wb_diff2_batch_scratch_bytes.restype = C.c_size_t
+    _lib.wb_diff2_batch_scratch_bytes.argtypes = [C.c_size_t]
+    return int(_lib.wb_diff2_batch_scratch_bytes(n_fields))
+
+
+def wb_diff2_nonzeros_batch(fields: np.ndarray, scratch_ptr: int, scratch_bytes: int, out_ptr: int, cap: int,
+                            count_ptr: int, stream: int = 0) -> None:
+    """diff2 of many device id fields in one launch; `fields` is a host array of DIFF2_FIELD_DTYPE."""
+    load()
+    fields = np.ascontiguousarray(fields, dtype=DIFF2_FIELD_DTYPE)
+    _lib.wb_diff2_nonzeros_batch.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint64,
+                                             C.c_void_p, C.c_void_p]
+    _check(_lib.wb_diff2_nonzeros_batch(fields.ctypes.data, len(fields), scratch_ptr, scratch_bytes, out_ptr, cap,
+                                        count_ptr, stream), "wb_diff2_nonzeros_batch")
 
 
 def wb_diff2_recombine(passes: Sequence[np.ndarray], chunk_bits: int) -> np.ndarray:

@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <new>
+#include <vector>
 
 #include "wb.h"
 
@@ -113,10 +115,20 @@ __device__ __forceinline__ void row_load(const void* field, unsigned long long r
 
 // Horizontal second difference of one row of values v (with halo ve1 = v[c0-1], ve2 = v[c0-2] in
 // lane 0), and compaction of its non-zero entries.
+__device__ __forceinline__ void put_entry(wb_diff2_entry* out, unsigned long long slot, unsigned long long row,
+                                          unsigned long long col, long long value, unsigned) {
+  out[slot] = wb_diff2_entry{row, col, value};
+}
+__device__ __forceinline__ void put_entry(wb_diff2_tagged_entry* out, unsigned long long slot, unsigned long long row,
+                                          unsigned long long col, long long value, unsigned tag) {
+  out[slot] = wb_diff2_tagged_entry{row, col, value, tag, 0u};
+}
+
+template <typename Entry>
 __device__ __forceinline__ void emit_row(const long long v[kV], long long ve1, long long ve2, unsigned long long row,
                                          unsigned long long c0, unsigned long long cols, unsigned lane,
-                                         wb_diff2_entry* __restrict__ out, unsigned long long cap,
-                                         unsigned long long* __restrict__ count) {
+                                         Entry* __restrict__ out, unsigned long long cap,
+                                         unsigned long long* __restrict__ count, unsigned tag = 0) {
   const unsigned from = (lane + 31u) & 31u;
   long long carry1 = ve1, carry2 = ve2;                        // lane 0: the two values left of the group
 #pragma unroll
@@ -156,7 +168,7 @@ __device__ __forceinline__ void emit_row(const long long v[kV], long long ve1, l
 #pragma unroll
     for (int q = 0; q < kQ; ++q)
       if (d[q] != 0) {
-        if (slot < cap) out[slot] = wb_diff2_entry{row, c + q, d[q]};
+        if (slot < cap) put_entry(out, slot, row, c + q, d[q], tag);
         ++slot;
       }
   }
@@ -194,11 +206,11 @@ __device__ __forceinline__ void visit_load(const void* field, const Visit& v, un
 
 // The rows a warp holds live in a ring of register sets addressed by the position in an unrolled
 // loop (current row, the row being fetched and the two rows above), so advancing a row moves no registers.
-template <int KIND>
+template <int KIND, typename Entry>
 __global__ void __launch_bounds__(256, 2)
 wb_diff2_kernel(const void* __restrict__ field, unsigned long long rows, unsigned long long cols,
-                unsigned long long rows_per_task, wb_diff2_entry* __restrict__ out, unsigned long long cap,
-                unsigned long long* __restrict__ count) {
+                unsigned long long rows_per_task, Entry* __restrict__ out, unsigned long long cap,
+                unsigned long long* __restrict__ count, unsigned tag) {
   constexpr int kRing = 4;
   const unsigned lane = threadIdx.x & 31;
   const unsigned strips = (unsigned)((cols + kStrip - 1) / kStrip);
@@ -234,7 +246,7 @@ wb_diff2_kernel(const void* __restrict__ field, unsigned long long rows, unsigne
         const long long ve1 = cur.e1 - 2 * p1.e1 + p2.e1, ve2 = cur.e2 - 2 * p1.e2 + p2.e2;
         nz |= (ve1 | ve2) != 0;
         if (__any_sync(0xFFFFFFFFu, nz))
-          emit_row(vv, ve1, ve2, (unsigned long long)v.row, v.c0, cols, lane, out, cap, count);
+          emit_row(vv, ve1, ve2, (unsigned long long)v.row, v.c0, cols, lane, out, cap, count, tag);
       }
       if (!more) return;
       v = w;
@@ -245,10 +257,10 @@ wb_diff2_kernel(const void* __restrict__ field, unsigned long long rows, unsigne
 // A field with one row (a flat shard): diff2 is the second difference along the row, every task is
 // one strip, and a warp alternates between two register sets so that the next strip is in flight
 // while the current one is consumed.
-template <int KIND>
+template <int KIND, typename Entry>
 __global__ void __launch_bounds__(256, 3)
-wb_diff2_row_kernel(const void* __restrict__ field, unsigned long long cols, wb_diff2_entry* __restrict__ out,
-                    unsigned long long cap, unsigned long long* __restrict__ count) {
+wb_diff2_row_kernel(const void* __restrict__ field, unsigned long long cols, Entry* __restrict__ out,
+                    unsigned long long cap, unsigned long long* __restrict__ count, unsigned tag) {
   const unsigned lane = threadIdx.x & 31;
   const unsigned long long stride = (((unsigned long long)gridDim.x * blockDim.x) >> 5) * kStrip;
   unsigned long long c0 = ((((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5)) * kStrip;
@@ -258,24 +270,92 @@ wb_diff2_row_kernel(const void* __restrict__ field, unsigned long long cols, wb_
   for (;;) {
     const unsigned long long c1 = c0 + stride;
     if (c1 < cols) row_load<KIND>(field, 0, cols, c1, lane, r1);
-    emit_row(r0.a, r0.e1, r0.e2, 0, c0, cols, lane, out, cap, count);
+    emit_row(r0.a, r0.e1, r0.e2, 0, c0, cols, lane, out, cap, count, tag);
     if (c1 >= cols) return;
     c0 = c1 + stride;
     if (c0 < cols) row_load<KIND>(field, 0, cols, c0, lane, r0);
-    emit_row(r1.a, r1.e1, r1.e2, 0, c1, cols, lane, out, cap, count);
+    emit_row(r1.a, r1.e1, r1.e2, 0, c1, cols, lane, out, cap, count, tag);
     if (c0 >= cols) return;
+  }
+}
+
+// ---- many fields in one launch ---------------------------------------------------------------------
+// A model has thousands of local tensors, most of them small: one launch per tensor is bound by launch
+// latency.  Here the tasks (strip x block of kRowsPerTask rows) of all fields form one list; a warp
+// finds the field of a task by bisection over the fields' first task numbers and walks the task with
+// the two rows above it primed, the next row's loads in flight.
+// fields of at least this many elements are launched on their own by the batched entry point
+constexpr unsigned long long kBatchLargeField = 1ull << 24;
+
+struct BatchField {
+  const void* field;
+  unsigned long long rows, cols, task_begin;
+  unsigned id_kind, tag;
+};
+
+template <int KIND>
+__device__ __forceinline__ void batch_task(const BatchField& f, unsigned long long local, unsigned lane,
+                                           wb_diff2_tagged_entry* __restrict__ out, unsigned long long cap,
+                                           unsigned long long* __restrict__ count) {
+  const unsigned long long strips = (f.cols + kStrip - 1) / kStrip;
+  const unsigned long long rb = local / strips, c0 = (local - rb * strips) * kStrip;
+  const unsigned long long i0 = rb * kRowsPerTask, i1 = i0 + kRowsPerTask < f.rows ? i0 + kRowsPerTask : f.rows;
+  RowRegs p2, p1, cur, nxt;
+#pragma unroll
+  for (int k = 0; k < kV; ++k) p1.a[k] = p2.a[k] = 0;
+  p1.e1 = p1.e2 = p2.e1 = p2.e2 = 0;
+  if (i0 >= 2) row_load<KIND>(f.field, (i0 - 2) * f.cols, f.cols, c0, lane, p2);
+  if (i0 >= 1) row_load<KIND>(f.field, (i0 - 1) * f.cols, f.cols, c0, lane, p1);
+  row_load<KIND>(f.field, i0 * f.cols, f.cols, c0, lane, cur);
+  for (unsigned long long i = i0; i < i1; ++i) {
+    if (i + 1 < i1) row_load<KIND>(f.field, (i + 1) * f.cols, f.cols, c0, lane, nxt);
+    long long vv[kV];
+    bool nz = false;
+#pragma unroll
+    for (int k = 0; k < kV; ++k) {
+      vv[k] = cur.a[k] - 2 * p1.a[k] + p2.a[k];
+      nz |= vv[k] != 0;
+    }
+    const long long ve1 = cur.e1 - 2 * p1.e1 + p2.e1, ve2 = cur.e2 - 2 * p1.e2 + p2.e2;
+    nz |= (ve1 | ve2) != 0;
+    if (__any_sync(0xFFFFFFFFu, nz)) emit_row(vv, ve1, ve2, i, c0, f.cols, lane, out, cap, count, f.tag);
+    p2 = p1;
+    p1 = cur;
+    cur = nxt;
+  }
+}
+
+__global__ void __launch_bounds__(256, 2)
+wb_diff2_batch_kernel(const BatchField* __restrict__ fields, unsigned n_fields, unsigned long long n_tasks,
+                      wb_diff2_tagged_entry* __restrict__ out, unsigned long long cap,
+                      unsigned long long* __restrict__ count) {
+  const unsigned lane = threadIdx.x & 31;
+  const unsigned long long warp0 = ((unsigned long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const unsigned long long n_warps = ((unsigned long long)gridDim.x * blockDim.x) >> 5;
+  for (unsigned long long task = warp0; task < n_tasks; task += n_warps) {
+    unsigned lo = 0, hi = n_fields - 1;                        // last field whose first task is <= task
+    while (lo < hi) {
+      const unsigned mid = (lo + hi + 1) >> 1;
+      if (fields[mid].task_begin <= task) lo = mid; else hi = mid - 1;
+    }
+    const BatchField f = fields[lo];
+    const unsigned long long local = task - f.task_begin;
+    switch (f.id_kind) {
+      case WB_ID_I64: batch_task<WB_ID_I64>(f, local, lane, out, cap, count); break;
+      case WB_ID_U16: batch_task<WB_ID_U16>(f, local, lane, out, cap, count); break;
+      case WB_ID_F32: batch_task<WB_ID_F32>(f, local, lane, out, cap, count); break;
+      default: batch_task<WB_ID_BF16>(f, local, lane, out, cap, count); break;
+    }
   }
 }
 
 }  // namespace
 
-extern "C" wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols,
-                                       wb_diff2_entry* out, uint64_t cap, uint64_t* count, void* cuda_stream) {
-  if (!field || !count || (!out && cap) || id_kind > WB_ID_BF16) return WB_ERR_INVALID_ARG;
-  if (rows == 0 || cols == 0) return WB_OK;
-  if (rows > (1ull << 40) || cols > (1ull << 40) || rows * cols > (1ull << 48)) return WB_ERR_INVALID_ARG;
-  if (rows > 1 && (rows >= (1ull << 31) || cols >= (1ull << 31))) return WB_ERR_INVALID_ARG;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+namespace {
+// One field, one launch of the tuned kernels (entries of type Entry, all carrying `tag`).
+template <typename Entry>
+cudaError_t launch_field(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols, Entry* out, uint64_t cap,
+                         unsigned long long* cnt, unsigned tag, cudaStream_t stream) {
   // Tasks are dealt to warps round robin, so the rows per task are chosen to give every warp the
   // same number of tasks (about kRowsPerTask rows each) instead of leaving a last, partly filled turn.
   const unsigned long long strips = (cols + kStrip - 1) / kStrip;
@@ -291,11 +371,10 @@ extern "C" wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint
   const unsigned long long tasks = strips * ((rows + rows_per_task - 1) / rows_per_task);
   const unsigned long long want = (tasks + 7) / 8;
   const unsigned grid = (unsigned)(want < resident ? want : resident);
-  auto* cnt = reinterpret_cast<unsigned long long*>(count);
-#define WB_DIFF2_LAUNCH(KIND)                                                                         \
-  do {                                                                                               \
-    if (rows == 1) wb_diff2_row_kernel<KIND><<<grid, 256, 0, stream>>>(field, cols, out, cap, cnt);   \
-    else wb_diff2_kernel<KIND><<<grid, 256, 0, stream>>>(field, rows, cols, rows_per_task, out, cap, cnt);   \
+#define WB_DIFF2_LAUNCH(KIND)                                                                                  \
+  do {                                                                                                        \
+    if (rows == 1) wb_diff2_row_kernel<KIND, Entry><<<grid, 256, 0, stream>>>(field, cols, out, cap, cnt, tag);  \
+    else wb_diff2_kernel<KIND, Entry><<<grid, 256, 0, stream>>>(field, rows, cols, rows_per_task, out, cap, cnt, tag); \
   } while (0)
   switch (id_kind) {
     case WB_ID_I64: WB_DIFF2_LAUNCH(WB_ID_I64); break;
@@ -304,5 +383,59 @@ extern "C" wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint
     default: WB_DIFF2_LAUNCH(WB_ID_BF16); break;
   }
 #undef WB_DIFF2_LAUNCH
+  return cudaGetLastError();
+}
+inline bool field_size_ok(uint64_t rows, uint64_t cols) {
+  if (rows > (1ull << 40) || cols > (1ull << 40) || rows * cols > (1ull << 48)) return false;
+  return !(rows > 1 && (rows >= (1ull << 31) || cols >= (1ull << 31)));
+}
+}  // namespace
+
+extern "C" wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols,
+                                       wb_diff2_entry* out, uint64_t cap, uint64_t* count, void* cuda_stream) {
+  if (!field || !count || (!out && cap) || id_kind > WB_ID_BF16) return WB_ERR_INVALID_ARG;
+  if (rows == 0 || cols == 0) return WB_OK;
+  if (!field_size_ok(rows, cols)) return WB_ERR_INVALID_ARG;
+  return launch_field(field, id_kind, rows, cols, out, cap, reinterpret_cast<unsigned long long*>(count), 0u,
+                      static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? WB_OK : WB_ERR_CUDA;
+}
+
+extern "C" size_t wb_diff2_batch_scratch_bytes(size_t n_fields) { return n_fields * sizeof(BatchField); }
+
+extern "C" wb_status wb_diff2_nonzeros_batch(const wb_diff2_field* fields, size_t n_fields, void* scratch,
+                                             size_t scratch_bytes, wb_diff2_tagged_entry* out, uint64_t cap,
+                                             uint64_t* count, void* cuda_stream) {
+  if (!count || (!out && cap) || (n_fields && (!fields || !scratch))) return WB_ERR_INVALID_ARG;
+  if (n_fields == 0) return WB_OK;
+  if (n_fields > (1u << 30) || scratch_bytes < n_fields * sizeof(BatchField) || ((uintptr_t)scratch & 15u))
+    return WB_ERR_INVALID_ARG;
+  std::vector<BatchField> host;
+  try { host.reserve(n_fields); } catch (const std::bad_alloc&) { return WB_ERR_OOM; }
+  unsigned long long tasks = 0;
+  for (size_t k = 0; k < n_fields; ++k) {
+    const wb_diff2_field& f = fields[k];
+    if (f.id_kind > WB_ID_BF16) return WB_ERR_INVALID_ARG;
+    if (f.rows == 0 || f.cols == 0) continue;                  // empty fields have no tasks
+    if (!f.field || !field_size_ok(f.rows, f.cols)) return WB_ERR_INVALID_ARG;
+    if (f.rows * f.cols >= kBatchLargeField) continue;          // launched on its own below
+    host.push_back(BatchField{f.field, f.rows, f.cols, tasks, f.id_kind, f.tag});
+    tasks += ((f.cols + kStrip - 1) / kStrip) * ((f.rows + kRowsPerTask - 1) / kRowsPerTask);
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  auto* cnt = reinterpret_cast<unsigned long long*>(count);
+  // large fields: the tuned single-field kernels keep the memory system busy by themselves
+  for (size_t k = 0; k < n_fields; ++k) {
+    const wb_diff2_field& f = fields[k];
+    if (f.rows == 0 || f.cols == 0 || f.rows * f.cols < kBatchLargeField) continue;
+    if (launch_field(f.field, f.id_kind, f.rows, f.cols, out, cap, cnt, f.tag, stream) != cudaSuccess) return WB_ERR_CUDA;
+  }
+  if (host.empty()) return WB_OK;
+  // the descriptors are copied before the call returns (pageable source), so `host` may go out of scope
+  if (cudaMemcpyAsync(scratch, host.data(), host.size() * sizeof(BatchField), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return WB_ERR_CUDA;
+  const unsigned long long want = (tasks + 7) / 8;
+  const unsigned grid = (unsigned)(want < 148ull * 2 ? want : 148ull * 2);
+  wb_diff2_batch_kernel<<<grid, 256, 0, stream>>>(static_cast<const BatchField*>(scratch), (unsigned)host.size(), tasks, out,
+                                                  cap, cnt);
   return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
 }

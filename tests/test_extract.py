@@ -154,3 +154,22 @@ def test_diff2_kernel_entry_point_checks_its_arguments_on_the_host():
     assert lib.wb_diff2_nonzeros(p, 0, 2, 1 << 31, p, 1, p, None) == INVALID
     assert lib.wb_diff2_nonzeros(p, 0, 1, (1 << 48) + 1, p, 1, p, None) == INVALID
     assert lib.wb_diff2_nonzeros(p, 0, 0, 4, p, 1, p, None) == 0                    # empty field: nothing to do
+
+
+def test_batched_diff2_entry_point_checks_its_arguments_on_the_host():
+    fields = np.zeros(2, wb.DIFF2_FIELD_DTYPE)
+    fields["field"] = 4096
+    fields["rows"], fields["cols"] = 4, 4
+    assert wb.wb_diff2_batch_scratch_bytes(2) >= 2 * 32
+    with pytest.raises(wb.WbError):                              # scratch too small
+        wb.wb_diff2_nonzeros_batch(fields, 4096, 8, 4096, 1, 4096)
+    with pytest.raises(wb.WbError):                              # scratch not 16-byte aligned
+        wb.wb_diff2_nonzeros_batch(fields, 4100, 1024, 4096, 1, 4096)
+    bad = fields.copy()
+    bad["id_kind"][1] = 7
+    with pytest.raises(wb.WbError):                              # unknown field kind
+        wb.wb_diff2_nonzeros_batch(bad, 4096, 1024, 4096, 1, 4096)
+    empty = fields.copy()
+    empty["rows"] = 0
+    wb.wb_diff2_nonzeros_batch(empty, 4096, 1024, 4096, 1, 4096)   # only empty fields: nothing is launched
+    wb.wb_diff2_nonzeros_batch(fields[:0], 0, 0, 4096, 1, 4096)    # no fields at all

@@ -182,3 +182,49 @@ def test_extracted_source_maps_give_the_same_remap(name, scale, bits):
     case.plan.check()
     for k, got in enumerate(case.dst_bits()):
         assert np.array_equal(got[want.written[k]], want.dst[k][want.written[k]]), wl.rollout.names[k]
+
+
+def test_batched_diff2_over_many_fields():
+    """One launch over fields of every kind and shape (one-row, thin, wide, tall, empty) returns, per tag,
+    exactly the entries of the definition."""
+    rng = np.random.default_rng(21)
+    shapes = [(1, 1), (1, 5000), (7, 33), (300, 700), (2, 9000), (0, 10), (1000, 3), (65, 257), (129, 1)] * 3
+    shapes += [(4100, 4100), (1, 16800000)]       # large fields: launched on their own by the entry point
+    tensors, want, desc = [], {}, []
+    for k, shp in enumerate(shapes):
+        kind = [wb.WB_ID_I64, wb.WB_ID_U16, wb.WB_ID_F32, wb.WB_ID_BF16][k % 4]
+        if shp[0] * shp[1] == 0:
+            desc.append((0, shp[0], shp[1], kind, k))
+            continue
+        a = _piecewise_affine(shp, rng, n_rect=4)
+        if kind == wb.WB_ID_I64:
+            t, ref = torch.from_numpy(a).to(DEV), a
+        elif kind == wb.WB_ID_U16:
+            ref = id_chunk(a, 0, 16)
+            t = torch.from_numpy(ref.astype(np.uint16).view(np.int16)).to(DEV)
+        elif kind == wb.WB_ID_F32:
+            ref = id_chunk(a, 0, 24)
+            t = torch.from_numpy(ref.astype(np.float32)).to(DEV)
+        else:
+            ref = id_chunk(a, 1, 8)
+            t = torch.from_numpy(ref.astype(np.float32)).to(torch.bfloat16).to(DEV)
+        tensors.append(t)
+        want[k] = oracle_entries(ref)
+        desc.append((t.data_ptr(), shp[0], shp[1], kind, k))
+    fields = np.array(desc, dtype=wb.DIFF2_FIELD_DTYPE)
+    nb = wb.wb_diff2_batch_scratch_bytes(len(fields))
+    scratch = torch.zeros(nb, dtype=torch.uint8, device=DEV)
+    cap = 1 << 18
+    out = torch.zeros(cap * 32, dtype=torch.uint8, device=DEV)
+    count = torch.zeros(1, dtype=torch.int64, device=DEV)
+    wb.wb_diff2_nonzeros_batch(fields, scratch.data_ptr(), nb, out.data_ptr(), cap, count.data_ptr(),
+                               torch.cuda.current_stream().cuda_stream)
+    n = int(count.item())
+    assert n == sum(len(v) for v in want.values()) and n <= cap
+    e = out.cpu().numpy().view(wb.DIFF2_TAGGED_ENTRY_DTYPE)[:n]
+    for k, w in want.items():
+        mine = np.sort(e[e["tag"] == k], order=["row", "col"])
+        assert len(mine) == len(w), k
+        assert np.array_equal(mine["row"], w["row"]) and np.array_equal(mine["col"], w["col"]) \
+            and np.array_equal(mine["value"], w["value"]), k
+    assert set(np.unique(e["tag"]).tolist()) <= set(want)
