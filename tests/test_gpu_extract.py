@@ -122,7 +122,31 @@ def test_diff2_kernel_reports_overflow_of_the_list():
     assert n2 == n == len(full)
 
 
-def extract_on_gpu(wl, side, chunk_bits):
+def batch_entries(tensors, kind, cap=1 << 20):
+    """wb_diff2_nonzeros_batch over {tag: 2-D device tensor}; returns {tag: sorted plain entries}."""
+    tags = sorted(tensors)
+    fields = np.array([(tensors[t].data_ptr(), tensors[t].shape[0], tensors[t].shape[1], kind, t) for t in tags],
+                      dtype=wb.DIFF2_FIELD_DTYPE)
+    nb = wb.wb_diff2_batch_scratch_bytes(len(fields))
+    scratch = torch.zeros(max(nb, 16), dtype=torch.uint8, device=DEV)
+    out = torch.zeros(cap * 32, dtype=torch.uint8, device=DEV)
+    count = torch.zeros(1, dtype=torch.int64, device=DEV)
+    wb.wb_diff2_nonzeros_batch(fields, scratch.data_ptr(), nb, out.data_ptr(), cap, count.data_ptr(),
+                               torch.cuda.current_stream().cuda_stream)
+    n = int(count.item())
+    assert n <= cap
+    e = out.cpu().numpy().view(wb.DIFF2_TAGGED_ENTRY_DTYPE)[:n]
+    res = {}
+    for t in tags:
+        m = e[e["tag"] == t]
+        plain = np.zeros(len(m), wb.DIFF2_ENTRY_DTYPE)
+        for f in ("row", "col", "value"):
+            plain[f] = m[f]
+        res[t] = np.sort(plain, order=["row", "col"])
+    return res
+
+
+def extract_on_gpu(wl, side, chunk_bits, batched=False):
     """Algorithm 1 on one side: K passes of load_weights with b-bit id chunks in the parameters' own
     dtype, diff2 per local tensor on the device, recombination and scan in the library."""
     declared = wl.trainer if side == "trainer" else wl.rollout
@@ -147,9 +171,16 @@ def extract_on_gpu(wl, side, chunk_bits):
             if x.dtype not in (torch.float32, torch.bfloat16):        # integer padding of the loaders
                 x = x.clamp_min(0)
             shapes[t] = tuple(x.shape)
+            if batched:
+                held[t] = x.contiguous()
+                return
             passes[t][k], n = gpu_entries(x, kind, cap=1 << 18)
             assert n == len(passes[t][k])
+        held = {}
         wl.load_side_shaped(side, values, sink)
+        if batched:                                   # every local tensor of the pass in one launch
+            for t, ent in batch_entries(held, kind).items():
+                passes[t][k] = ent
     base = wl.ckpt_base().astype(np.uint64)
     rows = np.array([c.rows for c in wl.ckpt], np.uint64)
     cols = np.array([c.cols for c in wl.ckpt], np.uint64)
@@ -169,8 +200,9 @@ def extract_on_gpu(wl, side, chunk_bits):
                                               ("cfg5", "small", 16), ("cfg1b", "full", 16)])
 def test_extracted_source_maps_give_the_same_remap(name, scale, bits):
     wl = make_workload(name, scale)
-    tl = extract_on_gpu(wl, "trainer", bits)
-    rl = extract_on_gpu(wl, "rollout", bits)
+    batched = name in ("cfg5", "cfg4")                # the many-tensor configurations go through the batched scan
+    tl = extract_on_gpu(wl, "trainer", bits, batched)
+    rl = extract_on_gpu(wl, "rollout", bits, batched)
     for lay, declared in ((tl, wl.trainer), (rl, wl.rollout)):
         for a, b in zip(predict_ids(lay, wl), predict_ids(declared, wl)):
             assert np.array_equal(a, b)                # same source map, element for element
