@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--grid-ctas", type=int, default=0)
     ap.add_argument("--path", default="remap",
-                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "rounds_fp8", "extract"],
+                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "rounds_fp8", "rounds_fp8_pipelined", "extract"],
                     help="remap: fused launch; pack_unpack: wb_pack + wb_unpack per round on one stream; "
                          "rounds: wb_transfer_rounds (depth-2 buckets, two streams); rounds_serial: its "
                          "unpipelined baseline; rounds_fp8: amax pass, then per round pack, quantise the bucket to FP8, "
@@ -332,9 +332,12 @@ def main():
                    for _ in range(2)]
 
     amax = qbucket = None
-    if args.path == "rounds_fp8":
+    qbuckets = None
+    if args.path in ("rounds_fp8", "rounds_fp8_pipelined"):
         amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
-        qbucket = torch.empty(max(plan.qbucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
+        qbuckets = [torch.empty(max(plan.qbucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
+                    for _ in range(2)]
+        qbucket = qbuckets[0]
 
     graph = None
     if args.cuda_graph and args.path == "remap":
@@ -354,6 +357,10 @@ def main():
             else:
                 plan.remap(stream)
             return 1
+        if args.path == "rounds_fp8_pipelined":
+            plan.transfer_rounds_fp8(buckets[0].data_ptr(), buckets[1].data_ptr(), qbuckets[0].data_ptr(),
+                                     qbuckets[1].data_ptr(), amax.data_ptr(), stream)
+            return 1 + 4 * n_rounds
         if args.path == "rounds_fp8":
             plan.absmax(amax.data_ptr(), stream)
             for r in range(n_rounds):

@@ -294,6 +294,15 @@ wb_status wb_bucket_quantize(const wb_plan* plan, size_t round, const void* buck
                              const float* amax, void* cuda_stream);
 wb_status wb_bucket_dequantize(const wb_plan* plan, size_t round, const void* qbucket, void* bucket,
                                const float* amax, void* cuda_stream);
+/* wb_transfer_rounds_fp8: wb_absmax and then every round of pack -> quantise | dequantise -> unpack with
+ * two bucket pairs in flight on the plan's two internal streams, ordered like wb_transfer_rounds
+ * (round r uses bucket r mod 2 and qbucket r mod 2; the transfer of the FP8 bucket would sit between
+ * the two halves).  Buffers DEVICE, 16-byte aligned, pairwise distinct: buckets >= the largest
+ * wb_plan_bucket_bytes, qbuckets >= the largest wb_plan_qbucket_bytes, amax wb_plan_num_ckpts floats.
+ * Work starts after what `cuda_stream` already holds; `cuda_stream` completes after the last assembly.
+ * Errors: INVALID_ARG, NOT_BOUND, OOM, CUDA. */
+wb_status wb_transfer_rounds_fp8(const wb_plan* plan, void* bucket0, void* bucket1, void* qbucket0, void* qbucket1,
+                                 float* amax, void* cuda_stream);
 
 /* wb_remap_host: the same transfer for callers whose weights are in HOST memory.  The remap
  * is cut into groups of consecutive tiles; for each group the trainer bytes it reads are copied

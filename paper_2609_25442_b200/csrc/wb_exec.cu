@@ -289,7 +289,8 @@ extern "C" wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bu
 
 // Internal streams and events shared by the multi-stream entry points (created on first use,
 // destroyed with the device tables).
-static wb_status ensure_pipeline(wb_plan* plan, size_t n_events) {
+namespace wbi {
+wb_status ensure_pipeline(wb_plan* plan, size_t n_events) {
   if (!plan->h2d_stream) {
     cudaStream_t a, b;
     if (cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking) != cudaSuccess) return WB_ERR_CUDA;
@@ -304,6 +305,8 @@ static wb_status ensure_pipeline(wb_plan* plan, size_t n_events) {
   }
   return WB_OK;
 }
+}  // namespace wbi
+using wbi::ensure_pipeline;
 
 // wb_transfer_rounds: all rounds of the two-pass path with two buckets in flight (Section 3.2:
 // consecutive rounds overlap; Section 4: a depth-2 buffer system).  Packing runs on one internal

@@ -193,6 +193,8 @@ struct wb_plan {
 namespace wbi {
 // implemented in wb_exec.cu
 void release_device_tables(wb_plan* plan);
+// the plan's two internal streams and at least n_events events (created on first use)
+wb_status ensure_pipeline(wb_plan* plan, size_t n_events);
 // implemented in wb_quant.cu
 void release_quant_tables(wb_plan* plan);
 }

@@ -380,3 +380,43 @@ extern "C" wb_status wb_bucket_dequantize(const wb_plan* plan, size_t round, con
                                                              static_cast<char*>(bucket), amax);
   return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
 }
+
+// All rounds of the quantised two-pass path with two bucket pairs in flight, like wb_transfer_rounds:
+// the packing stream runs amax, then per round pack -> quantise; the assembly stream dequantise -> unpack.
+extern "C" wb_status wb_transfer_rounds_fp8(const wb_plan* plan_c, void* bucket0, void* bucket1, void* qbucket0,
+                                            void* qbucket1, float* amax, void* cuda_stream) {
+  if (!plan_c || !bucket0 || !bucket1 || !qbucket0 || !qbucket1 || !amax) return WB_ERR_INVALID_ARG;
+  if (bucket0 == bucket1 || qbucket0 == qbucket1) return WB_ERR_INVALID_ARG;
+  if ((((uintptr_t)bucket0 | (uintptr_t)bucket1 | (uintptr_t)qbucket0 | (uintptr_t)qbucket1) & 15u)) return WB_ERR_INVALID_ARG;
+  if (!plan_c->bound) return WB_ERR_NOT_BOUND;
+  wb_plan* plan = const_cast<wb_plan*>(plan_c);      // lazily built pipeline state, not the plan itself
+  const size_t R = plan->rounds.size();
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  wb_status st = WB_OK;
+  try { st = ensure_pipeline(plan, 2 * R + 1); } catch (const std::bad_alloc&) { return WB_ERR_OOM; }
+  if (st != WB_OK) return st;
+  cudaStream_t ps = static_cast<cudaStream_t>(plan->h2d_stream), us = static_cast<cudaStream_t>(plan->d2h_stream);
+  auto packed = [&](size_t r) { return static_cast<cudaEvent_t>(plan->host_events[2 * r]); };
+  auto unpacked = [&](size_t r) { return static_cast<cudaEvent_t>(plan->host_events[2 * r + 1]); };
+  cudaEvent_t start = static_cast<cudaEvent_t>(plan->host_events[2 * R]);
+  if (cudaEventRecord(start, stream) != cudaSuccess) return WB_ERR_CUDA;
+  if (cudaStreamWaitEvent(ps, start, 0) != cudaSuccess || cudaStreamWaitEvent(us, start, 0) != cudaSuccess) return WB_ERR_CUDA;
+  if ((st = wb_absmax(plan, amax, ps)) != WB_OK) return st;
+  for (size_t r = 0; r < R; ++r) {
+    void* b = (r & 1) ? bucket1 : bucket0;
+    void* q = (r & 1) ? qbucket1 : qbucket0;
+    if (r >= 2 && cudaStreamWaitEvent(ps, unpacked(r - 2), 0) != cudaSuccess) return WB_ERR_CUDA;
+    if ((st = wb_pack(plan, r, b, ps)) != WB_OK) return st;
+    if ((st = wb_bucket_quantize(plan, r, b, q, amax, ps)) != WB_OK) return st;
+    if (cudaEventRecord(packed(r), ps) != cudaSuccess || cudaStreamWaitEvent(us, packed(r), 0) != cudaSuccess) return WB_ERR_CUDA;
+    // (the transfer of q would happen here)
+    if ((st = wb_bucket_dequantize(plan, r, q, b, amax, us)) != WB_OK) return st;
+    if ((st = wb_unpack(plan, r, b, us)) != WB_OK) return st;
+    if (cudaEventRecord(unpacked(r), us) != cudaSuccess) return WB_ERR_CUDA;
+  }
+  // with no rounds the amax pass is all there is: the caller's stream waits for the packing stream
+  cudaEvent_t last = R ? unpacked(R - 1) : start;
+  if (R == 0 && cudaEventRecord(start, ps) != cudaSuccess) return WB_ERR_CUDA;
+  if (cudaStreamWaitEvent(stream, last, 0) != cudaSuccess) return WB_ERR_CUDA;
+  return WB_OK;
+}

@@ -158,3 +158,36 @@ def test_rebinding_rebuilds_the_work_lists():
     plan.absmax(amax.data_ptr())
     torch.cuda.synchronize()
     assert torch.equal(amax, first * 2)
+
+
+@pytest.mark.parametrize("name,scale,budget", [("cfg1b", "full", 1 << 20), ("cfg3", "small", 1 << 20),
+                                               ("cfg5", "medium", 16 << 20)])
+def test_pipelined_quantised_rounds(name, scale, budget):
+    """wb_transfer_rounds_fp8 (two bucket pairs in flight on two internal streams) leaves the rollout tensors
+    the step-by-step quantised transfer leaves, which is the oracle's."""
+    wl = make_workload(name, scale)
+    dev = torch.device(DEV)
+    case = DeviceCase(wl, dev, bucket_budget_bytes=budget)
+    shapes = ckpt_shapes(wl)
+    want = run_quantised_transfer(case, wl.src_dtype, wl.dst_dtype, shapes, lambda t: t)
+    plan = case.plan
+    assert plan.num_rounds() > 2
+    nb = max(plan.bucket_bytes(r) for r in range(plan.num_rounds()))
+    nq = max(plan.qbucket_bytes(r) for r in range(plan.num_rounds()))
+    b = [torch.full((nb + 64,), 0x5A, dtype=torch.uint8, device=dev) for _ in range(2)]
+    q = [torch.full((nq + 64,), 0xA5, dtype=torch.uint8, device=dev) for _ in range(2)]
+    amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
+    side = torch.cuda.Stream(device=dev)
+    for stream in (None, side):
+        case.reset_dst()
+        torch.cuda.synchronize()
+        sp = 0 if stream is None else stream.cuda_stream
+        plan.transfer_rounds_fp8(b[0].data_ptr(), b[1].data_ptr(), q[0].data_ptr(), q[1].data_ptr(), amax.data_ptr(), sp)
+        (torch.cuda if stream is None else stream).synchronize()
+        dst_bits = case.dst_bits()
+        for t, v in want.items():
+            assert np.array_equal(checkpoint_view(t, shapes[t], case.rollout.slices, dst_bits)[0], v), wl.ckpt[t].name
+        plan.check()
+        assert all(bool((x[nb:] == 0x5A).all()) for x in b) and all(bool((x[nq:] == 0xA5).all()) for x in q)
+    with pytest.raises(wb.WbError):
+        plan.transfer_rounds_fp8(b[0].data_ptr(), b[0].data_ptr(), q[0].data_ptr(), q[1].data_ptr(), amax.data_ptr())

@@ -288,6 +288,9 @@ def test_error_bucket_too_small_and_unbound_execution():
     _expect("WB_ERR_NOT_BOUND", lambda: plan.bucket_quantize(0, 256, 512, 1024))
     _expect("WB_ERR_INVALID_ARG", lambda: plan.bucket_quantize(0, 258, 512, 1024))     # not 16-byte aligned
     _expect("WB_ERR_INVALID_ARG", lambda: plan.bucket_dequantize(99, 256, 512, 1024))  # no such round
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.transfer_rounds_fp8(256, 512, 1024, 2048, 4096))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds_fp8(256, 256, 1024, 2048, 4096))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds_fp8(256, 512, 1024, 2050, 4096))
     _expect("WB_ERR_INVALID_ARG", lambda: plan.bind([0] * plan.n_src, [0] * plan.n_dst))
     lib = wb.load()
     assert lib.wb_remap(None, None) == 1
