@@ -53,14 +53,17 @@ namespace {
 template <int ES, int ED>
 cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add, uint64_t dst_add,
                        cudaStream_t stream, uint32_t tile_off, uint32_t tile_count, bool whole) {
-  static bool configured[16] = {};
+  // the kernel needs more dynamic shared memory than the default limit: raise it once per device
+  // (on every launch for device ordinals beyond the table)
+  static std::atomic<bool> configured[64];
   int dev = 0;
-  cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 16 && !configured[dev]) {
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (!tracked || !configured[dev].load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(wb_exec_kernel<ES, ED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)Rings<ES, ED>::kDyn);
     if (e != cudaSuccess) return e;
-    configured[dev] = true;
+    if (tracked) configured[dev].store(true, std::memory_order_release);
   }
   wb_exec_kernel<ES, ED><<<dim3(plan->grid), dim3(kThreads), Rings<ES, ED>::kDyn, stream>>>(
       T.d_tiles + tile_off, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err, tile_count,
