@@ -199,16 +199,7 @@ template <int ES, int ED> __device__ __forceinline__ typename Elem<ES, ED>::V ca
   else if constexpr (ES == 4) return f32_to_bf16(raw);
   else return raw << 16;
 }
-// Shared-memory word accesses at a compile-time offset from a 32-bit shared-space address, and a
-// loop over compile-time indices (so that unrolled code uses immediate offsets).
-template <int OFF> __device__ __forceinline__ uint32_t lds32_at(uint32_t base) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(base), "n"(OFF));
-  return v;
-}
-template <int OFF> __device__ __forceinline__ void sts32_at(uint32_t base, uint32_t v) {
-  asm volatile("st.shared.u32 [%0+%1], %2;" ::"r"(base), "n"(OFF), "r"(v));
-}
+// A loop over compile-time indices (so that unrolled code can use immediate offsets).
 template <int I> struct Idx { static constexpr int value = I; };
 template <int I, int N, typename F> __device__ __forceinline__ void static_for(F&& fn) {
   if constexpr (I < N) {
@@ -247,9 +238,8 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
   // (multiple of 8, at most 64); no halo is needed when every run starts on a 16-byte boundary
   const uint32_t share = patch_bytes / 4;                    // words
   const bool aligned = (((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0;
-  // rows read past a block's end to complete its last window: NV-1 are needed; with 2-byte
-  // destinations 8 are read, which keeps the row count of a whole block a multiple of UA
-  const uint32_t halo = aligned ? 0u : (ED == 2 ? 8u : NV - 1), room = aligned ? 0u : 8u;
+  // rows read past a block's end to complete its last window
+  const uint32_t halo = aligned ? 0u : NV - 1, room = aligned ? 0u : 8u;
   const uint32_t rb = min(64u, ((share / 32 - 1) * PER_WORD - room) & ~7u);
   const uint32_t pitch_w = (rb + room) / PER_WORD + 1;      // odd: (rb+room)/PER_WORD is even
   const uint32_t tbase = smem_u32(patch);
@@ -258,28 +248,15 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
   const size_t sps = (size_t)f.ssr * ES;
   if (warp >= nb) return;
 
-  // nl: rows loaded = own rows + halo.  full: every lane has a column and every batch all its rows,
-  // so loads and shared-memory writes need no predicates; whole: in addition the block has all its
-  // rows and halo and does not begin a run, so every window it owns is a full vector.
-  struct Block { uint32_t i0, j0, ni, nj, nl; bool full, whole; };
+  struct Block { uint32_t i0, j0, ni, nj, nl; };      // nl: rows loaded = own rows + halo
   auto block_of = [&](uint32_t b) {
     const uint32_t bi = b / nbj, bj = b - bi * nbj;
     const uint32_t i0 = bi * rb, ni = min(rb, f.nr - i0);
-    const uint32_t nj = min(32u, f.nc - bj * 32), nl = min(ni + halo, f.nr - i0);
-    const bool full = nj == 32 && nl % UA == 0;
-    return Block{i0, bj * 32, ni, nj, nl, full, full && nl == rb + halo && (aligned || i0 != 0)};
+    return Block{i0, bj * 32, ni, min(32u, f.nc - bj * 32), min(ni + halo, f.nr - i0)};
   };
   // phase A, loads: UA rows of this lane's column into registers
   auto issue = [&](const Block& k, uint32_t r0, uint32_t (&dst)[UA]) {
     const char* src = f.s + ((size_t)(k.i0 + r0) * f.ssr + k.j0 + lane) * ES;
-    if (k.full) {
-#pragma unroll
-      for (int u = 0; u < UA; ++u, src += sps) {
-        if constexpr (ES == 4) dst[u] = __ldcs(reinterpret_cast<const uint32_t*>(src));
-        else dst[u] = __ldcs(reinterpret_cast<const uint16_t*>(src));
-      }
-      return;
-    }
 #pragma unroll
     for (int u = 0; u < UA; ++u) {
       dst[u] = 0;
@@ -293,20 +270,6 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
   auto consume = [&](const Block& k, uint32_t r0, const uint32_t (&v)[UA]) {
     if (lane >= k.nj) return;
     const uint32_t trow = tbase + lane * pitch_w * 4;
-    if (k.full) {
-      const uint32_t at = trow + r0 * ED;
-      if constexpr (ED == 2)
-        static_for<0, UA / 2>([&](auto uc) {
-          constexpr int u = decltype(uc)::value * 2;
-          sts32_at<u * 2>(at, pack_pair16<ES>(v[u], v[u + 1]));
-        });
-      else
-        static_for<0, UA>([&](auto uc) {
-          constexpr int u = decltype(uc)::value;
-          sts32_at<u * 4>(at, (uint32_t)cast_raw<ES, ED>(v[u]));
-        });
-      return;
-    }
     if constexpr (ED == 2) {
 #pragma unroll
       for (int u = 0; u < UA; u += 2)
@@ -325,34 +288,6 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
   // 16-byte pieces.
   auto phase_b = [&](const Block& k) {
     __syncwarp();
-    if (k.whole) {
-      // lane = destination run; rb / NV full windows, the first one `lead` rows into the block
-      char* run = f.d + (size_t)(k.j0 + lane) * f.dsc * ED;
-      const uint32_t a = (uint32_t)(((uintptr_t)run / ED + k.i0) & (NV - 1));
-      const uint32_t lead = a ? NV - a : 0;
-      char* out = run + (size_t)(k.i0 + lead) * ED;
-      const uint32_t trow = tbase + lane * pitch_w * 4;
-      if constexpr (ED == 4) {
-        uint32_t p = trow + lead * 4;
-        for (uint32_t w = 0; w < rb / NV; ++w, p += 16, out += 16)
-          st16(out, make_uint4(lds32_at<0>(p), lds32_at<4>(p), lds32_at<8>(p), lds32_at<12>(p)));
-      } else if (aligned) {
-        uint32_t p = trow;
-        for (uint32_t w = 0; w < rb / NV; ++w, p += 16, out += 16)
-          st16(out, make_uint4(lds32_at<0>(p), lds32_at<4>(p), lds32_at<8>(p), lds32_at<12>(p)));
-      } else {
-        uint32_t p = trow + (lead >> 1) * 4;
-        const uint32_t sh = (lead & 1u) * 16u;                     // odd lead: windows straddle the words
-        for (uint32_t w = 0; w < rb / NV; ++w, p += 16, out += 16) {
-          const uint32_t w0 = lds32_at<0>(p), w1 = lds32_at<4>(p), w2 = lds32_at<8>(p), w3 = lds32_at<12>(p),
-                         w4 = lds32_at<16>(p);
-          st16(out, make_uint4(__funnelshift_r(w0, w1, sh), __funnelshift_r(w1, w2, sh),
-                               __funnelshift_r(w2, w3, sh), __funnelshift_r(w3, w4, sh)));
-        }
-      }
-      __syncwarp();
-      return;
-    }
     const uint32_t wins = (k.ni + NV - 1) / NV;                    // windows per run, at most
     const uint32_t total = k.nj * wins;
     for (uint32_t idx = lane; idx < total; idx += 32) {
