@@ -149,22 +149,18 @@ __device__ __forceinline__ uint4 staged_unit(const char* row, uint32_t o) {
 
 // Workers: rows staged in shared memory -> destination rows.  Every row is cut into 16-byte
 // aligned destination slots; full slots are one vector store, ragged first/last slots are
-// element stores.  A group of G lanes (G = 32, 16 or 8 by row length) takes G consecutive slots
-// of one row; groups are independent (no barrier).  `t` is the rotated worker thread index.
+// element stores.  Threads are independent (no barrier).  `t` is the rotated worker thread index.
 template <int ES, int ED>
 __device__ __forceinline__ void staged_rows(const ChunkDesc& d, const char* stage, uint32_t t) {
   using E = Elem<ES, ED>;
   constexpr uint32_t NV = 16 / ED;
   const uint32_t n = d.nc;
   const uint32_t smax = (n + 2 * NV - 2) / NV;     // slots a row can touch
-  const uint32_t gs = smax > 16 ? 5u : (smax > 8 ? 4u : 3u);
-  const uint32_t G = 1u << gs;
-  const uint32_t nb = (smax + G - 1) >> gs;        // slot blocks per row
-  const uint32_t tasks = d.nr * nb;
   const uint32_t lead0 = (uint32_t)d.src & 15u, dlead = (uint32_t)d.sps & 15u;
-  const uint32_t lig = t & (G - 1);
-  for (uint32_t task = t >> gs; task < tasks; task += (uint32_t)kWorkers >> gs) {
-    const uint32_t r = task / nb, k = (task - r * nb) * G + lig;
+  // the slots of all rows, numbered row by row, are dealt to the threads in order: neighbouring
+  // lanes take neighbouring slots of a row, and no lane idles at the end of a row
+  for (uint32_t idx = t; idx < d.nr * smax; idx += (uint32_t)kWorkers) {
+    const uint32_t r = idx / smax, k = idx - r * smax;
     const uint64_t D = d.dst + (uint64_t)r * d.dps;
     const uint32_t a = (uint32_t)(D & 15u) / ED;   // elements of slot 0 that precede the row
     const int32_t e0 = (int32_t)(k * NV) - (int32_t)a;
