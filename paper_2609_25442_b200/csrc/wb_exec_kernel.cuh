@@ -273,7 +273,7 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     } else if (f.kind == KIND_TRANS && f.n_extra == 0 && (size_t)f.nc * ES >= kTransMinPiece && f.nr >= kTransMinRows) {
       // staged transposition: chunks of kTransPiece bytes of columns x kOwn rows (+ halo), rows fastest
       constexpr uint32_t kOwn = (((uint32_t)kSlotBytes / kTransPitch) - kTransHalo) & ~7u;
-      constexpr uint32_t kCols = (kTransPiece - 16) / ES;
+      constexpr uint32_t kCols = kTransChunkBytes / ES;
       // no halo when every destination run starts on a 16-byte boundary: windows never straddle chunks
       const uint32_t halo = ((((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0 && kOwn % (16 / ED) == 0) ? 0u : kTransHalo;
       for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += kCols)

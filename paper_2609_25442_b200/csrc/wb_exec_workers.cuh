@@ -43,7 +43,7 @@ constexpr int kWorkerWarps = kWorkers / 32;
 constexpr size_t kStagedMinRowBytes = WB_STAGED_MIN_ROW_BYTES;   // shorter rows take the warp-level path
 
 enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3, MODE_TRANS = 4 };
-// Staged transposition: a chunk is up to kTransPiece - 16 bytes of consecutive source columns (the
+// Staged transposition: a chunk is kTransChunkBytes of consecutive source columns (the
 // 16-byte aligned superset of a row piece is one 16-byte asynchronous copy per lane of the producer
 // warp - bulk copies this small are limited by their issue rate) by as many source rows as fit a slot.  Row r of the chunk lands at r * kTransPitch + 16 * ((r / NV) & 7) in the slot
 // (NV = destination elements per 16 bytes): the pitch is a multiple of 128 bytes, so lanes that
@@ -54,6 +54,10 @@ enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3, MO
 #endif
 constexpr uint32_t kTransPiece = WB_TRANS_PIECE;                      // bytes one warp instruction copies per row (aligned superset)
 constexpr uint32_t kTransPitch = kTransPiece + 128;
+// source bytes of a chunk's row pieces: at most kTransPiece - 16 (the aligned superset must fit);
+// 480 makes 120 four-byte columns x 8 windows = 960 windows, two for each of the 480 worker threads
+constexpr uint32_t kTransChunkBytes = 480;
+static_assert(kTransChunkBytes + 16 <= kTransPiece, "the aligned superset of a row piece must fit the copy");
 constexpr uint32_t kTransHalo = 8;
 #ifndef WB_TRANS_MIN_PIECE
 #define WB_TRANS_MIN_PIECE 128

@@ -209,7 +209,7 @@ struct TileBuilder {
     }
     const uint32_t kind = trans ? KIND_TRANS : KIND_ELEM;
     // 2-D blocks, multiples of 64 on both axes where the extent allows
-    // transposed: one staged transposition chunk of the executor wide (496 source bytes) and as tall
+    // transposed: one staged transposition chunk of the executor wide (480 source bytes) and as tall
     // as the tile size allows, so that a tile writes long pieces of few destination runs and the
     // element stores at the two ends of a run piece are rare
 #ifndef WB_TRANS_NARROW_MIN_BYTES
@@ -217,7 +217,7 @@ struct TileBuilder {
 #endif
     // (small slabs keep four chunks per tile: there the number of tiles matters more)
     const bool narrow = nr * nc * (uint64_t)(es + ed) >= WB_TRANS_NARROW_MIN_BYTES;
-    uint64_t tc = std::min<uint64_t>(nc, trans ? (narrow ? 496 / es : 496) : 512);
+    uint64_t tc = std::min<uint64_t>(nc, trans ? (narrow ? 480 / es : 480) : 512);
     uint64_t tr = std::min<uint64_t>(nr, std::max<uint64_t>(64, roundup(T / tc, 64)));
     if (trans) {
       // rows fastest: consecutive tiles continue the same destination runs
