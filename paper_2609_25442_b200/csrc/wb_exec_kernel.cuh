@@ -276,10 +276,13 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
       constexpr uint32_t kCols = kTransChunkBytes / ES;
       // no halo when every destination run starts on a 16-byte boundary: windows never straddle chunks
       const uint32_t halo = ((((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0 && kOwn % (16 / ED) == 0) ? 0u : kTransHalo;
-      for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += kCols)
+      // equal column shares per chunk (no thin last chunk), a multiple of four columns
+      const uint32_t n_col = (f.nc + kCols - 1) / kCols;
+      const uint32_t cols = min(kCols, (((f.nc + n_col - 1) / n_col) + 3u) & ~3u);
+      for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cols)
         for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += kOwn)
           push_trans(f.s + ((size_t)i0 * f.ssr + j0) * ES, f.d + ((size_t)j0 * f.dsc + i0) * ED,
-                     min(kOwn + halo, f.nr - i0), min(kCols, f.nc - j0), (uint64_t)f.ssr * ES,
+                     min(kOwn + halo, f.nr - i0), min(cols, f.nc - j0), (uint64_t)f.ssr * ES,
                      (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0), i0 == 0 ? 1u : 0u);
     } else {
       push_simple(MODE_COOP, k, 1, &cur);   // narrow transposes, short rows, fan-out: the workers share the tile

@@ -218,6 +218,12 @@ struct TileBuilder {
     // (small slabs keep four chunks per tile: there the number of tiles matters more)
     const bool narrow = nr * nc * (uint64_t)(es + ed) >= WB_TRANS_NARROW_MIN_BYTES;
     uint64_t tc = std::min<uint64_t>(nc, trans ? (narrow ? 480 / es : 480) : 512);
+    if (trans && nc > tc) {
+      // equal column shares instead of full tiles plus a thin remainder (which would be too narrow
+      // for the staged path)
+      const uint64_t n_col = (nc + tc - 1) / tc;
+      tc = std::min<uint64_t>(tc, roundup((nc + n_col - 1) / n_col, 8));
+    }
     uint64_t tr = std::min<uint64_t>(nr, std::max<uint64_t>(64, roundup(T / tc, 64)));
     if (trans) {
       // rows fastest: consecutive tiles continue the same destination runs
