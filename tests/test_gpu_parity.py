@@ -162,6 +162,40 @@ def test_fuzz_layouts(device, seed):
         assert np.array_equal(to_bits(t), want.dst[k]), k
 
 
+@pytest.mark.parametrize("seed", range(40))
+def test_fuzz_layouts_with_larger_tensors(device, seed):
+    """The same fuzz with dimensions up to 2500, so that staged rows, staged transposition chunks and
+    multi-tile slabs are reached; automatic, 64 KiB and 4 KiB tiles."""
+    src_dt, dst_dt = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][seed % 4]
+    shapes, tl, rl = fuzz_case(50000 + seed, src_dt, dst_dt, max_dim=[300, 900, 2500][seed % 3])
+    rng = np.random.default_rng(seed)
+    ck = [random_bits(rng, r * c, src_dt) for (r, c) in shapes]
+    src_host = scatter_checkpoint(tl, ck)
+    src = RankArenas(tl.tensors, device, fill_byte=0)
+    dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+    for t, h in zip(src.tensors, src_host):
+        t.copy_(from_bits(h))
+    plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices),
+                   tile_bytes=[0, 65536, 4096][seed % 3], bucket_budget_bytes=[0, 1 << 16][seed % 2])
+    bind(plan, src, dst)
+    want = remap_oracle(shapes, tl.tensors, tl.slices, rl.tensors, rl.slices, src_host,
+                        prefill_bits(rl, BITS[dst_dt]))
+    plan.remap()
+    torch.cuda.synchronize()
+    for k, t in enumerate(dst.tensors):
+        assert np.array_equal(to_bits(t), want.dst[k]), k
+    for a in dst.arenas.values():
+        a.fill_(CANARY)
+    for r in range(plan.num_rounds()):
+        bucket = torch.empty(plan.bucket_bytes(r) + 16, dtype=torch.uint8, device=device)
+        plan.pack(r, bucket.data_ptr())
+        plan.unpack(r, bucket.data_ptr())
+    torch.cuda.synchronize()
+    for k, t in enumerate(dst.tensors):
+        assert np.array_equal(to_bits(t), want.dst[k]), k
+    plan.check()
+
+
 def _one_tensor_plan(n, src_dt, dst_dt, device, src_off=0, dst_off=0):
     tl, rl = Layout("t"), Layout("r")
     tl.add_tensor("T", 0, src_dt, n + src_off)
