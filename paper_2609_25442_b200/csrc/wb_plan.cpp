@@ -225,6 +225,11 @@ struct TileBuilder {
       tc = std::min<uint64_t>(tc, roundup((nc + n_col - 1) / n_col, 8));
     }
     uint64_t tr = std::min<uint64_t>(nr, std::max<uint64_t>(64, roundup(T / tc, 64)));
+    if (trans && nr > tr) {
+      // equal row shares too (multiples of a chunk's 64 rows): no tile of a few left-over rows
+      const uint64_t n_row = (nr + tr - 1) / tr;
+      tr = std::min<uint64_t>(tr, roundup((nr + n_row - 1) / n_row, 64));
+    }
     if (trans) {
       // rows fastest: consecutive tiles continue the same destination runs
       for (uint64_t j = 0; j < nc; j += tc)
