@@ -63,6 +63,10 @@ def parse_args():
                          "experiment of the paper's Appendix D, on the kernels alone)")
     ap.add_argument("--static-schedule", action="store_true",
                     help="fixed per-block tile ranges instead of run-time batches")
+    ap.add_argument("--also", default="cfg4,cfg3,cfg5",
+                    help="default run (cfg2, fused remap, one GPU): after the headline measurement, time these "
+                         "workloads too through the same wb_remap call and list them in config.workloads "
+                         "(empty string: none)")
     return ap.parse_args()
 
 
@@ -210,7 +214,8 @@ def run_reference(args):
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "u16" if wl.src_dtype == 1 else "f32->bf16",
            "data": "synthetic", "config": {"workload": wl.name, "note": "each step = bounded sample"},
-           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
+                            "sample": desc},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out))
@@ -285,6 +290,67 @@ def run_extract(args):
                       "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
                                    "frac": gbs / peak, "traffic": None, "kernel": "wb_diff2_kernel"},
                       "gpu_launches": args.steps * len(fields)}))
+
+
+def hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def measure_remap(name, scale, args, dev, local_rank):
+    """One more workload through the same call as the headline one: build, bind, warm up, time
+    `steps` wb_remap launches with CUDA events on the launching stream, sample the clocks, check the
+    plan's error word.  Returns the entry of config.workloads; releases everything it allocated."""
+    from paper_2609_25442_b200 import binding as wb
+    from paper_2609_25442_b200.device import RankArenas, bind
+    wl = make_workload(name, scale)
+    es, ed = (4 if wl.src_dtype == 0 else 2), (4 if wl.dst_dtype == 0 else 2)
+    need = sum(int(t["numel"]) for t in wl.trainer.tensors) * es + sum(int(t["numel"]) for t in wl.rollout.tensors) * ed
+    free = torch.cuda.mem_get_info(dev)[0]
+    entry = {"workload": wl.name, "dtype": {0: "f32", 1: "bf16"}[wl.src_dtype] + "->" + {0: "f32", 1: "bf16"}[wl.dst_dtype]}
+    if need * 1.02 + (2 << 30) > free:
+        entry["skipped"] = f"needs {need / 1e9:.1f} GB of device memory, {free / 1e9:.1f} GB free"
+        return entry
+    t0 = time.perf_counter()
+    plan = wb.Plan(wb.Layout(wl.trainer.tensors, wl.trainer.slices), wb.Layout(wl.rollout.tensors, wl.rollout.slices),
+                   tile_bytes=args.tile_bytes, grid_ctas=args.grid_ctas)
+    plan_s = time.perf_counter() - t0
+    stats = plan.stats()
+    src = RankArenas(wl.trainer.tensors, dev, fill_byte=0)
+    dst = RankArenas(wl.rollout.tensors, dev, fill_byte=0)
+    wl.load_side("trainer", lambda i: wl.ckpt_values(i, dev), lambda k, t: src.tensors[k].copy_(t))
+    bind(plan, src, dst)
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream().cuda_stream
+    bytes_step = stats["src_bytes_read"] + stats["dst_bytes_written"]
+    for _ in range(max(args.warmup, 3)):
+        plan.remap(stream)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    evs[0].record()
+    for k in range(args.steps):
+        plan.remap(stream)
+        evs[k + 1].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    plan.check()                                   # a bounded wait that ran out inside a launch fails the run
+    per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
+    ms = float(np.mean(per_step))
+    gbs = bytes_step / (ms * 1e-3) / 1e9
+    peak, peak_src = hbm_peak()
+    entry.update({"bytes_per_step": bytes_step, "ms_per_step": ms, "best_ms": float(min(per_step)), "gbs": gbs,
+                  "frac_of_measured": gbs / peak, "peak_source": peak_src, "frac_of_8TBs": gbs / 8000.0,
+                  "tiles": stats["n_tiles_remap"], "plan_build_s": plan_s, "steps": args.steps,
+                  "gpu_launches": args.steps, "l2": "inputs_larger_than_l2", "clocks": clocks,
+                  "traffic": int(NCU_TRAFFIC_RATIO[name] * bytes_step) if name in NCU_TRAFFIC_RATIO else None})
+    del plan, src, dst
+    torch.cuda.empty_cache()
+    return entry
 
 
 # ------------------------------------------------------------------------------------------------
@@ -399,6 +465,7 @@ def main():
     barrier()
     torch.cuda.nvtx.range_pop()
     clocks = sampler.stop() if rank == 0 else None
+    plan.check()                                       # a bounded wait that ran out inside a launch fails the run
     total_ms = evs[0].elapsed_time(evs[-1])
     per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
     total_ms = wbdist.max_over_ranks(dist, total_ms, dev)
@@ -406,12 +473,7 @@ def main():
     value = wbdist.aggregate_gbs(world, bytes_step, ms_per_step)
 
     # ---- roofline of the dominant (only) kernel --------------------------------------------------
-    peak, peak_src = FALLBACK_HBM_GBS, "fallback"
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
-    except Exception:
-        pass
+    peak, peak_src = hbm_peak()
     launch_ms = float(np.mean(per_step)) / (1 if args.path == "remap" else 1)
     achieved = bytes_step / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -507,8 +569,23 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         dt, moved, desc = oracle_sample(wl, lambda k: to_bits_np(src.tensors[k]))
-        cpu = {"value": moved / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
-               "seconds": dt}
+        cpu = {"value": moved / dt / 1e9, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
+               "sample": desc, "seconds": dt}
+
+    # ---- the other workloads, through the same call (default run on one GPU only) -------------------
+    others = None
+    if rank == 0 and world == 1 and args.path == "remap" and args.workload == "cfg2" and args.scale == "full" and args.also:
+        headline = {"workload": wl.name, "dtype": {0: "f32", 1: "bf16"}[wl.src_dtype] + "->" + {0: "f32", 1: "bf16"}[wl.dst_dtype],
+                    "bytes_per_step": bytes_step, "ms_per_step": ms_per_step, "best_ms": float(min(per_step)),
+                    "gbs": value, "frac_of_measured": value / peak, "peak_source": peak_src,
+                    "frac_of_8TBs": value / 8000.0, "tiles": stats["n_tiles_remap"], "plan_build_s": plan_s,
+                    "steps": args.steps, "gpu_launches": launches, "l2": "inputs_larger_than_l2", "clocks": clocks,
+                    "traffic": roofline["traffic"]}
+        del plan, src, dst, buckets
+        torch.cuda.empty_cache()
+        others = [headline]
+        for name in [x for x in args.also.split(",") if x]:
+            others.append(measure_remap(name, args.scale, args, dev, local_rank))
 
     if rank == 0:
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -526,6 +603,8 @@ def main():
                           "multi_gpu": "independent replicas, no collective"},
                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                "gpu_launches": launches, "pct_of_8TBs_nominal": 100.0 * value / world / 8000.0}
+        if others is not None:
+            out["config"]["workloads"] = others
         if sweep is not None:
             out["budget_sweep"] = sweep
         if fp8 is not None:

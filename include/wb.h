@@ -164,8 +164,8 @@ typedef struct {
 enum { WB_TABLE_REMAP = 0, WB_TABLE_PACK = 1, WB_TABLE_UNPACK = 2 };
 
 /* ---- layouts (host only) --------------------------------------------------------------
- * wb_layout_describe: ingest one side's source map (Section 3.1, "sequence of slice-copy
- * operations ... each optionally involving transpose").  `tensors` and `slices` are host
+ * wb_layout_describe: ingest one side's source map (Section 3.1: a list of slice-copy
+ * operations, any of which may also transpose).  `tensors` and `slices` are host
  * arrays, copied.  Checks indices, dtypes, stride shapes, that every slice stays inside its
  * checkpoint tensor and its local tensor, and that a checkpoint tensor has one shape.
  * Errors: INVALID_ARG, DTYPE, SHAPE_MISMATCH, OUT_OF_RANGE, OOM. */
@@ -229,6 +229,12 @@ wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, size_t n_src,
  * applied here so the bucket carries destination-dtype bytes.
  * wb_unpack: Section 3.2 assembly kernel: payloads of `bucket` -> rollout tensors (fused
  * qkv / gate_up concatenation, head regrouping, expert stacking, transposition, fan-out).
+ * The device that was current at wb_plan_bind must be current for every call that launches on the plan
+ * (INVALID_ARG otherwise: the tables hold that device's addresses).
+ * One launch of a tile table at a time: the run-time tile scheduler keeps its counters per table in the
+ * plan's device memory, so two calls on the same plan whose GPU work can overlap (different streams
+ * with no ordering between them) must not use the same table - wb_remap twice, or wb_pack / wb_unpack
+ * of the same round twice.  Calls ordered on one stream, or by events, are fine.
  * Errors: INVALID_ARG, NOT_BOUND, CUDA. */
 wb_status wb_remap(const wb_plan* plan, void* cuda_stream);
 wb_status wb_pack(const wb_plan* plan, size_t round, void* bucket, void* cuda_stream);
@@ -240,7 +246,7 @@ wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bucket, void*
 wb_status wb_plan_check(const wb_plan* plan);
 
 /* wb_plan_check_replicas (device, synchronous): the plan reads a replicated checkpoint region from
- * one trainer replica only (Section 3.2: "the trainer workers collectively send only one copy"),
+ * one trainer replica only (Section 3.2: together the trainers send a single copy of the model),
  * which presumes the replicas are bit-identical.  This debug pass compares every pair of replicas
  * the source layout declares, element by element, on the bound tensors.  *n_mismatches (host, may
  * be NULL) receives the number of differing elements.  OK, REPLICA_MISMATCH, NOT_BOUND, CUDA. */
@@ -252,9 +258,9 @@ wb_status wb_plan_check_replicas(const wb_plan* plan, uint64_t* n_mismatches, vo
  * did not have to, CUDA / OOM on runtime errors.  The context stays usable afterwards. */
 wb_status wb_wait_probe(uint32_t limit_ms, void* cuda_stream);
 
-/* wb_transfer_rounds: every round of the two-pass path, pipelined (Section 3.2: "overlapping
- * consecutive rounds"; Section 4: a depth-2 buffer system lets adjacent rounds proceed in
- * parallel).  Round r packs into bucket r mod 2 on one internal stream and is assembled from it on
+/* wb_transfer_rounds: every round of the two-pass path, pipelined (Section 3.2: consecutive
+ * rounds overlap; Section 4: with two buffers per side, neighbouring rounds run at the same
+ * time).  Round r packs into bucket r mod 2 on one internal stream and is assembled from it on
  * a second internal stream; pack(r) waits until unpack(r-2) has released that bucket, unpack(r)
  * waits for pack(r).  Equivalent to wb_pack + wb_unpack for rounds 0..R-1 in order; the rollout
  * tensors end up as after wb_remap.  Work starts after what `cuda_stream` already holds and
@@ -270,12 +276,14 @@ wb_status wb_transfer_rounds(const wb_plan* plan, void* bucket0, void* bucket1, 
 
 /* ---- FP8 quantisation of a round's bucket (device; asynchronous on `cuda_stream`) -----------------
  * Section 5 ("Parameter precision mismatch") sketches it: trainer tensors are quantised before the
- * transfer, which needs the full tensor gathered first; "in each transfer round, the trainers would
- * gather the sharded tensors to be quantized" before the write.  The paper fixes no rule.  The one
+ * transfer, which needs the full tensor, so every round starts with the trainers gathering the
+ * shards of the tensors to be quantised.  The paper fixes no rule.  The one
  * built: FP8 E4M3 (largest finite value 448), one scale per checkpoint tensor, s = amax / 448 and
- * r = 448 / amax in fp32 (s = r = 1 if amax = 0), amax = the tensor's largest magnitude in the
- * destination dtype; q = e4m3(x * r), fp32 multiplication, round to nearest even, saturating,
- * NaN -> 0x7F; x' = cast_dst(value(q) * s).  Checkpoint tensors are numbered 0 .. wb_plan_num_ckpts-1 in ascending
+ * r = 448 / amax in fp32 (s = r = 1 if amax = 0; an s that rounds to zero becomes 2^-149), amax =
+ * the tensor's largest magnitude in the destination dtype; q = e4m3(x * r), fp32 multiplication,
+ * round to nearest even, saturating, NaN -> 0x7F; a tensor whose r is not finite (amax below
+ * 448 / FLT_MAX, about 1.3e-36) is encoded as q = e4m3(x / s) instead, so that zeros stay zeros and
+ * nothing turns NaN whatever the magnitudes; x' = cast_dst(value(q) * s).  Checkpoint tensors are numbered 0 .. wb_plan_num_ckpts-1 in ascending
  * order of their ids (wb_plan_ckpt_ids).
  * wb_absmax: the gather, as a maximum: one pass over the de-duplicated trainer regions of the bound
  *   tensors; amax (DEVICE, wb_plan_num_ckpts floats) is zeroed and then filled.  A tensor that holds a
@@ -346,8 +354,14 @@ wb_status wb_remap_host(const wb_plan* plan, const void* const* host_src, size_t
  *   - All calls on a device share the one array, and it keeps the previous call's contents: each
  *     call rewrites the table it needs and zeroes the error word, in stream order.  Two calls
  *     whose GPU work can overlap (different streams without an ordering between them) race on
- *     the array; order them on one stream or with events.  Host-side preparation is serialised
- *     internally.
+ *     the array; order them on one stream or with events.  Host-side preparation, the upload of
+ *     the table and the launch are serialised internally, so host threads that call on one stream
+ *     cannot interleave.
+ *   - The table (up to 4 MiB) is uploaded from ordinary host memory: the call blocks the host
+ *     until the runtime has staged it.  A call on a stream that is being captured is refused with
+ *     WB_ERR_INVALID_ARG (a replay would upload whatever a later call left in the staging image).
+ *   - A bounded wait that ran out inside the kernel is reported only by a call made with
+ *     WB_STATIC_SYNC_CHECK (there is no bound plan whose wb_plan_check could be asked).
  * Errors: INVALID_ARG, STATIC_LIMIT, CUDA, INTERNAL (only with WB_STATIC_SYNC_CHECK). */
 #define WB_STATIC_SCRATCH_BYTES (4u << 20)
 #define WB_STATIC_SYNC_CHECK 1u

@@ -1,19 +1,26 @@
 """FP8 quantisation of a transfer bucket (test infrastructure).
 
 Section 5 of the paper ("Parameter precision mismatch") only sketches this step: trainer tensors
-are quantised before the transfer, which needs the full tensor gathered first, and "in each
-transfer round, the trainers would gather the sharded tensors to be quantized" before the write.
-It fixes no quantisation rule.  The reading taken here (parity unpinned by the paper, pinned to
-the arithmetic below):
+are quantised before the transfer, which needs the full tensor gathered first, so in every round
+the trainers first gather the shards of the tensors that are to be quantised.  It fixes no
+quantisation rule.  The reading taken here (parity unpinned by the paper, pinned to the arithmetic
+below):
 
   format   FP8 E4M3 (4 exponent bits, bias 7, 3 mantissa bits, no infinities, largest finite
            value 448, NaN = S.1111.111).
   scale    one per checkpoint tensor: s = amax / 448 and its counterpart r = 448 / amax, both one
            fp32 division, amax the largest magnitude of the tensor's elements in the destination
-           dtype (the "gather"); s = r = 1 if amax = 0.
+           dtype (the "gather"); s = r = 1 if amax = 0.  A quotient amax / 448 that rounds to zero
+           (amax at most 224 units of the smallest subnormal) is replaced by the smallest subnormal,
+           2^-149, so that s is never zero for a tensor that is not.
   encode   q = e4m3(x * r): fp32 multiplication with the reciprocal scale (the convention of FP8
            training libraries: one division per tensor, none per element), round to nearest with
            ties to even, magnitudes beyond the largest finite value saturate to it, NaN -> 0x7F.
+           The rule must be total: for amax below 448 / FLT_MAX (about 1.3e-36, still a normal
+           number) r overflows to infinity, which would turn every zero into NaN and every other
+           element into +-amax.  A tensor whose r is not finite is therefore encoded by division,
+           q = e4m3(x / s), which is finite for every element because s is not zero.  (A NaN amax
+           keeps r and s NaN: the whole tensor is NaN either way.)
   decode   x' = cast_dst(value(q) * s): fp32 multiplication, then the destination dtype's rounding.
 
 The quantised object is the bucket payload (checkpoint format, destination dtype), so for an
@@ -89,11 +96,16 @@ def amax_bits(bits: np.ndarray, dtype: int) -> np.uint32:
 
 
 def scale_of(amax: np.uint32) -> np.float32:
+    """The scale amax / 448 (fp32 division; 1 for an all-zero tensor; never zero otherwise: a
+    quotient that rounds to zero becomes the smallest subnormal)."""
     a = np.array([amax], np.uint32).view(np.float32)[0]
     if a == 0:
         return np.float32(1.0)
-    with np.errstate(invalid="ignore"):
-        return np.float32(a / np.float32(E4M3_MAX))
+    with np.errstate(invalid="ignore", under="ignore"):
+        s = np.float32(a / np.float32(E4M3_MAX))
+    if s == 0:
+        s = np.array([1], np.uint32).view(np.float32)[0]          # 2^-149
+    return s
 
 
 def rscale_of(amax: np.uint32) -> np.float32:
@@ -105,13 +117,16 @@ def rscale_of(amax: np.uint32) -> np.float32:
         return np.float32(np.float32(E4M3_MAX) / a)
 
 
-def quantize(bits: np.ndarray, dtype: int, rscale: np.float32) -> np.ndarray:
-    with np.errstate(invalid="ignore", over="ignore"):
-        y = to_f32(bits, dtype) * np.float32(rscale)
+def quantize(bits: np.ndarray, dtype: int, scale: np.float32, rscale: np.float32) -> np.ndarray:
+    """Codes of a tensor's elements: x * rscale, or x / scale when rscale is not finite (a tensor
+    of tiny magnitudes, or one that holds a NaN)."""
+    x = to_f32(bits, dtype)
+    with np.errstate(invalid="ignore", over="ignore", under="ignore", divide="ignore"):
+        y = x * np.float32(rscale) if np.isfinite(rscale) else x / np.float32(scale)
     return e4m3_encode(y)
 
 
 def dequantize(codes: np.ndarray, dtype: int, scale: np.float32) -> np.ndarray:
-    with np.errstate(invalid="ignore", over="ignore"):
+    with np.errstate(invalid="ignore", over="ignore", under="ignore"):
         v = e4m3_decode(codes) * np.float32(scale)
     return from_f32(v, dtype)

@@ -77,6 +77,7 @@ wb_status launch_table(const wb_plan* plan, const TileTable& T, uint64_t src_add
                        uint32_t es, uint32_t ed, cudaStream_t stream, uint32_t tile_off = 0,
                        uint32_t tile_count = 0) {
   if (T.tiles.empty()) return WB_OK;
+  if (!wbi::on_bound_device(plan)) return WB_ERR_INVALID_ARG;
   const bool whole = tile_count == 0;
   if (whole) tile_count = (uint32_t)T.tiles.size();
   cudaError_t e;
@@ -93,6 +94,10 @@ inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 }  // namespace
 
 namespace wbi {
+bool on_bound_device(const wb_plan* plan) {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev == plan->device;
+}
 void release_device_tables(wb_plan* plan) {
   release_quant_tables(plan);
   if (plan->d_arena) {
@@ -227,6 +232,7 @@ __global__ void wb_compare_kernel(const DCompare* __restrict__ ops, uint32_t n_o
 extern "C" wb_status wb_plan_check_replicas(const wb_plan* plan, uint64_t* n_mismatches, void* cuda_stream) {
   if (!plan) return WB_ERR_INVALID_ARG;
   if (!plan->bound) return WB_ERR_NOT_BOUND;
+  if (!wbi::on_bound_device(plan)) return WB_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   unsigned long long bad = 0;
   const uint32_t n = (uint32_t)plan->replica_pairs.size();
@@ -264,6 +270,7 @@ extern "C" wb_status wb_wait_probe(uint32_t limit_ms, void* cuda_stream) {
 extern "C" wb_status wb_plan_check(const wb_plan* plan) {
   if (!plan) return WB_ERR_INVALID_ARG;
   if (!plan->bound) return WB_ERR_NOT_BOUND;
+  if (!wbi::on_bound_device(plan)) return WB_ERR_INVALID_ARG;
   uint32_t e = 0;
   if (cudaMemcpy(&e, plan->d_err, sizeof(e), cudaMemcpyDeviceToHost) != cudaSuccess) return WB_ERR_CUDA;
   return e == 0 ? WB_OK : WB_ERR_INTERNAL;
@@ -532,9 +539,21 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxStaticDevices) return WB_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  g_static_lock.lock();
+  // The table is uploaded from one shared host image: a captured copy would read that image again at
+  // every replay, with whatever a later call left there.  Refuse instead of recording that.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) return WB_ERR_CUDA;
+  if (cap != cudaStreamCaptureStatusNone) return WB_ERR_INVALID_ARG;
+  // One lock covers building the image, the upload and the launch: two host threads that call on
+  // the same stream must not interleave as copy A, copy B, kernel B, kernel A (kernel A would walk
+  // B's table).
+  struct Guard {
+    SpinLock& l;
+    explicit Guard(SpinLock& x) : l(x) { l.lock(); }
+    ~Guard() { l.unlock(); }
+  } guard(g_static_lock);
   wb_status st = static_setup(dev);
-  if (st != WB_OK) { g_static_lock.unlock(); return st; }
+  if (st != WB_OK) return st;
   char* dbase = static_cast<char*>(g_static_ptr[dev]);
   // the array keeps the previous call's contents: rebuild everything this launch reads, and
   // zero the error word and the scheduling counters (first 256 bytes)
@@ -556,11 +575,9 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
     hx[k] = DDst{(uint64_t)(uintptr_t)dst_base[h.tensor] + h.off * ed, h.sr, h.sc};
   }
   std::memcpy(g_static_stage + off_begin, T.cta_begin.data(), T.cta_begin.size() * sizeof(uint32_t));
-  // pageable source: the runtime has taken its copy of the image when this returns, so the host
-  // image can be reused by the next call
-  cudaError_t e = cudaMemcpyAsync(dbase, g_static_stage, total, cudaMemcpyHostToDevice, stream);
-  g_static_lock.unlock();
-  if (e != cudaSuccess) return WB_ERR_CUDA;
+  // pageable source: the runtime has taken its copy of the image when this returns (the call
+  // blocks the host for that long), so the host image can be reused by the next call
+  if (cudaMemcpyAsync(dbase, g_static_stage, total, cudaMemcpyHostToDevice, stream) != cudaSuccess) return WB_ERR_CUDA;
 
   const DTile* d_tiles = reinterpret_cast<const DTile*>(dbase + off_tiles);
   const DDst* d_extras = reinterpret_cast<const DDst*>(dbase + off_extras);

@@ -195,6 +195,9 @@ namespace wbi {
 void release_device_tables(wb_plan* plan);
 // the plan's two internal streams and at least n_events events (created on first use)
 wb_status ensure_pipeline(wb_plan* plan, size_t n_events);
+// true if the current device is the one the plan's tables and tensors were bound on (a launch from
+// another device would dereference addresses of the bound one)
+bool on_bound_device(const wb_plan* plan);
 // implemented in wb_quant.cu
 void release_quant_tables(wb_plan* plan);
 }

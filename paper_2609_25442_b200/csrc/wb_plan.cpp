@@ -8,7 +8,7 @@
 //   tiles            slabs cut into near-equal-byte tiles, contiguous tile ranges per
 //                    thread block balanced by bytes
 //   rounds           payload chunks assigned to roughly equal rounds whose buckets fit the
-//                    budget (Section 3.2 "round-based, batched transfer pipeline";
+//                    budget (Section 3.2: the transfer runs in rounds, each a batch;
 //                    Appendix D: the round count follows from the buffer budget)
 #include <algorithm>
 #include <chrono>

@@ -3,7 +3,10 @@
 // The paper fixes no rule; the one built here: FP8 E4M3, one scale per checkpoint tensor,
 // s = amax / 448 and r = 448 / amax with amax the tensor's largest magnitude in the destination dtype
 // (the gather becomes a maximum over every trainer shard of the tensor), q = e4m3(x * r) with round
-// to nearest even and saturation, x' = cast(value(q) * s).
+// to nearest even and saturation, x' = cast(value(q) * s).  The rule is total: a quotient amax / 448
+// that rounds to zero becomes the smallest subnormal, and a tensor whose r is not finite (amax below
+// 448 / FLT_MAX, or NaN) is encoded as q = e4m3(x / s) instead, so zeros stay zeros whatever the
+// tensor's magnitude.
 //
 //   wb_absmax            one pass over the de-duplicated trainer regions -> amax per checkpoint tensor
 //   wb_bucket_quantize   a packed round's bucket (destination dtype) -> FP8 bucket, same element offsets
@@ -65,7 +68,9 @@ __device__ __forceinline__ uint32_t f32x2_to_bf16x2(float lo, float hi) {
 }
 __device__ __forceinline__ float scale_of(const float* __restrict__ amax, uint32_t ckpt) {
   const float a = __ldg(amax + ckpt);
-  return a == 0.f ? 1.f : __fdiv_rn(a, 448.f);
+  if (a == 0.f) return 1.f;
+  const float s = __fdiv_rn(a, 448.f);
+  return s == 0.f ? __uint_as_float(1u) : s;      // never zero for a tensor that is not: 2^-149
 }
 __device__ __forceinline__ float rscale_of(const float* __restrict__ amax, uint32_t ckpt) {
   const float a = __ldg(amax + ckpt);
@@ -143,6 +148,17 @@ wb_quantize_kernel(const QuantItem* __restrict__ items, uint32_t n_items, const 
     const char* x = bucket + it.off * ED;
     uint8_t* out = q + it.off;
     const uint32_t body = it.n & ~7u;
+    if (!isfinite(r)) {
+      // tiny magnitudes (448 / amax overflows) or a NaN maximum: divide by the scale, element by element
+      const float s = scale_of(amax, it.ckpt);
+      for (uint32_t e = threadIdx.x; e < it.n; e += blockDim.x) {
+        float f;
+        if (ED == 2) f = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(x)[e] << 16);
+        else f = reinterpret_cast<const float*>(x)[e];
+        out[e] = (uint8_t)(f32x2_to_e4m3x2(__fdiv_rn(f, s), 0.f) & 0xFFu);
+      }
+      continue;
+    }
 #pragma unroll 2
     for (uint32_t e = threadIdx.x * 8; e < body; e += blockDim.x * 8) {
       float f[8];
@@ -318,6 +334,7 @@ extern "C" size_t wb_plan_qbucket_bytes(const wb_plan* plan, size_t round) {
 extern "C" wb_status wb_absmax(const wb_plan* plan_c, float* amax, void* cuda_stream) {
   if (!plan_c || !amax) return WB_ERR_INVALID_ARG;
   if (!plan_c->bound) return WB_ERR_NOT_BOUND;
+  if (!on_bound_device(plan_c)) return WB_ERR_INVALID_ARG;
   wb_plan* plan = const_cast<wb_plan*>(plan_c);      // lazily built work lists, not the plan itself
   wb_status st = WB_OK;
   try { st = build_tables(plan); } catch (const std::bad_alloc&) { return WB_ERR_OOM; }
@@ -339,6 +356,7 @@ static wb_status quant_common(const wb_plan* plan_c, size_t round, const void* a
   if (!plan_c || !a || !b || !amax || round >= plan_c->rounds.size()) return WB_ERR_INVALID_ARG;
   if (((uintptr_t)a & 15u) || ((uintptr_t)b & 15u)) return WB_ERR_INVALID_ARG;
   if (!plan_c->bound) return WB_ERR_NOT_BOUND;
+  if (!on_bound_device(plan_c)) return WB_ERR_INVALID_ARG;
   wb_plan* plan = const_cast<wb_plan*>(plan_c);
   wb_status st = WB_OK;
   try { st = build_tables(plan); } catch (const std::bad_alloc&) { return WB_ERR_OOM; }

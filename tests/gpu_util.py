@@ -3,7 +3,8 @@ its C ABI, bring results back as raw bits."""
 import numpy as np
 import torch
 
-from helpers import to_bits
+from helpers import ckpt_shapes, to_bits
+from oracle import remap_oracle
 from paper_2609_25442_b200 import binding as wb
 from paper_2609_25442_b200.device import RankArenas, bind
 
@@ -60,3 +61,11 @@ def prefill_bits(rollout, dtype_bits):
     if dtype_bits == np.uint32:
         pat |= pat << 16
     return [np.full(int(t["numel"]), pat, dtype_bits) for t in rollout.tensors]
+
+
+def oracle_for(case: DeviceCase):
+    """The CPU oracle's rollout tensors for the trainer bits a case holds on the device."""
+    bits = np.uint32 if case.dst.tensors[0].dtype == torch.float32 else np.uint16
+    return remap_oracle(ckpt_shapes(case.wl), case.trainer.tensors, case.trainer.slices,
+                        case.rollout.tensors, case.rollout.slices, case.src_bits(),
+                        prefill_bits(case.rollout, bits))

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import CANARY, DeviceCase, prefill_bits
+from gpu_util import CANARY, DeviceCase, oracle_for, prefill_bits
 from helpers import ckpt_shapes, from_bits, fuzz_case, random_bits, scatter_checkpoint, to_bits
 from oracle import checkpoint_view, remap_oracle
 from oracle.cast import cast_bits, f32_to_bf16_bits
@@ -23,13 +23,6 @@ CASES = [("cfg1", "full"), ("cfg1b", "full"), ("cfg1c", "full"), ("cfg2", "small
 def device():
     assert torch.cuda.is_available()
     return torch.device("cuda:0")
-
-
-def oracle_for(case: DeviceCase):
-    wl = case.wl
-    return remap_oracle(ckpt_shapes(wl), case.trainer.tensors, case.trainer.slices,
-                        case.rollout.tensors, case.rollout.slices, case.src_bits(),
-                        prefill_bits(case.rollout, BITS[int(case.rollout.tensors[0]["dtype"])]))
 
 
 def assert_dst_equals(case, want):

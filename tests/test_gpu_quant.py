@@ -62,7 +62,7 @@ def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id)
             r0, c0, nr, nc = (int(e[k]) for k in ("r0", "c0", "nr", "nc"))
             rect = views[t][r0:r0 + nr, c0:c0 + nc].reshape(-1)
             off = int(e["bucket_off"]) // ed
-            codes = quant.quantize(rect, wl_dst_dtype, rscales[t])
+            codes = quant.quantize(rect, wl_dst_dtype, scales[t], rscales[t])
             assert np.array_equal(q[off:off + nr * nc], codes), (r, t)
             back = quant.dequantize(codes, wl_dst_dtype, scales[t])
             assert same_bits(b2[off:off + nr * nc], back, wl_dst_dtype), (r, t)
@@ -73,7 +73,7 @@ def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id)
         plan.unpack(r, bucket2.data_ptr())
     torch.cuda.synchronize()
     plan.check()
-    return {t: quant.dequantize(quant.quantize(v.reshape(-1), wl_dst_dtype, rscales[t]), wl_dst_dtype,
+    return {t: quant.dequantize(quant.quantize(v.reshape(-1), wl_dst_dtype, scales[t], rscales[t]), wl_dst_dtype,
                                 scales[t]).reshape(v.shape) for t, v in views.items()}
 
 
@@ -96,7 +96,9 @@ def test_quantised_rounds_match_the_oracle(name, scale, budget):
 @pytest.mark.parametrize("dts", [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)])
 def test_special_tensors(dts):
     """All-zero tensors (scale 1), a tensor with an infinity (scale infinite), one with a NaN (no scale), odd
-    lengths (scalar tails) and values that land exactly between two codes."""
+    lengths (scalar tails), values that land exactly between two codes, tensors of tiny magnitudes (the
+    reciprocal scale overflows: encoded by division; zeros must stay zeros), a subnormal maximum so small
+    that amax / 448 rounds to zero (scale = smallest subnormal), and a maximum of FLT_MAX."""
     sdt, ddt = dts
     n = 1003
     rng = np.random.default_rng(3)
@@ -106,7 +108,16 @@ def test_special_tensors(dts):
             np.concatenate([[np.nan, 2.0], rng.normal(0, 1, n - 2)]).astype(np.float32),
             # amax = 448, so the scale is 1 and the midpoints between codes are hit exactly
             np.concatenate([[448.0, -448.0, 1.0625, 1.1875, 0.0009765625, 17.0, 27.0, 464.0 / 2], rng.uniform(-448, 448, n - 8)]
-                           ).astype(np.float32)]
+                           ).astype(np.float32),
+            np.concatenate([[0.0, 1e-37, -5e-38, 2e-38, -0.0], rng.normal(0, 3e-38, n - 5)]).astype(np.float32),
+            np.concatenate([[0.0, 1.2e-39, -0.0], rng.normal(0, 4e-40, n - 3)]).astype(np.float32),       # subnormals
+            (np.concatenate([[0, 150, -3, 1, -0.0], rng.integers(-150, 151, n - 5)]) * 2.0 ** -149).astype(np.float32),
+            np.concatenate([[3.4028234663852886e38, 0.0, -1e38], np.clip(rng.normal(0, 1e38, n - 3), -3e38, 3e38)]).astype(np.float32)]
+    if WB_BF16 in (sdt, ddt):
+        # bf16 on either side: the fp32 subnormal-count tensor would round to zero or to coarse steps; use bf16's own
+        # smallest subnormals (2^-133) instead, and the largest finite bf16 value
+        vals[7] = (np.concatenate([[0, 2, -1, 1, -0.0], rng.integers(-2, 3, n - 5)]) * 2.0 ** -133).astype(np.float32)
+        vals[8] = np.concatenate([[3.3895313892515355e38, 0.0, -1e38], np.clip(rng.normal(0, 1e38, n - 3), -3e38, 3e38)]).astype(np.float32)
     tl, rl = Layout("t"), Layout("r")
     for k in range(len(vals)):
         tl.add_tensor(f"T{k}", k % 2, sdt, n)

@@ -1,8 +1,9 @@
 """wb_remap_static: the remap for callers that cannot allocate device memory (an inference
 engine whose KV-cache pool already owns all free HBM, a fixed start-up memory budget).  Its
 tile table lives in the library's fixed 4 MiB device array instead of a cudaMalloc'd arena.
-The output must equal what the ordinary bind + wb_remap path writes, bit for bit, on two calls
-in a row that use different plans (so stale contents of the shared array would show).
+The output must equal the CPU oracle's rollout tensors, and what the ordinary bind + wb_remap
+path writes, bit for bit, on two calls in a row that use different plans (so stale contents of
+the shared array would show).
 
 This file is named to be collected last."""
 import gc
@@ -11,7 +12,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import DeviceCase
+from gpu_util import DeviceCase, oracle_for
 from paper_2609_25442_b200 import binding as wb
 from paper_2609_25442_b200.device import RankArenas
 from wb_workloads import WB_BF16, Layout, make_workload
@@ -21,9 +22,11 @@ pytestmark = pytest.mark.gpu
 
 def _reference_and_static(device, name, scale, **opts):
     case = DeviceCase(make_workload(name, scale), device, **opts)
+    want = oracle_for(case).dst                           # the CPU oracle
     case.plan.remap()                                     # existing entry point
     torch.cuda.synchronize()
-    want = case.dst_bits()
+    for got, w in zip(case.dst_bits(), want):
+        assert np.array_equal(got, w)
     case.reset_dst()
     # a second, never-bound plan of the same layouts goes through the no-allocation entry point
     plan = wb.Plan(wb.Layout(case.trainer.tensors, case.trainer.slices),
