@@ -173,6 +173,22 @@ wb_status wb_layout_describe(const wb_tensor_desc* tensors, size_t n_tensors,
                              const wb_slice* slices, size_t n_slices, wb_layout** out);
 void wb_layout_free(wb_layout* layout);
 
+/* wb_layout_add_flat_range (host, pure arithmetic): the slice-copy operations of one piece of a
+ * flat shard (Section 3.1: a source map is a list of slice copies over the checkpoint's 2-D views).
+ * A trainer that keeps parameters flattened (FSDP-style flat shards) holds, of the row-major
+ * ckpt_rows x ckpt_cols checkpoint tensor `ckpt_tensor`, the flat element range [begin, end)
+ * contiguously in local tensor `tensor` from element `local_off` on.  In checkpoint coordinates that
+ * range is at most three rectangles - the rest of the first row, the full rows, the start of the
+ * last row.  Writes them to out[0 .. cap) as wb_slice records (row-contiguous: stride_c = 1,
+ * stride_r = the rectangle's width), in ascending flat order, ready to be
+ * appended to the slice list given to wb_layout_describe, and stores their number (0..3) in *n_out;
+ * with out == NULL only the number is computed.  An empty range gives 0 slices.
+ * Errors: INVALID_ARG (n_out NULL, ckpt_cols 0, cap too small for the slices needed), OUT_OF_RANGE
+ * (begin > end or end > ckpt_rows * ckpt_cols). */
+wb_status wb_layout_add_flat_range(uint32_t tensor, uint64_t local_off, uint64_t ckpt_tensor,
+                                   uint64_t ckpt_rows, uint64_t ckpt_cols, uint64_t begin, uint64_t end,
+                                   wb_slice* out, size_t cap, size_t* n_out);
+
 /* ---- planning (host only, no CUDA call) -------------------------------------------------
  * wb_plan_build: Section 3.2.  Intersects the two source maps per checkpoint tensor
  * (element correspondence), de-duplicates replicas on both sides so that every consumed

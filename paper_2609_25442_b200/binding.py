@@ -75,7 +75,7 @@ TILE_VIEW_DTYPE = np.dtype([
 assert BUCKET_ENTRY_DTYPE.itemsize == 64 and TILE_VIEW_DTYPE.itemsize == 64
 
 EXPORTS = [
-    "wb_layout_describe", "wb_layout_free", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
+    "wb_layout_describe", "wb_layout_free", "wb_layout_add_flat_range", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
     "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
     "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_transfer_rounds",
@@ -102,6 +102,8 @@ def load() -> C.CDLL:
     lib.wb_layout_describe.argtypes = [vp, sz, vp, sz, C.POINTER(vp)]
     lib.wb_layout_free.argtypes = [vp]
     lib.wb_layout_free.restype = None
+    lib.wb_layout_add_flat_range.argtypes = [C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64,
+                                             C.c_uint64, vp, sz, C.POINTER(sz)]
     lib.wb_plan_build.argtypes = [vp, vp, C.POINTER(wb_plan_opts), C.POINTER(vp)]
     lib.wb_plan_free.argtypes = [vp]
     lib.wb_plan_free.restype = None
@@ -180,6 +182,17 @@ class Layout:
 
 def wb_layout_describe(tensors: np.ndarray, slices: np.ndarray) -> Layout:
     return Layout(tensors, slices)
+
+
+def wb_layout_add_flat_range(tensor: int, local_off: int, ckpt_tensor: int, ckpt_rows: int, ckpt_cols: int,
+                             begin: int, end: int) -> np.ndarray:
+    """The <= 3 slice records of flat checkpoint range [begin, end) held contiguously from local_off on."""
+    lib = load()
+    out = np.zeros(3, SLICE_DTYPE)
+    n = C.c_size_t()
+    _check(lib.wb_layout_add_flat_range(tensor, local_off, ckpt_tensor, ckpt_rows, ckpt_cols, begin, end,
+                                        out.ctypes.data, 3, C.byref(n)), "wb_layout_add_flat_range")
+    return out[:n.value]
 
 
 class Plan:

@@ -123,3 +123,42 @@ extern "C" wb_status wb_layout_describe(const wb_tensor_desc* tensors, size_t n_
 }
 
 extern "C" void wb_layout_free(wb_layout* layout) { delete layout; }
+
+// A flat range of a row-major matrix in checkpoint coordinates: the rest of the first row, the full
+// rows, the start of the last row (Section 3.1 slice copies of a flat shard).
+extern "C" wb_status wb_layout_add_flat_range(uint32_t tensor, uint64_t local_off, uint64_t ckpt_tensor,
+                                              uint64_t ckpt_rows, uint64_t ckpt_cols, uint64_t begin, uint64_t end,
+                                              wb_slice* out, size_t cap, size_t* n_out) {
+  if (!n_out || ckpt_cols == 0) return WB_ERR_INVALID_ARG;
+  const unsigned __int128 numel = (unsigned __int128)ckpt_rows * ckpt_cols;
+  if (begin > end || (unsigned __int128)end > numel) return WB_ERR_OUT_OF_RANGE;
+  wb_slice tmp[3];
+  size_t n = 0;
+  auto rect = [&](uint64_t r0, uint64_t c0, uint64_t nr, uint64_t nc) {
+    wb_slice s{};
+    s.tensor = tensor;
+    s.local_off = local_off + (r0 * ckpt_cols + c0 - begin);
+    s.stride_r = (int64_t)nc;
+    s.stride_c = 1;
+    s.ckpt_tensor = ckpt_tensor; s.ckpt_rows = ckpt_rows; s.ckpt_cols = ckpt_cols;
+    s.r0 = r0; s.c0 = c0; s.nr = nr; s.nc = nc;
+    tmp[n++] = s;
+  };
+  if (end > begin) {
+    uint64_t rb = begin / ckpt_cols, cb = begin % ckpt_cols;
+    const uint64_t re = end / ckpt_cols, ce = end % ckpt_cols;
+    if (rb == re) {
+      rect(rb, cb, 1, end - begin);
+    } else {
+      if (cb) { rect(rb, cb, 1, ckpt_cols - cb); ++rb; }
+      if (re > rb) rect(rb, 0, re - rb, ckpt_cols);
+      if (ce) rect(re, 0, 1, ce);
+    }
+  }
+  if (out) {
+    if (cap < n) return WB_ERR_INVALID_ARG;
+    for (size_t k = 0; k < n; ++k) out[k] = tmp[k];
+  }
+  *n_out = n;
+  return WB_OK;
+}

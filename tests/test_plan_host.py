@@ -13,6 +13,7 @@ from oracle.cast import cast_bits
 from paper_2609_25442_b200 import binding as wb
 from plan_interp import run_table
 from wb_workloads import SLICE_DTYPE, TENSOR_DTYPE, WB_BF16, WB_F32, Layout, make_workload
+from wb_workloads.rng import SplitMix64
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SMALL = [("cfg1", "full"), ("cfg1b", "full"), ("cfg1c", "full"), ("cfg2", "small"),
@@ -314,3 +315,46 @@ def test_interleaved_column_blocks_are_not_an_overlap():
     dst = [np.zeros(32, np.uint32)]
     run_table(plan.tiles(wb.WB_TABLE_REMAP), src, dst, None, WB_F32, WB_F32)
     assert np.array_equal(dst[0], src[0])
+
+
+def test_flat_range_helper_gives_the_rectangles_of_a_flat_shard():
+    """wb_layout_add_flat_range against brute force on ids (every element of the flat range is described
+    exactly once, at the local offset it has in the shard) and against the generator's own statement."""
+    from wb_workloads.configs import flat_range_rects
+    rng = SplitMix64(77)
+    cases = [(1, 1, 0, 1), (4, 6, 0, 24), (4, 6, 0, 0), (4, 6, 5, 7), (4, 6, 6, 12), (4, 6, 7, 11), (4, 6, 3, 23)]
+    for _ in range(300):
+        rows, cols = rng.randint(1, 12), rng.randint(1, 12)
+        b = rng.randint(0, rows * cols)
+        cases.append((rows, cols, b, rng.randint(b, rows * cols)))
+    for rows, cols, b, e in cases:
+        local_off = 5
+        got = wb.wb_layout_add_flat_range(3, local_off, 9, rows, cols, b, e)
+        assert len(got) <= 3
+        ids = np.arange(rows * cols)
+        local = np.full(local_off + (e - b), -1)
+        local[local_off:] = ids[b:e]
+        seen = np.zeros(local.size, bool)
+        for s in got:
+            assert (int(s["tensor"]), int(s["ckpt"]), int(s["ckpt_rows"]), int(s["ckpt_cols"])) == (3, 9, rows, cols)
+            for i in range(int(s["nr"])):
+                for j in range(int(s["nc"])):
+                    x = int(s["local_off"]) + i * int(s["stride_r"]) + j * int(s["stride_c"])
+                    assert local[x] == (int(s["r0"]) + i) * cols + int(s["c0"]) + j and not seen[x]
+                    seen[x] = True
+        assert seen[local_off:].all() and not seen[:local_off].any()
+        want = flat_range_rects(cols, b, e)
+        assert [(int(s["r0"]), int(s["c0"]), int(s["nr"]), int(s["nc"]), int(s["local_off"]) - local_off + b)
+                for s in got] == want
+    with pytest.raises(wb.WbError) as err:
+        wb.wb_layout_add_flat_range(0, 0, 0, 4, 6, 5, 25)
+    assert err.value.name == "WB_ERR_OUT_OF_RANGE"
+    with pytest.raises(wb.WbError) as err:
+        wb.wb_layout_add_flat_range(0, 0, 0, 4, 6, 7, 5)
+    assert err.value.name == "WB_ERR_OUT_OF_RANGE"
+    with pytest.raises(wb.WbError) as err:
+        wb.wb_layout_add_flat_range(0, 0, 0, 4, 0, 0, 0)
+    assert err.value.name == "WB_ERR_INVALID_ARG"
+    # the records are accepted by wb_layout_describe as they are
+    sl = wb.wb_layout_add_flat_range(0, 0, 0, 4, 6, 3, 23)
+    wb.Layout(np.array([(0, WB_F32, 20)], TENSOR_DTYPE), sl)
