@@ -219,6 +219,21 @@ size_t wb_plan_bucket_bytes(const wb_plan* plan, size_t round);   /* 0 if round 
  * and the total count to *n. */
 wb_status wb_plan_bucket_entries(const wb_plan* plan, size_t round, wb_bucket_entry* out,
                                  size_t cap, size_t* n);
+/* One (receiver, sender) region of a round's bucket (Section 3.2: packing builds one contiguous buffer
+ * per receiver; here the receivers' buffers are laid end to end, and inside a receiver's buffer each
+ * sender has its own 256-byte aligned piece).  Region k of wb_plan_bucket_regions covers bucket bytes
+ * [off, off + bytes): everything virtual trainer rank `sender` packs for virtual rollout rank `receiver`
+ * in this round.  Regions are listed in bucket order and do not overlap.  In a deployment with the
+ * virtual ranks spread over several GPUs, region (r, s) is what travels from the GPU of s to the GPU
+ * of r between wb_pack_ranks and wb_unpack_ranks; the sizes are fixed by the plan. */
+typedef struct {
+  uint32_t receiver, sender;
+  uint64_t off, bytes;
+} wb_bucket_region;
+wb_status wb_plan_bucket_regions(const wb_plan* plan, size_t round, wb_bucket_region* out, size_t cap,
+                                 size_t* n);
+/* Number of virtual ranks on each side (highest rank named by a tensor + 1). */
+wb_status wb_plan_num_ranks(const wb_plan* plan, uint32_t* n_trainer, uint32_t* n_rollout);
 /* Host view of a tile table (`which` = WB_TABLE_*; `round` ignored for WB_TABLE_REMAP). */
 wb_status wb_plan_tiles(const wb_plan* plan, int which, size_t round, wb_tile_view* out,
                         size_t cap, size_t* n);
@@ -255,6 +270,31 @@ wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, size_t n_src,
 wb_status wb_remap(const wb_plan* plan, void* cuda_stream);
 wb_status wb_pack(const wb_plan* plan, size_t round, void* bucket, void* cuda_stream);
 wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bucket, void* cuda_stream);
+
+/* wb_pack_ranks / wb_unpack_ranks: the part of a round that a subset of the virtual ranks executes
+ * (Section 3.2: every trainer worker packs its own shards, every rollout worker assembles its own
+ * parameters; the receive stage moves each sender's buffer to its receiver in between).
+ * wb_pack_ranks runs the packing tiles of the trainer ranks listed in `ranks` (host array, n_ranks
+ * entries, any order, duplicates ignored): it reads only those ranks' tensors and writes only the
+ * (receiver, sender) regions whose sender is listed.  wb_unpack_ranks runs the assembly tiles whose
+ * payload is addressed to a listed rollout rank: it reads only the regions whose receiver is listed and
+ * writes those payloads to every rollout tensor that needs them - the listed ranks' own tensors and,
+ * for a replicated checkpoint region, the other replicas' tensors (on one GPU a plain store; across
+ * GPUs that store is the exchange among replicas).  Packing all trainer ranks in any grouping fills the
+ * same bucket as wb_pack; assembling all rollout ranks in any grouping equals wb_unpack.  The tiles of
+ * consecutive ranks form one launch; a list with gaps takes one launch per run of consecutive ranks.
+ * Same stream, bucket and re-entrancy rules as wb_pack / wb_unpack.
+ * Errors: INVALID_ARG (also: a rank beyond the side's rank count), NOT_BOUND, CUDA. */
+wb_status wb_pack_ranks(const wb_plan* plan, size_t round, const uint32_t* ranks, size_t n_ranks, void* bucket,
+                        void* cuda_stream);
+wb_status wb_unpack_ranks(const wb_plan* plan, size_t round, const uint32_t* ranks, size_t n_ranks,
+                          const void* bucket, void* cuda_stream);
+
+/* Which entries of the wb_plan_tiles listing of a round's WB_TABLE_PACK / WB_TABLE_UNPACK table belong to
+ * virtual rank `rank` (a trainer rank for the pack table, a rollout rank for the unpack table): entries
+ * [*first, *first + *count).  For checking the partition on the host.  Errors: INVALID_ARG. */
+wb_status wb_plan_rank_tiles(const wb_plan* plan, int which, size_t round, uint32_t rank, size_t* first,
+                             size_t* count);
 
 /* wb_plan_check: synchronises with the device and reports whether any launch on this plan
  * recorded an error (the kernels bound every internal wait; a wait that ran out sets a

@@ -72,12 +72,14 @@ TILE_VIEW_DTYPE = np.dtype([
     ("src_tensor", "<i4"), ("dst_tensor", "<i4"), ("src_off", "<u8"), ("dst_off", "<u8"),
     ("nr", "<u4"), ("nc", "<u4"), ("src_sr", "<u4"), ("src_sc", "<u4"), ("dst_sr", "<u4"),
     ("dst_sc", "<u4"), ("kind", "<u4"), ("flags", "<u4"), ("cta", "<u4"), ("reserved", "<u4")])
-assert BUCKET_ENTRY_DTYPE.itemsize == 64 and TILE_VIEW_DTYPE.itemsize == 64
+BUCKET_REGION_DTYPE = np.dtype([("receiver", "<u4"), ("sender", "<u4"), ("off", "<u8"), ("bytes", "<u8")])
+assert BUCKET_ENTRY_DTYPE.itemsize == 64 and TILE_VIEW_DTYPE.itemsize == 64 and BUCKET_REGION_DTYPE.itemsize == 24
 
 EXPORTS = [
     "wb_layout_describe", "wb_layout_free", "wb_layout_add_flat_range", "wb_plan_build", "wb_plan_free", "wb_plan_verify",
     "wb_plan_stats", "wb_plan_rank_bytes", "wb_plan_num_rounds", "wb_plan_bucket_bytes",
-    "wb_plan_bucket_entries", "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
+    "wb_plan_bucket_entries", "wb_plan_bucket_regions", "wb_plan_num_ranks", "wb_pack_ranks", "wb_unpack_ranks", "wb_plan_rank_tiles",
+    "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
     "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_transfer_rounds",
     "wb_plan_num_ckpts", "wb_plan_ckpt_ids", "wb_plan_qbucket_bytes", "wb_absmax", "wb_bucket_quantize",
     "wb_bucket_dequantize", "wb_transfer_rounds_fp8",
@@ -116,6 +118,11 @@ def load() -> C.CDLL:
     lib.wb_plan_bucket_bytes.restype = sz
     lib.wb_plan_bucket_entries.argtypes = [vp, sz, vp, sz, C.POINTER(sz)]
     lib.wb_plan_tiles.argtypes = [vp, C.c_int, sz, vp, sz, C.POINTER(sz)]
+    lib.wb_plan_bucket_regions.argtypes = [vp, sz, vp, sz, C.POINTER(sz)]
+    lib.wb_plan_num_ranks.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+    lib.wb_plan_rank_tiles.argtypes = [vp, C.c_int, sz, C.c_uint32, C.POINTER(sz), C.POINTER(sz)]
+    lib.wb_pack_ranks.argtypes = [vp, sz, vp, sz, vp, vp]
+    lib.wb_unpack_ranks.argtypes = [vp, sz, vp, sz, vp, vp]
     lib.wb_plan_bind.argtypes = [vp, vp, sz, vp, sz]
     lib.wb_remap.argtypes = [vp, vp]
     lib.wb_pack.argtypes = [vp, sz, vp, vp]
@@ -240,6 +247,25 @@ class Plan:
                "wb_plan_bucket_entries")
         return out
 
+    def bucket_regions(self, rnd: int) -> np.ndarray:
+        n = C.c_size_t()
+        _check(_lib.wb_plan_bucket_regions(self.handle, rnd, None, 0, C.byref(n)), "wb_plan_bucket_regions")
+        out = np.zeros(n.value, BUCKET_REGION_DTYPE)
+        _check(_lib.wb_plan_bucket_regions(self.handle, rnd, out.ctypes.data, n.value, C.byref(n)),
+               "wb_plan_bucket_regions")
+        return out
+
+    def num_ranks(self):
+        a, b = C.c_uint32(), C.c_uint32()
+        _check(_lib.wb_plan_num_ranks(self.handle, C.byref(a), C.byref(b)), "wb_plan_num_ranks")
+        return a.value, b.value
+
+    def rank_tiles(self, which: int, rnd: int, rank: int) -> np.ndarray:
+        """The tile views of one virtual rank in a round's pack / unpack table."""
+        a, n = C.c_size_t(), C.c_size_t()
+        _check(_lib.wb_plan_rank_tiles(self.handle, which, rnd, rank, C.byref(a), C.byref(n)), "wb_plan_rank_tiles")
+        return self.tiles(which, rnd)[a.value:a.value + n.value]
+
     def tiles(self, which: int, rnd: int = 0) -> np.ndarray:
         n = C.c_size_t()
         _check(_lib.wb_plan_tiles(self.handle, which, rnd, None, 0, C.byref(n)), "wb_plan_tiles")
@@ -272,6 +298,14 @@ class Plan:
 
     def unpack(self, rnd: int, bucket_ptr: int, stream: int = 0) -> None:
         _check(_lib.wb_unpack(self.handle, rnd, bucket_ptr, stream), "wb_unpack")
+
+    def pack_ranks(self, rnd: int, ranks: Sequence[int], bucket_ptr: int, stream: int = 0) -> None:
+        r = np.ascontiguousarray(ranks, dtype=np.uint32)
+        _check(_lib.wb_pack_ranks(self.handle, rnd, r.ctypes.data, len(r), bucket_ptr, stream), "wb_pack_ranks")
+
+    def unpack_ranks(self, rnd: int, ranks: Sequence[int], bucket_ptr: int, stream: int = 0) -> None:
+        r = np.ascontiguousarray(ranks, dtype=np.uint32)
+        _check(_lib.wb_unpack_ranks(self.handle, rnd, r.ctypes.data, len(r), bucket_ptr, stream), "wb_unpack_ranks")
 
     def transfer_rounds(self, bucket0_ptr: int, bucket1_ptr: int, flags: int = 0, stream: int = 0) -> None:
         _check(_lib.wb_transfer_rounds(self.handle, bucket0_ptr, bucket1_ptr, flags, stream), "wb_transfer_rounds")

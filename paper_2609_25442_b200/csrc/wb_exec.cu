@@ -297,6 +297,52 @@ extern "C" wb_status wb_unpack(const wb_plan* plan, size_t round, const void* bu
                       esize(plan->dst.dtype), esize(plan->dst.dtype), static_cast<cudaStream_t>(cuda_stream));
 }
 
+// The tiles of a set of virtual ranks: maximal runs of consecutive ranks are contiguous tile ranges of
+// the round's table (the planner groups pack tiles by sender and unpack tiles by receiver).
+static wb_status launch_ranks(const wb_plan* plan, const TileTable& T, const std::vector<uint32_t>& rank_begin,
+                              const uint32_t* ranks, size_t n_ranks, uint64_t src_add, uint64_t dst_add, uint32_t es,
+                              uint32_t ed, cudaStream_t stream) {
+  if (!ranks && n_ranks) return WB_ERR_INVALID_ARG;
+  const size_t side_ranks = rank_begin.size() - 1;
+  try {
+    std::vector<uint32_t> sorted(ranks, ranks + n_ranks);
+    for (uint32_t r : sorted) if (r >= side_ranks) return WB_ERR_INVALID_ARG;
+    std::sort(sorted.begin(), sorted.end());
+    sorted.erase(std::unique(sorted.begin(), sorted.end()), sorted.end());
+    for (size_t a = 0; a < sorted.size();) {
+      size_t b = a + 1;
+      while (b < sorted.size() && sorted[b] == sorted[b - 1] + 1) ++b;
+      const uint32_t t0 = rank_begin[sorted[a]], t1 = rank_begin[sorted[b - 1] + 1];
+      if (t1 > t0) {
+        wb_status st = launch_table(plan, T, src_add, dst_add, es, ed, stream, t0, t1 - t0);
+        if (st != WB_OK) return st;
+      }
+      a = b;
+    }
+  } catch (const std::bad_alloc&) {
+    return WB_ERR_OOM;
+  }
+  return WB_OK;
+}
+
+extern "C" wb_status wb_pack_ranks(const wb_plan* plan, size_t round, const uint32_t* ranks, size_t n_ranks,
+                                   void* bucket, void* cuda_stream) {
+  if (!plan || !bucket || round >= plan->rounds.size() || ((uintptr_t)bucket & 15u)) return WB_ERR_INVALID_ARG;
+  if (!plan->bound) return WB_ERR_NOT_BOUND;
+  const Round& R = plan->rounds[round];
+  return launch_ranks(plan, R.pack, R.pack_rank_begin, ranks, n_ranks, 0, (uint64_t)(uintptr_t)bucket,
+                      esize(plan->src.dtype), esize(plan->dst.dtype), static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" wb_status wb_unpack_ranks(const wb_plan* plan, size_t round, const uint32_t* ranks, size_t n_ranks,
+                                     const void* bucket, void* cuda_stream) {
+  if (!plan || !bucket || round >= plan->rounds.size() || ((uintptr_t)bucket & 15u)) return WB_ERR_INVALID_ARG;
+  if (!plan->bound) return WB_ERR_NOT_BOUND;
+  const Round& R = plan->rounds[round];
+  return launch_ranks(plan, R.unpack, R.unpack_rank_begin, ranks, n_ranks, (uint64_t)(uintptr_t)bucket, 0,
+                      esize(plan->dst.dtype), esize(plan->dst.dtype), static_cast<cudaStream_t>(cuda_stream));
+}
+
 // Internal streams and events shared by the multi-stream entry points (created on first use,
 // destroyed with the device tables).
 namespace wbi {

@@ -153,10 +153,18 @@ struct HostGroup {
   std::vector<HostSpan> src, dst;
 };
 
+// One (receiver, sender) region of a round's bucket: the bytes virtual trainer rank `sender` packs for
+// virtual rollout rank `receiver` (what an exchange between GPUs would carry from one to the other).
+struct Region { uint32_t receiver, sender; uint64_t off, bytes; };
+
 struct Round {
-  std::vector<Payload> payloads;
+  std::vector<Payload> payloads;      // ordered by (receiver, sender), then checkpoint order
   uint64_t bucket_bytes = 0;
   TileTable pack, unpack;
+  std::vector<Region> regions;        // in bucket order
+  // pack tiles are grouped by sender rank, unpack tiles by (designated) receiver rank:
+  // rank k's tiles are [x_rank_begin[k], x_rank_begin[k + 1])
+  std::vector<uint32_t> pack_rank_begin, unpack_rank_begin;
 };
 
 }  // namespace wbi

@@ -587,9 +587,14 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
           for (uint32_t c : m) {
             const Slab& sl = P->slabs[chunks[c].slab];
             int64_t pair = (int64_t)sl.receiver * (1ll << 32) + sl.sender;
-            if (pair != last_pair) { off = roundup(off, kRegionAlign); last_pair = pair; }
+            if (pair != last_pair) {
+              off = roundup(off, kRegionAlign);
+              last_pair = pair;
+              R.regions.push_back(Region{sl.receiver, sl.sender, off, 0});
+            }
             R.payloads.push_back(Payload{chunks[c].slab, chunks[c].rect, off});
             off += chunks[c].bytes;
+            R.regions.back().bytes = off - R.regions.back().off;
           }
           R.bucket_bytes = roundup(off, kPayloadAlign);
           if (R.bucket_bytes > budget) fits = false;
@@ -600,16 +605,39 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
       }
       // per-round tile tables
       Ref src; std::vector<Ref> dsts;
+      // Pack tiles are grouped by sender rank and unpack tiles by receiver rank, so that the work of a
+      // set of virtual ranks - what one GPU of a multi-GPU deployment would execute, Section 3.2's
+      // per-worker packing and assembly - is a contiguous tile range of the round's table.
+      std::vector<uint32_t> by_sender;
       for (Round& R : P->rounds) {
         TileBuilder pk{&R.pack, es, ed, P->opts.tile_bytes};
         TileBuilder up{&R.unpack, ed, ed, P->opts.tile_bytes};
-        for (const Payload& pl : R.payloads) {
+        by_sender.resize(R.payloads.size());
+        std::iota(by_sender.begin(), by_sender.end(), 0u);
+        std::stable_sort(by_sender.begin(), by_sender.end(), [&](uint32_t a, uint32_t b) {
+          return P->slabs[R.payloads[a].slab].sender < P->slabs[R.payloads[b].slab].sender;
+        });
+        R.pack_rank_begin.assign(P->egress.size() + 1, 0);
+        R.unpack_rank_begin.assign(P->ingress.size() + 1, 0);
+        uint32_t next_rank = 0;
+        for (uint32_t k : by_sender) {
+          const Payload& pl = R.payloads[k];
           const Slab& sl = P->slabs[pl.slab];
+          while (next_rank <= sl.sender) R.pack_rank_begin[next_rank++] = (uint32_t)R.pack.tiles.size();
           slab_refs(sl, pl.rect, &src, &dsts);
           Ref bucket{-1, pl.bucket_off / ed, pl.rect.nc, 1};
           pk.add(src, std::vector<Ref>{bucket}, pl.rect.nr, pl.rect.nc);
+        }
+        while (next_rank <= P->egress.size()) R.pack_rank_begin[next_rank++] = (uint32_t)R.pack.tiles.size();
+        next_rank = 0;
+        for (const Payload& pl : R.payloads) {
+          const Slab& sl = P->slabs[pl.slab];
+          while (next_rank <= sl.receiver) R.unpack_rank_begin[next_rank++] = (uint32_t)R.unpack.tiles.size();
+          slab_refs(sl, pl.rect, &src, &dsts);
+          Ref bucket{-1, pl.bucket_off / ed, pl.rect.nc, 1};
           up.add(bucket, dsts, pl.rect.nr, pl.rect.nc);
         }
+        while (next_rank <= P->ingress.size()) R.unpack_rank_begin[next_rank++] = (uint32_t)R.unpack.tiles.size();
         if (!pk.ok || !up.ok) return fail(WB_ERR_INVALID_ARG);
         assign_ctas(&R.pack, P->grid);
         assign_ctas(&R.unpack, P->grid);
@@ -691,6 +719,26 @@ extern "C" wb_status wb_plan_bucket_entries(const wb_plan* plan, size_t round, w
   return WB_OK;
 }
 
+extern "C" wb_status wb_plan_bucket_regions(const wb_plan* plan, size_t round, wb_bucket_region* out, size_t cap,
+                                            size_t* n) {
+  if (!plan || !n || round >= plan->rounds.size()) return WB_ERR_INVALID_ARG;
+  const Round& R = plan->rounds[round];
+  *n = R.regions.size();
+  if (!out) return WB_OK;
+  for (size_t k = 0; k < R.regions.size() && k < cap; ++k) {
+    const Region& g = R.regions[k];
+    out[k] = wb_bucket_region{g.receiver, g.sender, g.off, g.bytes};
+  }
+  return WB_OK;
+}
+
+extern "C" wb_status wb_plan_num_ranks(const wb_plan* plan, uint32_t* n_trainer, uint32_t* n_rollout) {
+  if (!plan || !n_trainer || !n_rollout) return WB_ERR_INVALID_ARG;
+  *n_trainer = (uint32_t)plan->egress.size();
+  *n_rollout = (uint32_t)plan->ingress.size();
+  return WB_OK;
+}
+
 static const TileTable* pick_table(const wb_plan* plan, int which, size_t round) {
   if (which == WB_TABLE_REMAP) return &plan->remap;
   if (round >= plan->rounds.size()) return nullptr;
@@ -723,6 +771,22 @@ extern "C" wb_status wb_plan_tiles(const wb_plan* plan, int which, size_t round,
     }
   }
   *n = count;
+  return WB_OK;
+}
+
+extern "C" wb_status wb_plan_rank_tiles(const wb_plan* plan, int which, size_t round, uint32_t rank, size_t* first,
+                                        size_t* count) {
+  if (!plan || !first || !count || round >= plan->rounds.size()) return WB_ERR_INVALID_ARG;
+  if (which != WB_TABLE_PACK && which != WB_TABLE_UNPACK) return WB_ERR_INVALID_ARG;
+  const Round& R = plan->rounds[round];
+  const TileTable& T = which == WB_TABLE_PACK ? R.pack : R.unpack;
+  const std::vector<uint32_t>& rb = which == WB_TABLE_PACK ? R.pack_rank_begin : R.unpack_rank_begin;
+  if ((size_t)rank + 1 >= rb.size()) return WB_ERR_INVALID_ARG;
+  // the listing has one entry per destination of a tile
+  size_t a = 0, n = 0;
+  for (uint32_t k = 0; k < rb[rank + 1]; ++k) (k < rb[rank] ? a : n) += 1 + T.tiles[k].n_extra;
+  *first = a;
+  *count = n;
   return WB_OK;
 }
 
@@ -813,6 +877,44 @@ extern "C" wb_status wb_plan_verify(const wb_plan* plan) {
       if (R.bucket_bytes > plan->opts.bucket_budget_bytes) return WB_ERR_INTERNAL;
       if (!check_table(R.pack, false, true, R.bucket_bytes / ed, elems, elems)) return WB_ERR_INTERNAL;
       if (!check_table(R.unpack, true, false, R.bucket_bytes / ed, elems, elems_w)) return WB_ERR_INTERNAL;
+      // (4) rank partition: regions tile the bucket in order; a sender rank's pack tiles read only that
+      // rank's tensors and write only its regions; a receiver rank's unpack tiles read only its regions
+      {
+        uint64_t end = 0;
+        for (const Region& g : R.regions) {
+          if (g.off % kRegionAlign || g.off < end || g.off + g.bytes > R.bucket_bytes) return WB_ERR_INTERNAL;
+          end = g.off + g.bytes;
+        }
+        auto region_of = [&](uint64_t byte_lo, uint64_t byte_hi) -> const Region* {
+          for (const Region& g : R.regions)
+            if (byte_lo >= g.off && byte_hi <= g.off + g.bytes) return &g;
+          return nullptr;
+        };
+        auto span = [&](uint64_t off, const HTile& t, uint32_t sr, uint32_t sc, uint64_t* lo, uint64_t* hi) {
+          *lo = off * ed;
+          *hi = (off + (uint64_t)(t.nr - 1) * sr + (uint64_t)(t.nc - 1) * sc + 1) * ed;
+        };
+        if (R.pack_rank_begin.size() != plan->egress.size() + 1 || R.pack_rank_begin.back() != R.pack.tiles.size())
+          return WB_ERR_INTERNAL;
+        if (R.unpack_rank_begin.size() != plan->ingress.size() + 1 || R.unpack_rank_begin.back() != R.unpack.tiles.size())
+          return WB_ERR_INTERNAL;
+        for (size_t rank = 0; rank + 1 < R.pack_rank_begin.size(); ++rank)
+          for (uint32_t k = R.pack_rank_begin[rank]; k < R.pack_rank_begin[rank + 1]; ++k) {
+            const HTile& t = R.pack.tiles[k];
+            uint64_t lo, hi;
+            span(t.dst_off, t, t.dsr, t.dsc, &lo, &hi);
+            const Region* g = region_of(lo, hi);
+            if (S.tensors[t.src_tensor].rank != rank || !g || g->sender != rank) return WB_ERR_INTERNAL;
+          }
+        for (size_t rank = 0; rank + 1 < R.unpack_rank_begin.size(); ++rank)
+          for (uint32_t k = R.unpack_rank_begin[rank]; k < R.unpack_rank_begin[rank + 1]; ++k) {
+            const HTile& t = R.unpack.tiles[k];
+            uint64_t lo, hi;
+            span(t.src_off, t, t.ssr, t.ssc, &lo, &hi);
+            const Region* g = region_of(lo, hi);
+            if (!g || g->receiver != rank) return WB_ERR_INTERNAL;
+          }
+      }
       rd += elems; wr += elems_w;
     }
     if (rd != plan->stats.src_elems_read || wr != plan->stats.dst_elems_written) return WB_ERR_INTERNAL;

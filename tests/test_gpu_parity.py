@@ -470,3 +470,54 @@ def test_remap_in_a_cuda_graph(device):
         torch.cuda.synchronize()
         assert_dst_equals(case, want)
     case.plan.check()
+
+
+@pytest.mark.parametrize("name,scale,budget", [
+    ("cfg1b", "full", 1 << 20), ("cfg3", "small", 1 << 20), ("cfg4", "small", 1 << 19), ("cfg5", "small", 1 << 18),
+    ("cfg3", "medium", 32 << 20), ("cfg5", "medium", 16 << 20)])
+def test_rank_subsets_compose_to_the_whole_round(device, name, scale, budget):
+    """wb_pack_ranks / wb_unpack_ranks (Section 3.2: every worker packs its own shards and assembles its
+    own parameters): a trainer rank's call writes exactly its (receiver, sender) regions of the bucket,
+    the calls of all ranks together fill the bucket wb_pack fills, and assembling the rollout ranks one
+    group at a time gives the oracle's tensors."""
+    wl = make_workload(name, scale)
+    case = DeviceCase(wl, device, bucket_budget_bytes=budget)
+    want = oracle_for(case)
+    plan = case.plan
+    nt, nr = plan.num_ranks()
+    rng = np.random.default_rng(5)
+    for r in range(plan.num_rounds()):
+        nb = plan.bucket_bytes(r)
+        whole = torch.full((nb + 64,), 0x5A, dtype=torch.uint8, device=device)
+        plan.pack(r, whole.data_ptr())
+        regions = plan.bucket_regions(r)
+        parts = torch.full((nb + 64,), 0x5A, dtype=torch.uint8, device=device)
+        # one rank alone: only its regions change
+        for v in range(nt):
+            alone = torch.full((nb + 64,), 0x5A, dtype=torch.uint8, device=device)
+            plan.pack_ranks(r, [v], alone.data_ptr())
+            torch.cuda.synchronize()
+            mine = torch.zeros(nb + 64, dtype=torch.bool, device=device)
+            for g in regions:
+                if int(g["sender"]) == v:
+                    mine[int(g["off"]):int(g["off"]) + int(g["bytes"])] = True
+            assert torch.equal(alone[mine], whole[mine]) and bool((alone[~mine] == 0x5A).all()), (r, v)
+        # a random grouping of the ranks (lists with gaps and duplicates) fills the whole bucket
+        order = rng.permutation(nt)
+        cut = int(rng.integers(0, nt + 1))
+        for group in (order[:cut], order[cut:]):
+            plan.pack_ranks(r, [int(x) for x in group] + [int(x) for x in group[:1]], parts.data_ptr())
+        torch.cuda.synchronize()
+        assert torch.equal(parts, whole), r
+        order = rng.permutation(nr)
+        cut = int(rng.integers(0, nr + 1))
+        for group in (order[:cut], order[cut:]):
+            plan.unpack_ranks(r, [int(x) for x in group], parts.data_ptr())
+    torch.cuda.synchronize()
+    assert_dst_equals(case, want)
+    plan.check()
+    with pytest.raises(wb.WbError):
+        plan.pack_ranks(0, [nt], whole.data_ptr())
+    with pytest.raises(wb.WbError):
+        plan.unpack_ranks(0, [nr], whole.data_ptr())
+    plan.pack_ranks(0, [], whole.data_ptr())          # an empty set launches nothing
