@@ -173,3 +173,86 @@ def test_batched_diff2_entry_point_checks_its_arguments_on_the_host():
     empty["rows"] = 0
     wb.wb_diff2_nonzeros_batch(empty, 4096, 1024, 4096, 1, 4096)   # only empty fields: nothing is launched
     wb.wb_diff2_nonzeros_batch(fields[:0], 0, 0, 4096, 1, 4096)    # no fields at all
+
+
+# ---- Algorithm 1's chunk passes with carries (the oracle's reading, pinned to diff2 of the full ids) -------
+from oracle.extract import carry_stride, chunk_passes, emit_carry, expand_carry, strided_diff1
+
+
+def _balanced_digits(v: int, b: int, n: int):
+    """Digits d_k in [-2^(b-1), 2^(b-1)) with v = sum d_k 2^(bk), in Python integers."""
+    out = []
+    for _ in range(n):
+        d = ((v + (1 << (b - 1))) % (1 << b)) - (1 << (b - 1))
+        out.append(d)
+        v = (v - d) >> b
+    assert v == 0
+    return out
+
+
+def test_strided_diff1_is_lossless_and_is_diff1_at_stride_one():
+    rng = np.random.default_rng(4)
+    for shape in [(1, 1000), (37, 53), (300, 7), (5, 700)]:
+        c = rng.integers(-17, 18, size=shape)
+        assert np.array_equal(strided_diff1(c, 1)[:, 1:], diff1(c)[:, 1:])      # away from the left edge, where the
+        for s in (1, 2, 3, 16, 256, 65536):                                     # flat order wraps into the row above
+            g = strided_diff1(c, s)
+            assert np.array_equal(expand_carry(g, s), c)
+        # written out for one element: left neighbour s back in flat order, upper neighbour s rows up
+        if shape == (37, 53):
+            g, s, f = strided_diff1(c, 3), 3, c.reshape(-1)
+            x = 20 * 53 + 1
+            assert g.reshape(-1)[x] == f[x] - f[x - s] - f[x - s * 53] + f[x - s - s * 53]
+            assert g.reshape(-1)[2] == f[2] and g.reshape(-1)[5] == f[5] - f[2]
+
+
+def test_emit_carry_splits_into_a_balanced_digit_and_a_carry():
+    d = np.array([[0, 1, -1, 127, 128, -128, -129, 255, 256, -256, 4096 * 3 + 5, -(1 << 40) - 3]], np.int64)
+    z, c = emit_carry(d, 8)
+    assert np.array_equal(z + (c << 8), d) and z.min() >= -128 and z.max() <= 127
+    assert z.tolist()[0][:10] == [0, 1, -1, 127, -128, -128, 127, -1, 0, 0]
+    assert c.tolist()[0][:10] == [0, 0, 0, 0, 1, 0, -1, 1, 1, -1]
+
+
+@pytest.mark.parametrize("b", [8, 16])
+@pytest.mark.parametrize("name,side,pick", [("cfg3", "trainer", 5), ("cfg5", "rollout", None), ("cfg1b", "trainer", None)])
+def test_chunk_passes_give_the_balanced_digits_of_the_full_diff(name, side, pick, b):
+    """Algorithm 1 with carries: Recombine(H_Z) = diff2(full ids), the field comes back by two prefix sums,
+    every Z_k holds exactly the k-th balanced digit of diff2(ids) - so it is as sparse as diff2(ids) - and
+    the carry out of the last pass is zero."""
+    wl = make_workload(name, "small" if name != "cfg1b" else "full")
+    fields = id_fields(wl, side)
+    fields = [fields[pick]] if pick is not None else sorted(fields, key=lambda f: -f.size)[:6]
+    bits = (16 * (wl.ckpt_numel() + 1)).bit_length() + 1
+    K = -(-bits // b)
+    for f in fields:
+        h_z, h_g, last = chunk_passes(f, b, K)
+        full = diff2(f)
+        assert np.array_equal(recombine(h_z, b), full)
+        assert np.array_equal(undo_diff2(recombine(h_z, b)), f)
+        assert not last.any()
+        for (i, j) in zip(*np.nonzero(full)):
+            assert [int(z[i, j]) for z in h_z] == _balanced_digits(int(full[i, j]), b, K)
+        assert all(not z[full == 0].any() for z in h_z)
+        # the library's Recombine takes the same lists
+        got = wb.wb_diff2_recombine([entries(z) for z in h_z], b)
+        assert np.array_equal(got, entries(full))
+
+
+def test_entries_shipped_per_pass_stay_bounded_where_plain_chunk_diffs_do_not():
+    """A field of 2^24 ids as one flat shard and as a 4096 x 4096 tensor filled by two slice copies: every
+    pass ships a handful of entries (digits + strided carry differences), while diff2 of a bare 8-bit
+    chunk carries one cluster of wrap artifacts per 256 consecutive ids."""
+    n = 1 << 24
+    flat = (np.arange(n, dtype=np.int64) + 1 + (1 << 33) + 12345).reshape(1, n)
+    two = flat.reshape(4096, 4096).copy()
+    two[2048:, :] += 7 * 4096 * 4096 + 999 * 4096                  # a second checkpoint tensor further on
+    for field, n_ops in ((flat, 1), (two, 2)):
+        K = -(-((16 * int(field.max())).bit_length() + 1) // 8)
+        h_z, h_g, last = chunk_passes(field, 8, K)
+        assert np.array_equal(recombine(h_z, 8), diff2(field)) and not last.any()
+        for k in range(K):
+            shipped = np.count_nonzero(h_z[k]) + np.count_nonzero(h_g[k])
+            assert shipped <= 32 * n_ops, (k, shipped)
+        if field.shape[0] == 1:                   # (rows 4096 ids apart repeat their wrap pattern: those cancel vertically)
+            assert np.count_nonzero(diff2(id_chunk(field, 0, 8))) >= n // 256
