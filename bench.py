@@ -49,11 +49,13 @@ def parse_args():
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--grid-ctas", type=int, default=0)
     ap.add_argument("--path", default="remap",
-                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "rounds_fp8", "rounds_fp8_pipelined", "extract"],
+                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "rounds_fp8", "rounds_fp8_pipelined", "extract",
+                             "extract_chunks"],
                     help="remap: fused launch; pack_unpack: wb_pack + wb_unpack per round on one stream; "
                          "rounds: wb_transfer_rounds (depth-2 buckets, two streams); rounds_serial: its "
                          "unpipelined baseline; rounds_fp8: amax pass, then per round pack, quantise the bucket to FP8, "
-                         "dequantise, unpack; extract: source-map extraction kernel")
+                         "dequantise, unpack; extract: source-map extraction kernel; extract_chunks: Algorithm 1's 8-bit chunk "
+                         "passes with carries (entries shipped per pass with and without them)")
     ap.add_argument("--cuda-graph", action="store_true",
                     help="remap path: replay the launch from a captured CUDA graph (for the launch-bound tiny model)")
     ap.add_argument("--budget-mib", type=int, default=0, help="bucket budget per round (0: the 4 GiB default)")
@@ -292,6 +294,92 @@ def run_extract(args):
                       "gpu_launches": args.steps * len(fields)}))
 
 
+def run_extract_chunks(args):
+    """--path extract_chunks: Algorithm 1's inner loop on the trainer's id fields held as 8-bit chunks in bf16
+    tensors (first loader groups, up to ~2^28 elements): per pass, the entries that cross to the host with the
+    carry construction (digits + strided carry differences) and without it (plain diff2 of the chunk), and
+    the device time of the pass."""
+    from paper_2609_25442_b200 import binding as wb
+    from paper_2609_25442_b200.device import require_cuda
+    require_cuda()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    wl = make_workload(args.workload, args.scale)
+    fields, total = [], 0
+    for ckpt_idx, fn in wl.trainer_groups():
+        for _, t in fn([wl.ckpt_ids(i, dev) + 1 for i in ckpt_idx]).items():
+            t = (t.reshape(1, -1) if t.dim() == 1 else t.reshape(-1, t.shape[-1])).clamp_min(0).contiguous()
+            fields.append(t)
+            total += t.numel()
+        if total >= (1 << 28):
+            break
+    b = 8
+    K = -(-((16 * (wl.ckpt_numel() + 1)).bit_length() + 1) // b)
+    cap = 1 << 22
+    zo = torch.zeros(cap * 24, dtype=torch.uint8, device=dev)
+    go = torch.zeros(cap * 24, dtype=torch.uint8, device=dev)
+    counts = torch.zeros(2, dtype=torch.int64, device=dev)
+    nb = max(wb.wb_diff2_chunk_scratch_bytes(f.shape[0], f.shape[1]) for f in fields)
+    scratch = torch.empty(nb, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    carries = [None] * len(fields)
+    passes = []
+    for _ in range(3):                                   # untimed: module load, first-launch costs
+        f = fields[-1]
+        counts.zero_()
+        wb.wb_diff2_chunk_pass((f & 255).to(torch.bfloat16).data_ptr(), wb.WB_ID_BF16, f.shape[0], f.shape[1], b, 0, 0, 0,
+                               scratch.data_ptr(), nb, zo.data_ptr(), cap, counts.data_ptr(), go.data_ptr(), cap,
+                               counts.data_ptr() + 8, stream)
+        torch.cuda.synchronize()
+    for k in range(K):
+        row = {"pass": k, "digits": 0, "carry_records": 0, "plain": 0, "ms": 0.0, "plain_ms": 0.0}
+        for n, f in enumerate(fields):
+            chunk = ((f >> (b * k)) & ((1 << b) - 1)).to(torch.bfloat16)       # what load_weights leaves in a bf16 tensor
+            cin = carries[n]
+            counts.zero_()
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            wb.wb_diff2_chunk_pass(chunk.data_ptr(), wb.WB_ID_BF16, f.shape[0], f.shape[1], b, k,
+                                   cin.data_ptr() if cin is not None else 0, 0 if cin is None else cin.numel() // 24,
+                                   scratch.data_ptr(), nb, zo.data_ptr(), cap, counts.data_ptr(), go.data_ptr(), cap,
+                                   counts.data_ptr() + 8, stream)
+            e.record()
+            torch.cuda.synchronize()
+            row["ms"] += a.elapsed_time(e)
+            nz, ng = (int(x) for x in counts.cpu())
+            assert nz <= cap and ng <= cap
+            row["digits"] += nz
+            row["carry_records"] += ng
+            # the records go to the host and come back for the next pass
+            host = go[:ng * 24].cpu()
+            carries[n] = host.to(dev) if ng else None
+            counts.zero_()
+            a.record()
+            wb.wb_diff2_nonzeros(chunk.data_ptr(), wb.WB_ID_BF16, f.shape[0], f.shape[1], zo.data_ptr(), cap,
+                                 counts.data_ptr(), stream)
+            e.record()
+            torch.cuda.synchronize()
+            row["plain_ms"] += a.elapsed_time(e)
+            row["plain"] += int(counts[0].item())
+        row["gbs_field_bytes"] = total * 2 / (row["ms"] * 1e-3) / 1e9
+        passes.append(row)
+    peak, peak_src = hbm_peak()
+    ms = sum(r["ms"] for r in passes) / K
+    gbs = total * 2 / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "chunk pass with carries, GB/s of id-chunk field read (bf16 elements)", "value": gbs,
+                      "unit": "GB/s", "n_gpus": 1, "steps": K, "warmup": 0, "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "bf16 chunks -> int", "data": "synthetic",
+                      "config": {"workload": wl.name, "path": "extract_chunks", "fields": len(fields), "elements": total,
+                                 "chunk_bits": b, "passes": passes, "l2": "inputs_larger_than_l2",
+                                 "entries_shipped_with_carries": sum(r["digits"] + r["carry_records"] for r in passes),
+                                 "entries_shipped_plain": sum(r["plain"] for r in passes)},
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                   "traffic": None, "peak_source": peak_src, "kernel": "wb_chunk_pass_kernel",
+                                   "note": "algorithmic bytes = the 2-byte field; the one-byte carry field is read and "
+                                           "written by the pass and read again by the strided difference"},
+                      "gpu_launches": K * len(fields) * 2}))
+
+
 def hbm_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -361,6 +449,9 @@ def main():
         return
     if args.path == "extract":
         run_extract(args)
+        return
+    if args.path == "extract_chunks":
+        run_extract_chunks(args)
         return
 
     from paper_2609_25442_b200 import binding as wb

@@ -499,6 +499,32 @@ typedef struct wb_diff2_tagged_entry {
 size_t wb_diff2_batch_scratch_bytes(size_t n_fields);
 wb_status wb_diff2_nonzeros_batch(const wb_diff2_field* fields, size_t n_fields, void* scratch, size_t scratch_bytes,
                                   wb_diff2_tagged_entry* out, uint64_t cap, uint64_t* count, void* cuda_stream);
+/* wb_diff2_chunk_pass (device, asynchronous on cuda_stream): one pass of Algorithm 1's inner loop for one
+ * local tensor, with carries, so that O(N_c) entries per pass reach the host even for 8-bit chunks
+ * (Appendix B: diff2 of a truncated chunk overflows at regularly spaced positions; the overflow is carried
+ * into the next chunk, and a strided difference cancels the periodic pattern).  The paper sketches the
+ * step only; what this computes:
+ *   D = diff2(field) + Gamma          field = chunk `pass` of the ids as load_weights left it (values in
+ *                                     [0, 2^chunk_bits)), Gamma = ExpandCarry(carry_in), 0 for pass 0
+ *   D = Z + 2^chunk_bits C            EmitCarry: Z the balanced digit in [-2^(b-1), 2^(b-1)), C the carry
+ *   z_out    <- NonZeros(Z)           H_Z[pass]: the pass-th balanced digit of every entry of diff2(ids)
+ *   carry_out <- NonZeros(StridedDiff1(C))   H_Gamma[pass], with s = 2^(chunk_bits (pass + 1)), x = i cols + j:
+ *                                     G[x] = C[x] - C[x - s] - C[x - s cols] + C[x - s - s cols]
+ *   ExpandCarry inverts StridedDiff1 of the previous pass (s = 2^(chunk_bits pass)).
+ * Feeding the z_out lists of passes 0 .. K-1 to wb_diff2_recombine gives diff2 of the full ids when
+ * K chunk_bits >= bits(16 max id) + 1 (then the last carry_out list is empty).
+ * field: DEVICE, rows x cols, read as id_kind.  carry_in: DEVICE list of the previous pass's carry_out
+ * entries for this tensor (n_carry_in of them; NULL / 0 for pass 0 or an empty list).  scratch: DEVICE,
+ * 16-byte aligned, wb_diff2_chunk_scratch_bytes(rows, cols) bytes (one byte per element plus 256 KiB),
+ * contents irrelevant before and after.  z_out / carry_out (DEVICE, z_cap / carry_cap entries, no
+ * particular order) and *z_count / *carry_count (DEVICE uint64, zeroed by the caller) as for
+ * wb_diff2_nonzeros.  Several kernels per call.  Limits: chunk_bits 8 or 16, pass < 8, rows * cols <= 2^40.
+ * Errors: INVALID_ARG, CUDA. */
+size_t wb_diff2_chunk_scratch_bytes(uint64_t rows, uint64_t cols);
+wb_status wb_diff2_chunk_pass(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols, uint32_t chunk_bits,
+                              uint32_t pass, const wb_diff2_entry* carry_in, uint64_t n_carry_in, void* scratch,
+                              size_t scratch_bytes, wb_diff2_entry* z_out, uint64_t z_cap, uint64_t* z_count,
+                              wb_diff2_entry* carry_out, uint64_t carry_cap, uint64_t* carry_count, void* cuda_stream);
 /* wb_diff2_recombine (host): Algorithm 1, Recombine.  sum_k 2^(chunk_bits*k) * passes[k], merged
  * by position, zeros dropped, sorted by (row, col).  Writes up to cap entries, *n_out = total. */
 wb_status wb_diff2_recombine(const wb_diff2_entry* const* passes, const size_t* counts, size_t n_passes,

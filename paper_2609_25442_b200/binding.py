@@ -83,7 +83,7 @@ EXPORTS = [
     "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_transfer_rounds",
     "wb_plan_num_ckpts", "wb_plan_ckpt_ids", "wb_plan_qbucket_bytes", "wb_absmax", "wb_bucket_quantize",
     "wb_bucket_dequantize", "wb_transfer_rounds_fp8",
-    "wb_diff2_nonzeros", "wb_diff2_nonzeros_batch", "wb_diff2_batch_scratch_bytes", "wb_diff2_recombine", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
+    "wb_diff2_nonzeros", "wb_diff2_nonzeros_batch", "wb_diff2_batch_scratch_bytes", "wb_diff2_recombine", "wb_diff2_chunk_pass", "wb_diff2_chunk_scratch_bytes", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -412,6 +412,27 @@ def wb_diff2_nonzeros_batch(fields: np.ndarray, scratch_ptr: int, scratch_bytes:
                                              C.c_void_p, C.c_void_p]
     _check(_lib.wb_diff2_nonzeros_batch(fields.ctypes.data, len(fields), scratch_ptr, scratch_bytes, out_ptr, cap,
                                         count_ptr, stream), "wb_diff2_nonzeros_batch")
+
+
+def wb_diff2_chunk_scratch_bytes(rows: int, cols: int) -> int:
+    lib = load()
+    lib.wb_diff2_chunk_scratch_bytes.restype = C.c_size_t
+    lib.wb_diff2_chunk_scratch_bytes.argtypes = [C.c_uint64, C.c_uint64]
+    return int(lib.wb_diff2_chunk_scratch_bytes(rows, cols))
+
+
+def wb_diff2_chunk_pass(field_ptr: int, id_kind: int, rows: int, cols: int, chunk_bits: int, pass_index: int,
+                        carry_in_ptr: int, n_carry_in: int, scratch_ptr: int, scratch_bytes: int, z_out_ptr: int,
+                        z_cap: int, z_count_ptr: int, carry_out_ptr: int, carry_cap: int, carry_count_ptr: int,
+                        stream: int = 0) -> None:
+    """One chunk pass of Algorithm 1 with carries for one device tensor (all pointers are device)."""
+    lib = load()
+    lib.wb_diff2_chunk_pass.argtypes = [C.c_void_p, C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint32,
+                                        C.c_void_p, C.c_uint64, C.c_void_p, C.c_size_t, C.c_void_p, C.c_uint64,
+                                        C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p]
+    _check(lib.wb_diff2_chunk_pass(field_ptr, id_kind, rows, cols, chunk_bits, pass_index, carry_in_ptr, n_carry_in,
+                                   scratch_ptr, scratch_bytes, z_out_ptr, z_cap, z_count_ptr, carry_out_ptr, carry_cap,
+                                   carry_count_ptr, stream), "wb_diff2_chunk_pass")
 
 
 def wb_diff2_recombine(passes: Sequence[np.ndarray], chunk_bits: int) -> np.ndarray:

@@ -439,3 +439,417 @@ extern "C" wb_status wb_diff2_nonzeros_batch(const wb_diff2_field* fields, size_
                                                   cap, cnt);
   return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
 }
+
+// =================================================================================================
+// Chunk passes with carries (Algorithm 1, inner loop; Appendix B, "Difference encoding", last two
+// paragraphs).  The paper sketches this step only; the construction built here:
+//
+//   ids = sum_k 2^(bk) A_k, so diff2(ids) = sum_k 2^(bk) diff2(A_k) is evaluated like a multi-digit
+//   addition, least significant chunk first.  Pass k forms D = diff2(A_k) + Gamma, Gamma the carry out
+//   of pass k-1, and splits it (EmitCarry) into the balanced b-bit digit Z in [-2^(b-1), 2^(b-1)) and
+//   the carry C = (D - Z) / 2^b.  Z is zero wherever diff2(ids) is, so NonZeros(Z) has O(N_c) entries.
+//   C is non-zero wherever chunk k wraps, every s = 2^(b(k+1)) consecutive ids of a run; it goes to
+//   the host as NonZeros(StridedDiff1(C)),
+//       G[x] = C[x] - C[x - s] - C[x - s cols] + C[x - s - s cols]     (x = i cols + j, C = 0 before the tensor),
+//   Eq. diff1 with the left neighbour s elements back in flat order and the upper neighbour s rows up,
+//   which cancels the periodic pattern.  ExpandCarry inverts it on the device before the next pass:
+//   the records are scattered into a zeroed one-byte-per-element field, then summed over every s-th
+//   element of the flat order and over every s-th row.
+//
+// The carry field of the tensor lives in caller-provided scratch (one byte per element: |C| <= 17),
+// is overwritten in place by the pass (D at x needs Gamma at x only) and differenced by a last kernel.
+// =================================================================================================
+namespace {
+
+constexpr unsigned kCarryBlocks = 148 * 8;
+constexpr unsigned long long kCarryAuxEntries = 1ull << 16;        // partial column sums of the strided prefix
+
+__global__ void wb_carry_scatter_kernel(const wb_diff2_entry* __restrict__ rec, unsigned long long n_rec,
+                                        unsigned long long rows, unsigned long long cols, signed char* __restrict__ y) {
+  for (unsigned long long k = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; k < n_rec;
+       k += (unsigned long long)gridDim.x * blockDim.x) {
+    const wb_diff2_entry e = rec[k];
+    if (e.row < rows && e.col < cols) y[e.row * cols + e.col] = (signed char)e.value;
+  }
+}
+
+// y[x] += y[x - t] for all x, as the column-wise running sum of the [H, t] row-major view of y.  The H
+// rows are cut into nblk blocks of hb rows; a thread owns four adjacent columns (one 32-bit word) of
+// one block.  phase 0: block sums -> part; phase 1 (one block of rows only needs phase 2): exclusive
+// scan of part over the blocks; phase 2: running sums written back, starting from the scanned offset.
+// t is a multiple of 4 and y is padded to a multiple of 4 bytes.
+__device__ __forceinline__ void add4(int (&acc)[4], unsigned w) {
+  acc[0] += (signed char)(w & 0xFF); acc[1] += (signed char)((w >> 8) & 0xFF);
+  acc[2] += (signed char)((w >> 16) & 0xFF); acc[3] += (signed char)(w >> 24);
+}
+__global__ void wb_strided_prefix_kernel(signed char* __restrict__ y, unsigned long long n4, unsigned long long t,
+                                         unsigned long long H, unsigned long long hb, unsigned long long nblk,
+                                         int* __restrict__ part, int phase) {
+  const unsigned long long tw = t / 4;                         // words per row of the view
+  const unsigned long long total = phase == 1 ? tw : nblk * tw;
+  for (unsigned long long id = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; id < total;
+       id += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long blk = phase == 1 ? 0 : id / tw, w = id - blk * tw;
+    if (phase == 1) {
+      int run[4] = {0, 0, 0, 0};
+      for (unsigned long long b = 0; b < nblk; ++b) {
+        int4* p = reinterpret_cast<int4*>(part) + b * tw + w;
+        const int4 v = *p;
+        *p = make_int4(run[0], run[1], run[2], run[3]);
+        run[0] += v.x; run[1] += v.y; run[2] += v.z; run[3] += v.w;
+      }
+      continue;
+    }
+    int acc[4] = {0, 0, 0, 0};
+    if (phase == 2 && nblk > 1) {
+      const int4 v = reinterpret_cast<const int4*>(part)[blk * tw + w];
+      acc[0] = v.x; acc[1] = v.y; acc[2] = v.z; acc[3] = v.w;
+    }
+    const unsigned long long h0 = blk * hb, h1 = h0 + hb < H ? h0 + hb : H;
+    for (unsigned long long h = h0; h < h1; ++h) {
+      const unsigned long long x = h * t + 4 * w;
+      if (x >= n4) break;
+      unsigned* p = reinterpret_cast<unsigned*>(y + x);
+      add4(acc, *p);
+      if (phase == 2)
+        *p = (unsigned)(acc[0] & 0xFF) | ((unsigned)(acc[1] & 0xFF) << 8) | ((unsigned)(acc[2] & 0xFF) << 16) |
+             ((unsigned)(acc[3] & 0xFF) << 24);
+    }
+    if (phase == 0) reinterpret_cast<int4*>(part)[blk * tw + w] = make_int4(acc[0], acc[1], acc[2], acc[3]);
+  }
+}
+
+// Gamma at one element from the sorted carry records (see wb_carry_sort_kernel): ExpandCarry in closed
+// form.  C = prefix over every s-th element of the flat order, then over every s-th row, of G, so a record
+// (x_r, g) reaches x when x - x_r = m s with m >= 0, once for every split m = a + c cols (a, c >= 0) if the
+// row stride applies, i.e. floor(m / cols) + 1 times, else once.
+struct CarryRec { unsigned long long x; long long g; };
+struct CarryIndex {
+  const unsigned* first;          // 257 offsets into rec, by x mod 256
+  const unsigned char* has;       // 32 bytes: bit r set if some record has x mod 256 == r
+  const CarryRec* rec;
+  unsigned long long s, cols;
+  unsigned s_shift;
+  int use_up;
+};
+__device__ __forceinline__ int gamma_at(const CarryIndex& ci, unsigned long long x) {
+  const unsigned r = (unsigned)x & 255u;
+  int acc = 0;
+  for (unsigned k = __ldg(ci.first + r), e = __ldg(ci.first + r + 1); k < e; ++k) {
+    const unsigned long long xr = __ldg(&ci.rec[k].x);
+    if (x < xr || ((x - xr) & (ci.s - 1)) != 0) continue;
+    const unsigned long long m = (x - xr) >> ci.s_shift;
+    const long long mult = ci.use_up ? (long long)(m / ci.cols) + 1 : 1;
+    acc += (int)(__ldg(&ci.rec[k].g) * mult);
+  }
+  return acc;
+}
+
+// Sort the carry records by x mod 256 (one block): counts, offsets, placement.
+__global__ void __launch_bounds__(256)
+wb_carry_sort_kernel(const wb_diff2_entry* __restrict__ rec, unsigned n_rec, unsigned long long cols,
+                     unsigned* __restrict__ first, unsigned char* __restrict__ has, CarryRec* __restrict__ sorted) {
+  __shared__ unsigned bin[257], cur[256];
+  bin[threadIdx.x] = 0;
+  if (threadIdx.x == 0) bin[256] = 0;
+  __syncthreads();
+  for (unsigned k = threadIdx.x; k < n_rec; k += 256) atomicAdd(&bin[(unsigned)(rec[k].row * cols + rec[k].col) & 255u], 1u);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned run = 0;
+    for (int r = 0; r < 256; ++r) { const unsigned c = bin[r]; bin[r] = run; run += c; }
+    bin[256] = run;
+  }
+  __syncthreads();
+  cur[threadIdx.x] = bin[threadIdx.x];
+  first[threadIdx.x] = bin[threadIdx.x];
+  if (threadIdx.x == 0) first[256] = bin[256];
+  if (threadIdx.x < 32) {
+    unsigned char m = 0;
+    for (int q = 0; q < 8; ++q) m |= (unsigned char)((bin[threadIdx.x * 8 + q + 1] > bin[threadIdx.x * 8 + q]) << q);
+    has[threadIdx.x] = m;
+  }
+  __syncthreads();
+  for (unsigned k = threadIdx.x; k < n_rec; k += 256) {
+    const unsigned long long x = rec[k].row * cols + rec[k].col;
+    sorted[atomicAdd(&cur[(unsigned)x & 255u], 1u)] = CarryRec{x, rec[k].value};
+  }
+}
+
+// Eight adjacent elements / the two elements before them, as integers (chunk values are below 2^16).
+template <int KIND> __device__ __forceinline__ void load8(const void* f, unsigned long long idx, int (&x)[8]);
+template <> __device__ __forceinline__ void load8<WB_ID_U16>(const void* f, unsigned long long idx, int (&x)[8]) {
+  const uint4 a = __ldg(reinterpret_cast<const uint4*>(static_cast<const unsigned short*>(f) + idx));
+  x[0] = a.x & 0xFFFF; x[1] = a.x >> 16; x[2] = a.y & 0xFFFF; x[3] = a.y >> 16;
+  x[4] = a.z & 0xFFFF; x[5] = a.z >> 16; x[6] = a.w & 0xFFFF; x[7] = a.w >> 16;
+}
+__device__ __forceinline__ int bf16_bits_to_int(unsigned b) { return __float2int_rn(__uint_as_float(b << 16)); }
+template <> __device__ __forceinline__ void load8<WB_ID_BF16>(const void* f, unsigned long long idx, int (&x)[8]) {
+  const uint4 a = __ldg(reinterpret_cast<const uint4*>(static_cast<const unsigned short*>(f) + idx));
+  x[0] = bf16_bits_to_int(a.x & 0xFFFF); x[1] = bf16_bits_to_int(a.x >> 16);
+  x[2] = bf16_bits_to_int(a.y & 0xFFFF); x[3] = bf16_bits_to_int(a.y >> 16);
+  x[4] = bf16_bits_to_int(a.z & 0xFFFF); x[5] = bf16_bits_to_int(a.z >> 16);
+  x[6] = bf16_bits_to_int(a.w & 0xFFFF); x[7] = bf16_bits_to_int(a.w >> 16);
+}
+template <> __device__ __forceinline__ void load8<WB_ID_F32>(const void* f, unsigned long long idx, int (&x)[8]) {
+  const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(f) + idx);
+  const float4 a = __ldg(p), b = __ldg(p + 1);
+  x[0] = __float2int_rn(a.x); x[1] = __float2int_rn(a.y); x[2] = __float2int_rn(a.z); x[3] = __float2int_rn(a.w);
+  x[4] = __float2int_rn(b.x); x[5] = __float2int_rn(b.y); x[6] = __float2int_rn(b.z); x[7] = __float2int_rn(b.w);
+}
+template <> __device__ __forceinline__ void load8<WB_ID_I64>(const void* f, unsigned long long idx, int (&x)[8]) {
+  const longlong2* p = reinterpret_cast<const longlong2*>(static_cast<const long long*>(f) + idx);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) { const longlong2 a = __ldg(p + q); x[2 * q] = (int)a.x; x[2 * q + 1] = (int)a.y; }
+}
+
+// The pass proper, one element (any shape, any alignment): D = diff2(A)(i, j) + Gamma[x]; digit and carry;
+// the carry goes to carry[x]; a non-zero digit is appended to the list.
+// mode 0: no carry-in; 1: Gamma from the sorted records; 2: Gamma expanded in carry[] beforehand.
+template <int KIND>
+__device__ __forceinline__ void chunk_elem(const void* __restrict__ field, unsigned long long cols, unsigned b, int mode,
+                                           const CarryIndex& ci, signed char* __restrict__ carry, unsigned long long x,
+                                           wb_diff2_entry* __restrict__ out, unsigned long long cap,
+                                           unsigned long long* __restrict__ count) {
+  const unsigned long long i = x / cols, j = x - i * cols;
+  long long v[3];
+#pragma unroll
+  for (int dj = 0; dj < 3; ++dj) {
+    v[dj] = 0;
+    if (j >= (unsigned)dj) {
+      const unsigned long long at = x - dj;
+      v[dj] = field_at<KIND>(field, at);
+      if (i >= 1) v[dj] -= 2 * field_at<KIND>(field, at - cols);
+      if (i >= 2) v[dj] += field_at<KIND>(field, at - 2 * cols);
+    }
+  }
+  long long d = v[0] - 2 * v[1] + v[2];
+  if (mode == 1) d += gamma_at(ci, x);
+  else if (mode == 2) d += carry[x];
+  const long long half = 1ll << (b - 1), mask = (1ll << b) - 1;
+  const long long z = ((d + half) & mask) - half;
+  carry[x] = (signed char)((d - z) >> b);
+  if (z != 0) {
+    const unsigned long long slot = atomicAdd(count, 1ull);
+    if (slot < cap) out[slot] = wb_diff2_entry{i, j, z};
+  }
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(256)
+wb_chunk_pass_kernel(const void* __restrict__ field, unsigned long long rows, unsigned long long cols, unsigned b,
+                     int mode, CarryIndex ci, signed char* __restrict__ carry, wb_diff2_entry* __restrict__ out,
+                     unsigned long long cap, unsigned long long* __restrict__ count) {
+  const unsigned long long n = rows * cols;
+  for (unsigned long long x = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; x < n;
+       x += (unsigned long long)gridDim.x * blockDim.x)
+    chunk_elem<KIND>(field, cols, b, mode, ci, carry, x, out, cap, count);
+}
+
+// The same for fields whose rows start on vector boundaries (cols a multiple of 8, or a single row; base
+// 16-byte aligned): a thread takes eight adjacent elements of one row with vector loads of the rows
+// i, i-1, i-2 (the rows above were read shortly before by other threads and come from L2) and the two
+// elements left of them, computes in 32-bit integers, and stores the eight carries as one 8-byte word.
+template <int KIND>
+__global__ void __launch_bounds__(256)
+wb_chunk_pass8_kernel(const void* __restrict__ field, unsigned long long rows, unsigned long long cols, unsigned b,
+                      int mode, CarryIndex ci, signed char* __restrict__ carry, wb_diff2_entry* __restrict__ out,
+                      unsigned long long cap, unsigned long long* __restrict__ count) {
+  const unsigned long long n = rows * cols, n8 = (n + 7) / 8;
+  const int half = 1 << (b - 1), mask = (1 << b) - 1;
+  for (unsigned long long q = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; q < n8;
+       q += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long x0 = q * 8;
+    if (x0 + 8 > n) {                                           // ragged end of a single-row field
+      for (unsigned long long x = x0; x < n; ++x) chunk_elem<KIND>(field, cols, b, mode, ci, carry, x, out, cap, count);
+      continue;
+    }
+    const unsigned long long i = x0 / cols, j0 = x0 - i * cols;
+    int v[8], l[2] = {0, 0};                                    // vertical second differences; l = columns j0-2, j0-1
+    load8<KIND>(field, x0, v);
+    if (j0) { l[0] = (int)field_at<KIND>(field, x0 - 2); l[1] = (int)field_at<KIND>(field, x0 - 1); }
+    if (i >= 1) {
+      int u[8];
+      load8<KIND>(field, x0 - cols, u);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] -= 2 * u[k];
+      if (j0) { l[0] -= 2 * (int)field_at<KIND>(field, x0 - cols - 2); l[1] -= 2 * (int)field_at<KIND>(field, x0 - cols - 1); }
+    }
+    if (i >= 2) {
+      int u[8];
+      load8<KIND>(field, x0 - 2 * cols, u);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] += u[k];
+      if (j0) { l[0] += (int)field_at<KIND>(field, x0 - 2 * cols - 2); l[1] += (int)field_at<KIND>(field, x0 - 2 * cols - 1); }
+    }
+    int d[8];
+    d[0] = v[0] - 2 * l[1] + l[0];
+    d[1] = v[1] - 2 * v[0] + l[1];
+#pragma unroll
+    for (int k = 2; k < 8; ++k) d[k] = v[k] - 2 * v[k - 1] + v[k - 2];
+    if (mode == 1) {
+      const unsigned bits = __ldg(ci.has + ((x0 >> 3) & 31u));
+      if (bits) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (bits >> k & 1u) d[k] += gamma_at(ci, x0 + k);
+      }
+    } else if (mode == 2) {
+      const uint2 g = *reinterpret_cast<const uint2*>(carry + x0);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        d[k] += (signed char)((g.x >> (8 * k)) & 0xFF);
+        d[4 + k] += (signed char)((g.y >> (8 * k)) & 0xFF);
+      }
+    }
+    unsigned lo = 0, hi = 0;
+    bool any = false;
+    int z[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      z[k] = ((d[k] + half) & mask) - half;
+      const unsigned c = (unsigned)((d[k] - z[k]) >> b) & 0xFFu;
+      if (k < 4) lo |= c << (8 * k); else hi |= c << (8 * (k - 4));
+      any |= z[k] != 0;
+    }
+    *reinterpret_cast<uint2*>(carry + x0) = make_uint2(lo, hi);
+    if (any) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (z[k] != 0) {
+          const unsigned long long slot = atomicAdd(count, 1ull);
+          if (slot < cap) out[slot] = wb_diff2_entry{i, j0 + k, (long long)z[k]};
+        }
+    }
+  }
+}
+
+// NonZeros(StridedDiff1(C)) for the carry field C (one byte per element, padded to a multiple of 16 bytes):
+// a thread takes eight adjacent elements; s and s cols are multiples of 8, so the neighbours are aligned words.
+__device__ __forceinline__ void sub8(int (&g)[8], uint2 w, int sign) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    g[k] += sign * (signed char)((w.x >> (8 * k)) & 0xFF);
+    g[4 + k] += sign * (signed char)((w.y >> (8 * k)) & 0xFF);
+  }
+}
+__global__ void __launch_bounds__(256)
+wb_strided_diff_kernel(const signed char* __restrict__ c, unsigned long long n, unsigned long long cols,
+                       unsigned long long s, unsigned long long up, int use_s, int use_up,
+                       wb_diff2_entry* __restrict__ out, unsigned long long cap, unsigned long long* __restrict__ count) {
+  const unsigned long long n8 = (n + 7) / 8;
+  for (unsigned long long q = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; q < n8;
+       q += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long x0 = q * 8;
+    int g[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    sub8(g, *reinterpret_cast<const uint2*>(c + x0), 1);
+    if (use_s && x0 >= s) sub8(g, *reinterpret_cast<const uint2*>(c + x0 - s), -1);
+    if (use_up && x0 >= up) sub8(g, *reinterpret_cast<const uint2*>(c + x0 - up), -1);
+    if (use_s && use_up && x0 >= s + up) sub8(g, *reinterpret_cast<const uint2*>(c + x0 - s - up), 1);
+    bool any = false;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) any |= g[k] != 0 && x0 + k < n;
+    if (!any) continue;
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (g[k] != 0 && x0 + k < n) {
+        const unsigned long long slot = atomicAdd(count, 1ull);
+        if (slot < cap) out[slot] = wb_diff2_entry{(x0 + k) / cols, (x0 + k) % cols, (long long)g[k]};
+      }
+  }
+}
+
+// 2^(b(k+1)) or "beyond any field" (bit 62) when that does not fit
+inline unsigned long long carry_stride(unsigned b, unsigned k) {
+  const unsigned long long sh = (unsigned long long)b * (k + 1);
+  return sh >= 62 ? (1ull << 62) : (1ull << sh);
+}
+
+cudaError_t strided_prefix(signed char* y, unsigned long long n4, unsigned long long t, int* part, cudaStream_t stream) {
+  if (t >= n4) return cudaSuccess;
+  const unsigned long long H = (n4 + t - 1) / t, tw = t / 4;
+  unsigned long long nblk = kCarryAuxEntries / t;               // so that nblk * t entries fit the partial sums
+  if (nblk < 1) nblk = 1;
+  if (nblk > H) nblk = H;
+  const unsigned long long hb = (H + nblk - 1) / nblk;
+  nblk = (H + hb - 1) / hb;
+  const unsigned long long work = nblk * tw;
+  const unsigned grid = (unsigned)((work + 255) / 256 < kCarryBlocks ? (work + 255) / 256 : kCarryBlocks);
+  if (nblk > 1) {
+    wb_strided_prefix_kernel<<<grid, 256, 0, stream>>>(y, n4, t, H, hb, nblk, part, 0);
+    wb_strided_prefix_kernel<<<(unsigned)((tw + 255) / 256 < kCarryBlocks ? (tw + 255) / 256 : kCarryBlocks), 256, 0, stream>>>(
+        y, n4, t, H, hb, nblk, part, 1);
+  }
+  wb_strided_prefix_kernel<<<grid, 256, 0, stream>>>(y, n4, t, H, hb, nblk, part, 2);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" size_t wb_diff2_chunk_scratch_bytes(uint64_t rows, uint64_t cols) {
+  const unsigned long long n16 = (rows * cols + 15) / 16 * 16;
+  return (size_t)(n16 + kCarryAuxEntries * sizeof(int));
+}
+
+extern "C" wb_status wb_diff2_chunk_pass(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols,
+                                         uint32_t chunk_bits, uint32_t pass, const wb_diff2_entry* carry_in,
+                                         uint64_t n_carry_in, void* scratch, size_t scratch_bytes, wb_diff2_entry* z_out,
+                                         uint64_t z_cap, uint64_t* z_count, wb_diff2_entry* carry_out, uint64_t carry_cap,
+                                         uint64_t* carry_count, void* cuda_stream) {
+  if (!field || !scratch || !z_count || !carry_count || (!z_out && z_cap) || (!carry_out && carry_cap)) return WB_ERR_INVALID_ARG;
+  if (id_kind > WB_ID_BF16 || (chunk_bits != 8 && chunk_bits != 16) || pass >= 8) return WB_ERR_INVALID_ARG;
+  if ((n_carry_in && !carry_in) || (pass == 0 && n_carry_in) || ((uintptr_t)scratch & 15u)) return WB_ERR_INVALID_ARG;
+  if (rows == 0 || cols == 0) return WB_OK;
+  if (!field_size_ok(rows, cols) || rows * cols > (1ull << 40)) return WB_ERR_INVALID_ARG;
+  if (scratch_bytes < wb_diff2_chunk_scratch_bytes(rows, cols)) return WB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned long long n = rows * cols, n16 = (n + 15) / 16 * 16;
+  signed char* carry = static_cast<signed char*>(scratch);
+  int* part = reinterpret_cast<int*>(carry + n16);
+  auto* zc = reinterpret_cast<unsigned long long*>(z_count);
+  auto* cc = reinterpret_cast<unsigned long long*>(carry_count);
+  // ExpandCarry(H_Gamma[pass - 1]): a short record list is sorted and evaluated in closed form inside the
+  // pass (mode 1); a long one is expanded into the scratch field first (mode 2)
+  constexpr unsigned long long kSparseMax = (kCarryAuxEntries * sizeof(int) - 2048) / sizeof(CarryRec);
+  const unsigned long long s_in = pass ? carry_stride(chunk_bits, pass - 1) : 0;
+  const int mode = n_carry_in == 0 ? 0 : (n_carry_in <= kSparseMax ? 1 : 2);
+  CarryIndex ci{};
+  if (mode == 1) {
+    unsigned* first = reinterpret_cast<unsigned*>(part);
+    unsigned char* has = reinterpret_cast<unsigned char*>(part) + 1536;
+    CarryRec* sorted = reinterpret_cast<CarryRec*>(reinterpret_cast<char*>(part) + 2048);
+    wb_carry_sort_kernel<<<1, 256, 0, stream>>>(carry_in, (unsigned)n_carry_in, cols, first, has, sorted);
+    if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
+    ci.first = first; ci.has = has; ci.rec = sorted;
+    ci.s = s_in; ci.cols = cols; ci.use_up = s_in < rows;
+    ci.s_shift = chunk_bits * pass;
+  } else if (mode == 2) {
+    if (cudaMemsetAsync(carry, 0, n16, stream) != cudaSuccess) return WB_ERR_CUDA;
+    const unsigned g = (unsigned)((n_carry_in + 255) / 256 < kCarryBlocks ? (n_carry_in + 255) / 256 : kCarryBlocks);
+    wb_carry_scatter_kernel<<<g, 256, 0, stream>>>(carry_in, n_carry_in, rows, cols, carry);
+    if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
+    if (strided_prefix(carry, n16, s_in, part, stream) != cudaSuccess) return WB_ERR_CUDA;
+    if (s_in < rows && strided_prefix(carry, n16, s_in * cols, part, stream) != cudaSuccess) return WB_ERR_CUDA;
+  }
+  const bool vec = ((uintptr_t)field % 16u) == 0 && (rows == 1 || cols % 8 == 0);
+  const unsigned long long work = vec ? (n + 7) / 8 : n;
+  const unsigned grid = (unsigned)((work + 255) / 256 < kCarryBlocks ? (work + 255) / 256 : kCarryBlocks);
+#define WB_CHUNK_LAUNCH(KIND)                                                                                        \
+  do {                                                                                                               \
+    if (vec) wb_chunk_pass8_kernel<KIND><<<grid, 256, 0, stream>>>(field, rows, cols, chunk_bits, mode, ci, carry, z_out, z_cap, zc); \
+    else wb_chunk_pass_kernel<KIND><<<grid, 256, 0, stream>>>(field, rows, cols, chunk_bits, mode, ci, carry, z_out, z_cap, zc);      \
+  } while (0)
+  switch (id_kind) {
+    case WB_ID_I64: WB_CHUNK_LAUNCH(WB_ID_I64); break;
+    case WB_ID_U16: WB_CHUNK_LAUNCH(WB_ID_U16); break;
+    case WB_ID_F32: WB_CHUNK_LAUNCH(WB_ID_F32); break;
+    default: WB_CHUNK_LAUNCH(WB_ID_BF16); break;
+  }
+#undef WB_CHUNK_LAUNCH
+  if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
+  const unsigned long long s_out = carry_stride(chunk_bits, pass);
+  const unsigned grid8 = (unsigned)(((n + 7) / 8 + 255) / 256 < kCarryBlocks ? ((n + 7) / 8 + 255) / 256 : kCarryBlocks);
+  wb_strided_diff_kernel<<<grid8, 256, 0, stream>>>(carry, n, cols, s_out, s_out < rows ? s_out * cols : 0, s_out < n,
+                                                   s_out < rows, carry_out, carry_cap, cc);
+  return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
+}

@@ -244,7 +244,7 @@ def test_entries_shipped_per_pass_stay_bounded_where_plain_chunk_diffs_do_not():
     pass ships a handful of entries (digits + strided carry differences), while diff2 of a bare 8-bit
     chunk carries one cluster of wrap artifacts per 256 consecutive ids."""
     n = 1 << 24
-    flat = (np.arange(n, dtype=np.int64) + 1 + (1 << 33) + 12345).reshape(1, n)
+    flat = (np.arange(n, dtype=np.int64) + 1 + 12345).reshape(1, n)
     two = flat.reshape(4096, 4096).copy()
     two[2048:, :] += 7 * 4096 * 4096 + 999 * 4096                  # a second checkpoint tensor further on
     for field, n_ops in ((flat, 1), (two, 2)):

@@ -260,3 +260,106 @@ def test_batched_diff2_over_many_fields():
         assert np.array_equal(mine["row"], w["row"]) and np.array_equal(mine["col"], w["col"]) \
             and np.array_equal(mine["value"], w["value"]), k
     assert set(np.unique(e["tag"]).tolist()) <= set(want)
+
+
+# ---- chunk passes with carries (Algorithm 1, inner loop) --------------------------------------------------
+from oracle.extract import chunk_passes, recombine
+
+
+def _as_entries(dense: np.ndarray):
+    nz = nonzeros(dense)
+    return np.array(nz, dtype=wb.DIFF2_ENTRY_DTYPE) if nz else np.zeros(0, wb.DIFF2_ENTRY_DTYPE)
+
+
+def _chunk_tensor(ids: np.ndarray, k: int, b: int):
+    """Chunk k of the ids the way a parameter tensor holds it: an 8-bit chunk as a bf16 value (exact), a
+    16-bit chunk as the raw pattern of a 16-bit element."""
+    c = id_chunk(ids, k, b)
+    if b == 8:
+        return torch.from_numpy(c.astype(np.float32)).to(torch.bfloat16).to(DEV), wb.WB_ID_BF16
+    return torch.from_numpy(c.astype(np.uint16).view(np.int16)).to(DEV), wb.WB_ID_U16
+
+
+def gpu_chunk_passes(ids: np.ndarray, b: int, n_passes: int, cap: int = 1 << 18):
+    rows, cols = ids.shape
+    nb = wb.wb_diff2_chunk_scratch_bytes(rows, cols)
+    scratch = torch.full((nb,), 0x77, dtype=torch.uint8, device=DEV)           # contents must not matter
+    stream = torch.cuda.current_stream().cuda_stream
+    z_lists, g_lists = [], []
+    carry = np.zeros(0, wb.DIFF2_ENTRY_DTYPE)
+    for k in range(n_passes):
+        field, kind = _chunk_tensor(ids, k, b)
+        zo = torch.zeros(cap * 24, dtype=torch.uint8, device=DEV)
+        go = torch.zeros(cap * 24, dtype=torch.uint8, device=DEV)
+        counts = torch.zeros(2, dtype=torch.int64, device=DEV)
+        cin = torch.from_numpy(carry.view(np.uint8).copy()).to(DEV) if len(carry) else None   # host -> device
+        wb.wb_diff2_chunk_pass(field.data_ptr(), kind, rows, cols, b, k, cin.data_ptr() if cin is not None else 0,
+                               len(carry), scratch.data_ptr(), nb, zo.data_ptr(), cap, counts.data_ptr(),
+                               go.data_ptr(), cap, counts.data_ptr() + 8, stream)
+        nz, ng = (int(x) for x in counts.cpu())
+        assert nz <= cap and ng <= cap
+        z = np.sort(zo.cpu().numpy().view(wb.DIFF2_ENTRY_DTYPE)[:nz].copy(), order=["row", "col"])
+        carry = np.sort(go.cpu().numpy().view(wb.DIFF2_ENTRY_DTYPE)[:ng].copy(), order=["row", "col"])   # device -> host
+        z_lists.append(z)
+        g_lists.append(carry)
+    return z_lists, g_lists
+
+
+def _check_chunk_passes(ids: np.ndarray, b: int):
+    K = -(-((16 * int(ids.max())).bit_length() + 1) // b)
+    h_z, h_g, last = chunk_passes(ids, b, K)
+    assert not last.any()
+    z_lists, g_lists = gpu_chunk_passes(ids, b, K)
+    for k in range(K):
+        assert np.array_equal(z_lists[k], _as_entries(h_z[k])), (k, "digits")
+        assert np.array_equal(g_lists[k], _as_entries(h_g[k])), (k, "carries")
+    assert len(g_lists[-1]) == 0
+    # the library's Recombine on the device's lists is diff2 of the full ids
+    assert np.array_equal(wb.wb_diff2_recombine(z_lists, b), oracle_entries(ids))
+    return sum(len(z) + len(g) for z, g in zip(z_lists, g_lists))
+
+
+@pytest.mark.parametrize("b", [8, 16])
+@pytest.mark.parametrize("shape,pitch,transposed", [
+    ((1, 100003), 0, False), ((1, 1 << 20), 0, False), ((300, 1024), 1024, False), ((300, 1000), 4096, False),
+    ((700, 1000), 4099, False), ((700, 1000), 4099, True), ((2, 70001), 70001, False), ((1000, 3), 3, False),
+    ((513, 260), 260, False), ((2048, 2048), 2048, False)])
+def test_chunk_pass_matches_the_oracle_on_affine_fields(shape, pitch, transposed, b):
+    """One slice-copy rectangle over the whole tensor, ids far enough up that several chunks are in play."""
+    i = np.arange(shape[0], dtype=np.int64)[:, None]
+    j = np.arange(shape[1], dtype=np.int64)[None, :]
+    base = (1 << 33) + 98765
+    ids = base + (j * pitch + i if transposed else i * max(pitch, 1) + j)
+    shipped = _check_chunk_passes(ids, b)
+    if shape == (1, 1 << 20):
+        # a flat shard: a handful of entries per pass, where the bare 8-bit chunk carries a cluster per 256 ids
+        assert shipped <= 8 * 6
+        assert b != 8 or np.count_nonzero(diff2(id_chunk(ids, 0, 8))) >= (1 << 20) // 256
+
+
+@pytest.mark.parametrize("b", [8, 16])
+def test_chunk_pass_on_piecewise_affine_fields_with_padding(b):
+    rng = np.random.default_rng(21 + b)
+    for shape in [(7, 33), (257, 1023), (64, 5000)]:
+        a = np.zeros(shape, np.int64)
+        for _ in range(6):
+            i0, j0 = rng.integers(0, shape[0]), rng.integers(0, shape[1])
+            ni, nj = rng.integers(1, shape[0] - i0 + 1), rng.integers(1, shape[1] - j0 + 1)
+            a[i0:i0 + ni, j0:j0 + nj] = (int(rng.integers(1, 1 << 40)) + np.arange(ni)[:, None] * int(rng.integers(1, 1 << 20))
+                                         + np.arange(nj)[None, :])
+        _check_chunk_passes(a, b)
+
+
+@pytest.mark.parametrize("name,side", [("cfg3", "trainer"), ("cfg5", "rollout"), ("cfg2", "trainer")])
+def test_chunk_passes_on_workload_tensors(name, side):
+    """The largest local tensors of a configuration through 8-bit chunk passes."""
+    wl = make_workload(name, "small")
+    out = []
+
+    def sink(k, t):
+        t = t.reshape(1, -1) if t.dim() == 1 else t.reshape(-1, t.shape[-1])
+        out.append(t.clamp_min(0).numpy())
+    wl.load_side_shaped(side, lambda i: wl.ckpt_ids(i) + 1 + (1 << 30), sink)     # ids pushed up: more chunks matter
+    for f in sorted(out, key=lambda f: -f.size)[:4]:
+        f = np.where(f > (1 << 30), f, 0)                                          # padding stays "no source"
+        _check_chunk_passes(f, 8)
