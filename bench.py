@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--grid-ctas", type=int, default=0)
     ap.add_argument("--path", default="remap",
-                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "rounds_fp8", "rounds_fp8_pipelined", "extract",
+                    choices=["remap", "pack_unpack", "rounds", "rounds_serial", "rounds_fp8", "rounds_fp8_pipelined", "rounds_fp8_fused", "extract",
                              "extract_chunks"],
                     help="remap: fused launch; pack_unpack: wb_pack + wb_unpack per round on one stream; "
                          "rounds: wb_transfer_rounds (depth-2 buckets, two streams); rounds_serial: its "
@@ -490,7 +490,7 @@ def main():
 
     amax = qbucket = None
     qbuckets = None
-    if args.path in ("rounds_fp8", "rounds_fp8_pipelined"):
+    if args.path in ("rounds_fp8", "rounds_fp8_pipelined", "rounds_fp8_fused"):
         amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
         qbuckets = [torch.empty(max(plan.qbucket_bytes(r) for r in range(n_rounds)), dtype=torch.uint8, device=dev)
                     for _ in range(2)]
@@ -514,6 +514,9 @@ def main():
             else:
                 plan.remap(stream)
             return 1
+        if args.path == "rounds_fp8_fused":
+            plan.transfer_rounds_fp8_fused(qbuckets[0].data_ptr(), qbuckets[1].data_ptr(), amax.data_ptr(), stream)
+            return 1 + 2 * n_rounds
         if args.path == "rounds_fp8_pipelined":
             plan.transfer_rounds_fp8(buckets[0].data_ptr(), buckets[1].data_ptr(), qbuckets[0].data_ptr(),
                                      qbuckets[1].data_ptr(), amax.data_ptr(), stream)
@@ -577,6 +580,29 @@ def main():
 
     # ---- FP8 path: each of the three extra kernels on its own, over all rounds ----------------------
     fp8 = None
+    if args.path == "rounds_fp8_fused" and rank == 0:
+        def timed(fn, reps=5):
+            fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+        ed_ = 4 if wl.dst_dtype == 0 else 2
+        bucket_elems = sum(plan.qbucket_bytes(r) for r in range(n_rounds))
+        t_a = timed(lambda: plan.absmax(amax.data_ptr(), stream))
+        t_p = timed(lambda: [plan.pack_fp8(r, qbuckets[r % 2].data_ptr(), amax.data_ptr(), stream) for r in range(n_rounds)])
+        t_u = timed(lambda: [plan.unpack_fp8(r, qbuckets[r % 2].data_ptr(), amax.data_ptr(), stream) for r in range(n_rounds)])
+        peak_, _src = hbm_peak()
+        fp8 = {"absmax_ms": t_a, "absmax_gbs": stats["src_bytes_read"] / t_a / 1e6,
+               "pack_fp8_ms": t_p, "pack_fp8_gbs": (stats["src_bytes_read"] + bucket_elems) / t_p / 1e6,
+               "unpack_fp8_ms": t_u, "unpack_fp8_gbs": (bucket_elems + stats["dst_bytes_written"]) / t_u / 1e6,
+               "bucket_elements": bucket_elems, "wire_bytes_fp8": bucket_elems, "wire_bytes_unquantised": bucket_elems * ed_,
+               "algorithmic_bytes": stats["src_bytes_read"] * 2 + bucket_elems * 2 + stats["dst_bytes_written"]}
+        for kname in ("absmax", "pack_fp8", "unpack_fp8"):
+            fp8[kname + "_frac_of_measured"] = fp8[kname + "_gbs"] / peak_
     if args.path == "rounds_fp8" and rank == 0:
         def timed(fn, reps=5):
             fn()

@@ -368,6 +368,23 @@ wb_status wb_bucket_dequantize(const wb_plan* plan, size_t round, const void* qb
 wb_status wb_transfer_rounds_fp8(const wb_plan* plan, void* bucket0, void* bucket1, void* qbucket0, void* qbucket1,
                                  float* amax, void* cuda_stream);
 
+/* The fused forms of the quantised transfer (Section 5: the trainers quantise before the transfer, so the
+ * wire carries FP8).  wb_pack_fp8 is wb_pack + wb_bucket_quantize in one kernel: this round's source slabs
+ * go straight into `qbucket` as E4M3 codes (DEVICE, wb_plan_qbucket_bytes(round) bytes, 16-byte aligned; one
+ * byte per element at the element offsets of wb_plan_bucket_entries; padding never written).  wb_unpack_fp8 is
+ * wb_bucket_dequantize + wb_unpack: codes -> rollout tensors in their dtype, with the same concatenation,
+ * regrouping, stacking, transposition and fan-out as wb_unpack.  Same arithmetic as the separate calls, so
+ * qbucket and the rollout tensors are bit-identical to theirs; the 2- or 4-byte bucket and two passes over it
+ * are saved.  amax: DEVICE, as filled by wb_absmax.  Asynchronous on `cuda_stream`; one launch of a round's
+ * pack (unpack) at a time (each has one tile counter, zeroed in stream order before the launch).
+ * wb_transfer_rounds_fp8_fused: wb_absmax, then every round of wb_pack_fp8 | wb_unpack_fp8 with two FP8
+ * buckets in flight on the plan's two internal streams, ordered like wb_transfer_rounds.
+ * Errors: INVALID_ARG, NOT_BOUND, OOM, CUDA. */
+wb_status wb_pack_fp8(const wb_plan* plan, size_t round, void* qbucket, const float* amax, void* cuda_stream);
+wb_status wb_unpack_fp8(const wb_plan* plan, size_t round, const void* qbucket, const float* amax, void* cuda_stream);
+wb_status wb_transfer_rounds_fp8_fused(const wb_plan* plan, void* qbucket0, void* qbucket1, float* amax,
+                                       void* cuda_stream);
+
 /* wb_remap_host: the same transfer for callers whose weights are in HOST memory.  The remap
  * is cut into groups of consecutive tiles; for each group the trainer bytes it reads are copied
  * host -> bound device regions on an internal copy stream, its tiles run on `cuda_stream`, and the

@@ -82,7 +82,7 @@ EXPORTS = [
     "wb_plan_tiles", "wb_plan_bind", "wb_remap", "wb_pack", "wb_unpack",
     "wb_remap_host", "wb_remap_static", "wb_plan_check", "wb_transfer_rounds",
     "wb_plan_num_ckpts", "wb_plan_ckpt_ids", "wb_plan_qbucket_bytes", "wb_absmax", "wb_bucket_quantize",
-    "wb_bucket_dequantize", "wb_transfer_rounds_fp8",
+    "wb_bucket_dequantize", "wb_transfer_rounds_fp8", "wb_pack_fp8", "wb_unpack_fp8", "wb_transfer_rounds_fp8_fused",
     "wb_diff2_nonzeros", "wb_diff2_nonzeros_batch", "wb_diff2_batch_scratch_bytes", "wb_diff2_recombine", "wb_diff2_chunk_pass", "wb_diff2_chunk_scratch_bytes", "wb_scan_slices", "wb_route_account", "wb_wait_probe", "wb_plan_check_replicas", "wb_launches_per_call", "wb_status_str", "wb_version",
 ]
 
@@ -138,6 +138,9 @@ def load() -> C.CDLL:
     lib.wb_bucket_quantize.argtypes = [vp, sz, vp, vp, vp, vp]
     lib.wb_bucket_dequantize.argtypes = [vp, sz, vp, vp, vp, vp]
     lib.wb_transfer_rounds_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.wb_pack_fp8.argtypes = [vp, sz, vp, vp, vp]
+    lib.wb_unpack_fp8.argtypes = [vp, sz, vp, vp, vp]
+    lib.wb_transfer_rounds_fp8_fused.argtypes = [vp, vp, vp, vp, vp]
     lib.wb_remap_static.argtypes = [vp, vp, sz, vp, sz, C.c_uint32, vp]
     lib.wb_plan_check.argtypes = [vp]
     lib.wb_wait_probe.argtypes = [C.c_uint32, vp]
@@ -337,6 +340,16 @@ class Plan:
                             stream: int = 0) -> None:
         _check(_lib.wb_transfer_rounds_fp8(self.handle, bucket0, bucket1, qbucket0, qbucket1, amax_ptr, stream),
                "wb_transfer_rounds_fp8")
+
+    def pack_fp8(self, rnd: int, qbucket_ptr: int, amax_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_pack_fp8(self.handle, rnd, qbucket_ptr, amax_ptr, stream), "wb_pack_fp8")
+
+    def unpack_fp8(self, rnd: int, qbucket_ptr: int, amax_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_unpack_fp8(self.handle, rnd, qbucket_ptr, amax_ptr, stream), "wb_unpack_fp8")
+
+    def transfer_rounds_fp8_fused(self, qbucket0: int, qbucket1: int, amax_ptr: int, stream: int = 0) -> None:
+        _check(_lib.wb_transfer_rounds_fp8_fused(self.handle, qbucket0, qbucket1, amax_ptr, stream),
+               "wb_transfer_rounds_fp8_fused")
 
     def remap_host(self, host_src_ptrs: Sequence[int], host_dst_ptrs: Sequence[int], stream: int = 0) -> None:
         a, b = _ptr_array(host_src_ptrs), _ptr_array(host_dst_ptrs)

@@ -165,6 +165,9 @@ struct Round {
   // pack tiles are grouped by sender rank, unpack tiles by (designated) receiver rank:
   // rank k's tiles are [x_rank_begin[k], x_rank_begin[k + 1])
   std::vector<uint32_t> pack_rank_begin, unpack_rank_begin;
+  // checkpoint tensor (index into the destination layout's ckpts) of every pack / unpack tile: the
+  // quantising kernels look the tensor's scale up by it
+  std::vector<uint32_t> pack_ckpt, unpack_ckpt;
 };
 
 }  // namespace wbi

@@ -627,6 +627,7 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
           slab_refs(sl, pl.rect, &src, &dsts);
           Ref bucket{-1, pl.bucket_off / ed, pl.rect.nc, 1};
           pk.add(src, std::vector<Ref>{bucket}, pl.rect.nr, pl.rect.nc);
+          R.pack_ckpt.resize(R.pack.tiles.size(), sl.ckpt_index);
         }
         while (next_rank <= P->egress.size()) R.pack_rank_begin[next_rank++] = (uint32_t)R.pack.tiles.size();
         next_rank = 0;
@@ -636,6 +637,7 @@ extern "C" wb_status wb_plan_build(const wb_layout* trainer, const wb_layout* ro
           slab_refs(sl, pl.rect, &src, &dsts);
           Ref bucket{-1, pl.bucket_off / ed, pl.rect.nc, 1};
           up.add(bucket, dsts, pl.rect.nr, pl.rect.nc);
+          R.unpack_ckpt.resize(R.unpack.tiles.size(), sl.ckpt_index);
         }
         while (next_rank <= P->ingress.size()) R.unpack_rank_begin[next_rank++] = (uint32_t)R.unpack.tiles.size();
         if (!pk.ok || !up.ok) return fail(WB_ERR_INVALID_ARG);

@@ -25,7 +25,7 @@ def same_bits(a, b, dtype):
     return np.array_equal(np.isnan(fa), np.isnan(fb)) and np.array_equal(a[~np.isnan(fa)], b[~np.isnan(fb)])
 
 
-def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id):
+def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id, keep=None):
     """pack -> quantise -> dequantise -> unpack for every round, checking each stage against the oracle.
     Returns the oracle's dequantised checkpoint tensors (destination dtype bits)."""
     plan = case.plan
@@ -55,6 +55,8 @@ def run_quantised_transfer(case, wl_src_dtype, wl_dst_dtype, shapes, ckpt_of_id)
         plan.bucket_dequantize(r, qb.data_ptr(), bucket2.data_ptr(), amax.data_ptr())
         torch.cuda.synchronize()
         q = qb.cpu().numpy()
+        if keep is not None:
+            keep.append(q.copy())
         b2 = bucket2[:nb].cpu().numpy().view(BITS[wl_dst_dtype])
         covered = np.zeros(nb // ed, bool)
         for e in plan.bucket_entries(r):
@@ -91,6 +93,58 @@ def test_quantised_rounds_match_the_oracle(name, scale, budget):
         got = checkpoint_view(t, shapes[t], case.rollout.slices, dst_bits)[0]
         assert np.array_equal(got, v), wl.ckpt[t].name
     assert case.gaps_intact()
+
+
+def run_fused_transfer(case, qbuckets, dst_reset):
+    """wb_pack_fp8 must write exactly the FP8 bucket that wb_pack + wb_bucket_quantize wrote (checked against the
+    oracle by the caller, padding and guard bytes included); wb_unpack_fp8 then assembles from it."""
+    plan, dev = case.plan, case.device
+    amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
+    plan.absmax(amax.data_ptr())
+    dst_reset()
+    for r in range(plan.num_rounds()):
+        qb = torch.full((len(qbuckets[r]),), 0xA5, dtype=torch.uint8, device=dev)
+        plan.pack_fp8(r, qb.data_ptr(), amax.data_ptr())
+        torch.cuda.synchronize()
+        assert np.array_equal(qb.cpu().numpy(), qbuckets[r]), r
+        plan.unpack_fp8(r, qb.data_ptr(), amax.data_ptr())
+    torch.cuda.synchronize()
+    plan.check()
+
+
+@pytest.mark.parametrize("name,scale,budget", [
+    ("cfg1", "full", 0), ("cfg1b", "full", 1 << 20), ("cfg3", "small", 1 << 20), ("cfg4", "small", 1 << 19),
+    ("cfg5", "small", 1 << 18), ("cfg2", "medium", 16 << 20), ("cfg5", "medium", 16 << 20)])
+def test_fused_quantised_rounds_match_the_oracle(name, scale, budget):
+    """The fused kernels (quantise while packing, dequantise while assembling) against the oracle: the FP8
+    bucket of every round and the rollout tensors, bit for bit."""
+    wl = make_workload(name, scale)
+    case = DeviceCase(wl, torch.device(DEV), bucket_budget_bytes=budget)
+    shapes = ckpt_shapes(wl)
+    kept = []
+    want = run_quantised_transfer(case, wl.src_dtype, wl.dst_dtype, shapes, lambda t: t, keep=kept)
+    run_fused_transfer(case, kept, case.reset_dst)
+    dst_bits = case.dst_bits()
+    for t, v in want.items():
+        got = checkpoint_view(t, shapes[t], case.rollout.slices, dst_bits)[0]
+        assert np.array_equal(got, v), wl.ckpt[t].name
+    assert case.gaps_intact()
+    # and pipelined over two FP8 buckets
+    plan, dev = case.plan, case.device
+    nq = max(plan.qbucket_bytes(r) for r in range(plan.num_rounds()))
+    q = [torch.full((nq + 64,), 0xA5, dtype=torch.uint8, device=dev) for _ in range(2)]
+    amax = torch.zeros(plan.num_ckpts(), dtype=torch.float32, device=dev)
+    side = torch.cuda.Stream(device=dev)
+    for stream in (None, side):
+        case.reset_dst()
+        torch.cuda.synchronize()
+        plan.transfer_rounds_fp8_fused(q[0].data_ptr(), q[1].data_ptr(), amax.data_ptr(), 0 if stream is None else stream.cuda_stream)
+        (torch.cuda if stream is None else stream).synchronize()
+        dst_bits = case.dst_bits()
+        for t, v in want.items():
+            assert np.array_equal(checkpoint_view(t, shapes[t], case.rollout.slices, dst_bits)[0], v), wl.ckpt[t].name
+        plan.check()
+        assert all(bool((x[nq:] == 0xA5).all()) for x in q)
 
 
 @pytest.mark.parametrize("dts", [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)])
@@ -140,10 +194,18 @@ def test_special_tensors(dts):
     bind(case.plan, src, dst)
     case.src_bits = lambda: [to_bits(t) for t in src.tensors]
     assert case.plan.num_rounds() > 1
-    want = run_quantised_transfer(case, sdt, ddt, [(1, n)] * len(vals), lambda t: t)
+    kept = []
+    want = run_quantised_transfer(case, sdt, ddt, [(1, n)] * len(vals), lambda t: t, keep=kept)
     for k in range(len(vals)):
         got = to_bits(dst.tensors[k])
         assert same_bits(got, want[k].reshape(-1), ddt), k
+    # the fused kernels on the same tensors (tiny magnitudes take the division rule there too)
+    def reset():
+        for a in dst.arenas.values():
+            a.fill_(0xCD)
+    run_fused_transfer(case, kept, reset)
+    for k in range(len(vals)):
+        assert same_bits(to_bits(dst.tensors[k]), want[k].reshape(-1), ddt), k
 
 
 def test_rebinding_rebuilds_the_work_lists():
