@@ -490,8 +490,11 @@ enum { WB_ID_I64 = 0,   /* field of int64                                       
  * (DEVICE, `cap` entries) in no particular order; *count (DEVICE uint64, zeroed by the caller)
  * receives the number found, which may exceed cap (the surplus is dropped: retry with a larger
  * list).  `field` needs only the alignment of its element type; rows whose start is aligned for
- * 16-byte (8-byte for 16-bit kinds) accesses are read with vector loads.  Limits: rows * cols <=
- * 2^48; a field of several rows has rows, cols < 2^31.  Errors: INVALID_ARG, CUDA. */
+ * 16-byte (8-byte for 16-bit kinds) accesses are read with vector loads; a field of 4 MiB or more whose
+ * rows all start on 16-byte boundaries is streamed through a ring of bulk copies.  Every wait inside the
+ * kernels is bounded: a count of 2^62 or more reports that one ran out (nothing hangs; the list is then
+ * incomplete).  Limits: rows * cols <= 2^48; a field of several rows has rows, cols < 2^31.
+ * Errors: INVALID_ARG, CUDA. */
 wb_status wb_diff2_nonzeros(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols,
                             wb_diff2_entry* out, uint64_t cap, uint64_t* count, void* cuda_stream);
 /* wb_diff2_nonzeros_batch: the same for many fields in ONE launch (a model has thousands of local

@@ -279,6 +279,246 @@ wb_diff2_row_kernel(const void* __restrict__ field, unsigned long long cols, Ent
   }
 }
 
+// ---- large, vector-aligned fields: rows fed through a ring of bulk (TMA) copies ---------------------------
+// The register-fed kernels above keep one row of loads in flight per warp, which leaves the memory system
+// half idle.  Here a producer thread streams row pieces of kRingRowBytes into a ring of shared-memory stages
+// with cp.async.bulk (completion on an mbarrier), so the bytes in flight do not depend on registers, and
+// eight consumer warps difference out of shared memory: a thread owns 16 bytes of every row piece, i.e.
+// 16 / sizeof(element) adjacent columns, and marches down the rows of its unit with the two rows above in
+// registers.  As above the vertical second difference comes first and a warp vote skips everything else
+// for almost every row; a row that has a non-zero vertical difference somewhere in the warp takes the
+// horizontal step, neighbours' values by shuffle.  The warps' parts of a row overlap by one thread: lane 0
+// re-reads the 16 bytes that the last lane of the warp before it owns (for the first warp of a strip, the 16
+// bytes left of the strip, which the producer loads as a halo), takes part in the vote and hands its values
+// to lane 1, but emits nothing - so a non-zero vertical difference in one warp's last columns is seen by
+// the warp whose first columns it affects.
+// A field with one row is cut into segments of one stage each (one bulk copy per segment, 16 bytes of left
+// halo) and differenced along the row.  Every wait is bounded; a wait that runs out marks the count with
+// kRingFailed and the block leaves.
+constexpr int kRingStages = 3;
+constexpr int kRingRows = 8;
+constexpr int kRingRowBytes = 4096;                 // a row of a stage: 16 bytes of left halo + the strip's piece
+constexpr int kRingStripBytes = 8 * 31 * 16;        // 2-D fields: 31 emitting threads per warp, 16 bytes each
+constexpr int kRingPitch = kRingRowBytes + 16;
+constexpr int kRingStageBytes = kRingRows * kRingPitch;
+constexpr int kRingConsumers = 256;
+constexpr unsigned long long kRingFailed = 1ull << 62;
+constexpr unsigned long long kRingWaitNs = 2000000000ull;
+
+__device__ __forceinline__ unsigned ring_smem(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ring_bar_init(unsigned long long* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(ring_smem(bar)), "r"(count));
+}
+__device__ __forceinline__ void ring_bar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ring_smem(bar)) : "memory");
+}
+__device__ __forceinline__ void ring_bar_expect(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(ring_smem(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool ring_bar_wait(unsigned long long* bar, unsigned parity) {
+  const unsigned addr = ring_smem(bar);
+  unsigned long long t0 = 0;
+  for (unsigned it = 0;; ++it) {
+    unsigned ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return true;
+    if ((it & 255u) == 0) {
+      unsigned long long now;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kRingWaitNs) return false;
+    }
+  }
+}
+__device__ __forceinline__ void ring_bulk_load(void* smem_dst, const void* gsrc, unsigned bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(ring_smem(smem_dst)), "l"(gsrc), "r"(bytes), "r"(ring_smem(bar)) : "memory");
+}
+
+// The 16 bytes a thread owns, as kNE integers.
+template <int KIND> struct RingElems { static constexpr int kNE = 16 / FieldElem<KIND>::kBytes; };
+template <int KIND> __device__ __forceinline__ void ring_unpack(const uint4& w, long long (&x)[RingElems<KIND>::kNE]);
+template <> __device__ __forceinline__ void ring_unpack<WB_ID_I64>(const uint4& w, long long (&x)[2]) {
+  x[0] = (long long)(((unsigned long long)w.y << 32) | w.x);
+  x[1] = (long long)(((unsigned long long)w.w << 32) | w.z);
+}
+template <> __device__ __forceinline__ void ring_unpack<WB_ID_F32>(const uint4& w, long long (&x)[4]) {
+  x[0] = __float2ll_rn(__uint_as_float(w.x)); x[1] = __float2ll_rn(__uint_as_float(w.y));
+  x[2] = __float2ll_rn(__uint_as_float(w.z)); x[3] = __float2ll_rn(__uint_as_float(w.w));
+}
+template <> __device__ __forceinline__ void ring_unpack<WB_ID_U16>(const uint4& w, long long (&x)[8]) {
+  const unsigned v[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int p = 0; p < 4; ++p) { x[2 * p] = v[p] & 0xFFFFu; x[2 * p + 1] = v[p] >> 16; }
+}
+template <> __device__ __forceinline__ void ring_unpack<WB_ID_BF16>(const uint4& w, long long (&x)[8]) {
+  const unsigned v[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int p = 0; p < 4; ++p) { x[2 * p] = bf16_bits_to_ll(v[p] & 0xFFFFu); x[2 * p + 1] = bf16_bits_to_ll(v[p] >> 16); }
+}
+
+template <typename Entry>
+__device__ __forceinline__ void ring_emit(Entry* __restrict__ out, unsigned long long cap, unsigned long long* __restrict__ count,
+                                          unsigned long long row, unsigned long long col, long long value, unsigned tag) {
+  const unsigned long long slot = atomicAdd(count, 1ull);
+  if (slot < cap) put_entry(out, slot, row, col, value, tag);
+}
+
+template <int KIND, typename Entry>
+__global__ void __launch_bounds__(kRingConsumers + 32, 2)
+wb_diff2_ring_kernel(const void* __restrict__ field, unsigned long long rows, unsigned long long cols,
+                     unsigned long long rows_per_unit, Entry* __restrict__ out, unsigned long long cap,
+                     unsigned long long* __restrict__ count, unsigned tag) {
+  constexpr int ES = FieldElem<KIND>::kBytes, NE = RingElems<KIND>::kNE;
+  constexpr unsigned long long W = kRingStripBytes / ES;                  // columns of a strip
+  extern __shared__ __align__(128) char ring_smem_buf[];
+  __shared__ __align__(8) unsigned long long full[kRingStages], empty[kRingStages];
+  if (threadIdx.x == 0) {
+    for (int k = 0; k < kRingStages; ++k) { ring_bar_init(&full[k], 1); ring_bar_init(&empty[k], kRingConsumers / 32); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const unsigned long long strips = (cols + W - 1) / W, row_units = (rows + rows_per_unit - 1) / rows_per_unit;
+  const unsigned long long n_units = strips * row_units;
+  if (threadIdx.x >= kRingConsumers) {
+    // ---- producer: one thread streams the row pieces of this block's units
+    if (threadIdx.x != kRingConsumers) return;
+    unsigned n = 0;
+    for (unsigned long long u = blockIdx.x; u < n_units; u += gridDim.x) {
+      const unsigned long long strip = u % strips, ru = u / strips, c0 = strip * W;
+      const unsigned halo = c0 ? 16u : 0u;                              // the 16 bytes left of the strip
+      const unsigned bytes = (unsigned)((cols - c0 < W ? cols - c0 : W) * ES) + halo;
+      const unsigned long long i_begin = ru * rows_per_unit, i_end = i_begin + rows_per_unit < rows ? i_begin + rows_per_unit : rows;
+      for (unsigned long long r = i_begin >= 2 ? i_begin - 2 : 0; r < i_end; r += kRingRows, ++n) {
+        const unsigned nrow = (unsigned)(i_end - r < (unsigned long long)kRingRows ? i_end - r : kRingRows);
+        const unsigned st = n % kRingStages;
+        if (n >= (unsigned)kRingStages && !ring_bar_wait(&empty[st], ((n / kRingStages) - 1) & 1)) { atomicMax(count, kRingFailed); return; }
+        ring_bar_expect(&full[st], nrow * bytes);
+        for (unsigned k = 0; k < nrow; ++k)
+          ring_bulk_load(ring_smem_buf + (size_t)st * kRingStageBytes + (size_t)k * kRingPitch + 16 - halo,
+                         static_cast<const char*>(field) + ((r + k) * cols + c0) * ES - halo, bytes, &full[st]);
+      }
+    }
+    return;
+  }
+  // ---- consumers
+  const unsigned t = threadIdx.x, lane = t & 31;
+  unsigned n = 0;
+  for (unsigned long long u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const unsigned long long strip = u % strips, ru = u / strips, c0 = strip * W;
+    const unsigned long long wcols = cols - c0 < W ? cols - c0 : W;
+    const unsigned long long i_begin = ru * rows_per_unit, i_end = i_begin + rows_per_unit < rows ? i_begin + rows_per_unit : rows;
+    // window g of a row: g = 0 is the halo left of the strip, g >= 1 the strip's bytes [16 (g-1), 16 g);
+    // warp w takes windows 31 w .. 31 w + 31, its lane 0 sharing a window with the warp before
+    const unsigned g = (t >> 5) * 31 + lane;
+    const bool active = g == 0 ? c0 != 0 : (unsigned long long)(g - 1) * NE < wcols;
+    const unsigned long long j0 = c0 + (unsigned long long)g * NE - NE;   // this thread's first column (lane 0 of warp 0: left of the strip)
+    long long p1[NE], p2[NE];
+#pragma unroll
+    for (int q = 0; q < NE; ++q) p1[q] = p2[q] = 0;
+    for (unsigned long long r = i_begin >= 2 ? i_begin - 2 : 0; r < i_end; r += kRingRows, ++n) {
+      const unsigned nrow = (unsigned)(i_end - r < (unsigned long long)kRingRows ? i_end - r : kRingRows);
+      const unsigned st = n % kRingStages;
+      unsigned ok = 1;
+      if (lane == 0) ok = ring_bar_wait(&full[st], (n / kRingStages) & 1);
+      ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+      if (!ok) { if (t == 0) atomicMax(count, kRingFailed); return; }
+      const char* base = ring_smem_buf + (size_t)st * kRingStageBytes + (size_t)g * 16;
+      for (unsigned k = 0; k < nrow; ++k) {
+        const unsigned long long i = r + k;
+        long long cur[NE], v[NE];
+#pragma unroll
+        for (int q = 0; q < NE; ++q) cur[q] = 0;
+        if (active) ring_unpack<KIND>(*reinterpret_cast<const uint4*>(base + (size_t)k * kRingPitch), cur);
+        bool nz = false;
+#pragma unroll
+        for (int q = 0; q < NE; ++q) {
+          v[q] = cur[q] - 2 * p1[q] + p2[q];
+          nz |= v[q] != 0;
+          p2[q] = p1[q];
+          p1[q] = cur[q];
+        }
+        if (i < i_begin) continue;                                        // the two rows above the unit only prime
+        if (!__any_sync(0xFFFFFFFFu, nz)) continue;
+        // horizontal step: the two values left of this thread's columns come from the lane below, or from
+        // global memory for the first lane of the warp
+        const long long l1 = __shfl_up_sync(0xFFFFFFFFu, v[NE - 1], 1), l2 = __shfl_up_sync(0xFFFFFFFFu, v[NE - 2], 1);
+        if (!active || lane == 0) continue;                               // lane 0 only lends its values to lane 1
+#pragma unroll
+        for (int q = 0; q < NE; ++q) {
+          const long long a1 = q >= 1 ? v[q - 1] : l1, a2 = q >= 2 ? v[q - 2] : (q == 1 ? l1 : l2);
+          const long long d = v[q] - 2 * a1 + a2;
+          if (d != 0) ring_emit(out, cap, count, i, j0 + q, d, tag);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ring_bar_arrive(&empty[st]);
+    }
+  }
+}
+
+// One-row fields: segments of one stage each.
+template <int KIND, typename Entry>
+__global__ void __launch_bounds__(kRingConsumers + 32, 2)
+wb_diff2_ring_row_kernel(const void* __restrict__ field, unsigned long long cols, Entry* __restrict__ out,
+                         unsigned long long cap, unsigned long long* __restrict__ count, unsigned tag) {
+  constexpr int ES = FieldElem<KIND>::kBytes, NE = RingElems<KIND>::kNE;
+  constexpr unsigned long long kSegBytes = (unsigned long long)kRingRows * kRingRowBytes;   // 32 KiB of the row per stage
+  extern __shared__ __align__(128) char ring_smem_buf[];
+  __shared__ __align__(8) unsigned long long full[kRingStages], empty[kRingStages];
+  if (threadIdx.x == 0) {
+    for (int k = 0; k < kRingStages; ++k) { ring_bar_init(&full[k], 1); ring_bar_init(&empty[k], kRingConsumers / 32); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const unsigned long long total = cols * ES, n_seg = (total + kSegBytes - 1) / kSegBytes;
+  if (threadIdx.x >= kRingConsumers) {
+    if (threadIdx.x != kRingConsumers) return;
+    unsigned n = 0;
+    for (unsigned long long sg = blockIdx.x; sg < n_seg; sg += gridDim.x, ++n) {
+      const unsigned long long b0 = sg * kSegBytes;
+      const unsigned bytes = (unsigned)(total - b0 < kSegBytes ? total - b0 : kSegBytes);
+      const unsigned halo = sg ? 16u : 0u;
+      const unsigned st = n % kRingStages;
+      if (n >= (unsigned)kRingStages && !ring_bar_wait(&empty[st], ((n / kRingStages) - 1) & 1)) { atomicMax(count, kRingFailed); return; }
+      ring_bar_expect(&full[st], bytes + halo);
+      // the segment lands 16 bytes into the stage; its left halo, when there is one, right before it
+      ring_bulk_load(ring_smem_buf + (size_t)st * kRingStageBytes + 16 - halo, static_cast<const char*>(field) + b0 - halo,
+                     bytes + halo, &full[st]);
+    }
+    return;
+  }
+  const unsigned t = threadIdx.x, lane = t & 31;
+  unsigned n = 0;
+  for (unsigned long long sg = blockIdx.x; sg < n_seg; sg += gridDim.x, ++n) {
+    const unsigned long long b0 = sg * kSegBytes;
+    const unsigned bytes = (unsigned)(total - b0 < kSegBytes ? total - b0 : kSegBytes);
+    const unsigned st = n % kRingStages;
+    unsigned ok = 1;
+    if (lane == 0) ok = ring_bar_wait(&full[st], (n / kRingStages) & 1);
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    if (!ok) { if (t == 0) atomicMax(count, kRingFailed); return; }
+    const char* data = ring_smem_buf + (size_t)st * kRingStageBytes + 16;
+    for (unsigned off = t * 16; off < bytes; off += kRingConsumers * 16) {
+      long long x[NE], p[NE];
+      ring_unpack<KIND>(*reinterpret_cast<const uint4*>(data + off), x);
+#pragma unroll
+      for (int q = 0; q < NE; ++q) p[q] = 0;
+      if (b0 + off >= 16) ring_unpack<KIND>(*reinterpret_cast<const uint4*>(data + off - 16), p);
+      const unsigned long long j0 = (b0 + off) / ES;
+#pragma unroll
+      for (int q = 0; q < NE; ++q) {
+        const long long a1 = q >= 1 ? x[q - 1] : p[NE - 1], a2 = q >= 2 ? x[q - 2] : p[NE - 2 + q];
+        const long long d = x[q] - 2 * a1 + a2;
+        if (d != 0) ring_emit(out, cap, count, 0, j0 + q, d, tag);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) ring_bar_arrive(&empty[st]);
+  }
+}
+
 // ---- many fields in one launch ---------------------------------------------------------------------
 // A model has thousands of local tensors, most of them small: one launch per tensor is bound by launch
 // latency.  Here the tasks (strip x block of kRowsPerTask rows) of all fields form one list; a warp
@@ -356,6 +596,55 @@ namespace {
 template <typename Entry>
 cudaError_t launch_field(const void* field, uint32_t id_kind, uint64_t rows, uint64_t cols, Entry* out, uint64_t cap,
                          unsigned long long* cnt, unsigned tag, cudaStream_t stream) {
+  // Large fields whose rows start on 16-byte boundaries go through the bulk-copy ring.
+  {
+    const unsigned es = id_kind == WB_ID_I64 ? 8u : (id_kind == WB_ID_F32 ? 4u : 2u);
+    const bool aligned = ((uintptr_t)field & 15u) == 0 && (cols * es) % 16 == 0;
+    if (aligned && rows * cols * es >= (4ull << 20) && (rows == 1 || cols * es >= 2048)) {
+      const size_t dyn = (size_t)kRingStages * kRingStageBytes;
+      const unsigned blocks = 148 * 2;
+      cudaError_t e = cudaSuccess;
+      if (rows == 1) {
+        const unsigned long long n_seg = (cols * es + (unsigned long long)kRingRows * kRingRowBytes - 1) / ((unsigned long long)kRingRows * kRingRowBytes);
+        const unsigned grid = (unsigned)(n_seg < blocks ? n_seg : blocks);
+#define WB_RING_ROW(KIND)                                                                                                 \
+  do {                                                                                                                    \
+    e = cudaFuncSetAttribute(wb_diff2_ring_row_kernel<KIND, Entry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn); \
+    if (e == cudaSuccess) wb_diff2_ring_row_kernel<KIND, Entry><<<grid, kRingConsumers + 32, dyn, stream>>>(field, cols, out, cap, cnt, tag); \
+  } while (0)
+        switch (id_kind) {
+          case WB_ID_I64: WB_RING_ROW(WB_ID_I64); break;
+          case WB_ID_U16: WB_RING_ROW(WB_ID_U16); break;
+          case WB_ID_F32: WB_RING_ROW(WB_ID_F32); break;
+          default: WB_RING_ROW(WB_ID_BF16); break;
+        }
+#undef WB_RING_ROW
+      } else {
+        // units of one strip x rows_per_unit rows, about eight per block; two extra rows per unit prime the
+        // vertical difference
+        const unsigned long long strips = (cols * es + kRingStripBytes - 1) / kRingStripBytes;
+        unsigned long long row_units = (blocks * 8ull + strips - 1) / strips;
+        if (row_units > (rows + 63) / 64) row_units = (rows + 63) / 64;       // at least 64 rows per unit
+        if (row_units < 1) row_units = 1;
+        const unsigned long long rpu = (rows + row_units - 1) / row_units;
+        const unsigned long long n_units = strips * ((rows + rpu - 1) / rpu);
+        const unsigned grid = (unsigned)(n_units < blocks ? n_units : blocks);
+#define WB_RING_2D(KIND)                                                                                                  \
+  do {                                                                                                                    \
+    e = cudaFuncSetAttribute(wb_diff2_ring_kernel<KIND, Entry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);   \
+    if (e == cudaSuccess) wb_diff2_ring_kernel<KIND, Entry><<<grid, kRingConsumers + 32, dyn, stream>>>(field, rows, cols, rpu, out, cap, cnt, tag); \
+  } while (0)
+        switch (id_kind) {
+          case WB_ID_I64: WB_RING_2D(WB_ID_I64); break;
+          case WB_ID_U16: WB_RING_2D(WB_ID_U16); break;
+          case WB_ID_F32: WB_RING_2D(WB_ID_F32); break;
+          default: WB_RING_2D(WB_ID_BF16); break;
+        }
+#undef WB_RING_2D
+      }
+      return e != cudaSuccess ? e : cudaGetLastError();
+    }
+  }
   // Tasks are dealt to warps round robin, so the rows per task are chosen to give every warp the
   // same number of tasks (about kRowsPerTask rows each) instead of leaving a last, partly filled turn.
   const unsigned long long strips = (cols + kStrip - 1) / kStrip;

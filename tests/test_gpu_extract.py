@@ -363,3 +363,51 @@ def test_chunk_passes_on_workload_tensors(name, side):
     for f in sorted(out, key=lambda f: -f.size)[:4]:
         f = np.where(f > (1 << 30), f, 0)                                          # padding stays "no source"
         _check_chunk_passes(f, 8)
+
+
+# ---- the bulk-copy ring kernels (fields of 4 MiB or more whose rows start on 16-byte boundaries) ------------
+def _noisy(a, rng, rows, cols, maxval):
+    """Isolated entries around the seams of the ring kernels: strip edges (3968-byte pieces), the 16-byte windows
+    where one warp's part of a row ends and the next begins (every 496 bytes), unit and band edges."""
+    es = a.dtype.itemsize
+    for byte in (0, 16, 480, 496, 512, 3952, 3968, 3984, 4096, 7936, 32768, 32784):
+        for d in (-2, -1, 0, 1, 2):
+            c = byte // es + d
+            if 0 <= c < a.shape[1]:
+                a[rng.integers(0, a.shape[0]), c] = rng.integers(1, maxval)
+    for r in rows:
+        if 0 <= r < a.shape[0]:
+            a[r, rng.integers(0, a.shape[1])] = rng.integers(1, maxval)
+    for c in cols:
+        if 0 <= c < a.shape[1]:
+            a[rng.integers(0, a.shape[0]), c] = rng.integers(1, maxval)
+    return a
+
+
+@pytest.mark.parametrize("kind,shape", [
+    ("i64", (1, 3_000_000)), ("i64", (1, 600_002)), ("u16", (1, 4_000_000)), ("f32", (1, 2_000_004)),
+    ("i64", (700, 1100)), ("i64", (5000, 498)), ("u16", (600, 4000)), ("u16", (2100, 1984 + 8)), ("bf16", (1200, 2048)),
+    ("f32", (900, 1500)), ("f32", (4100, 512))])
+def test_ring_kernels_match_the_definition(kind, shape):
+    rng = np.random.default_rng(sum(map(ord, kind)) * 1000003 + shape[0] * 7919 + shape[1])
+    maxval = {"i64": 1 << 40, "u16": 1 << 16, "bf16": 256, "f32": 1 << 24}[kind]
+    a = np.zeros(shape, np.int64)
+    for _ in range(6):                                   # a few affine rectangles
+        i0, j0 = rng.integers(0, shape[0]), rng.integers(0, shape[1])
+        ni, nj = rng.integers(1, shape[0] - i0 + 1), rng.integers(1, shape[1] - j0 + 1)
+        base = int(rng.integers(1, maxval // 4))
+        pitch = int(rng.integers(1, max(2, maxval // (4 * max(ni, 1) * 2)))) if shape[0] > 1 else 0
+        a[i0:i0 + ni, j0:j0 + nj] = (base + np.arange(ni)[:, None] * pitch + np.arange(nj)[None, :]) % maxval
+    _noisy(a, rng, rows=(0, 1, 2, 7, 8, 9, 63, 64, 65, 66, shape[0] - 1), cols=(0, 1, shape[1] - 2, shape[1] - 1), maxval=maxval)
+    want = oracle_entries(a)
+    if kind == "i64":
+        t, k = torch.from_numpy(a), wb.WB_ID_I64
+    elif kind == "u16":
+        t, k = torch.from_numpy(a.astype(np.uint16).view(np.int16)), wb.WB_ID_U16
+    elif kind == "bf16":
+        t, k = torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16), wb.WB_ID_BF16
+    else:
+        t, k = torch.from_numpy(a.astype(np.float32)), wb.WB_ID_F32
+    assert t.numel() * t.element_size() >= 4 << 20 and (shape[1] * t.element_size()) % 16 == 0
+    got, n = gpu_entries(t.to(DEV), k, cap=1 << 18)
+    assert n == len(want) and np.array_equal(got, want)
