@@ -323,7 +323,10 @@ def _check_chunk_passes(ids: np.ndarray, b: int):
 @pytest.mark.parametrize("shape,pitch,transposed", [
     ((1, 100003), 0, False), ((1, 1 << 20), 0, False), ((300, 1024), 1024, False), ((300, 1000), 4096, False),
     ((700, 1000), 4099, False), ((700, 1000), 4099, True), ((2, 70001), 70001, False), ((1000, 3), 3, False),
-    ((513, 260), 260, False), ((2048, 2048), 2048, False)])
+    ((513, 260), 260, False), ((2048, 2048), 2048, False),
+    # 4 MiB and more with rows on 16-byte boundaries: the bulk-copy ring kernels
+    ((1, 1 << 22), 0, False), ((1100, 4096), 4096, False), ((1100, 4096), 3 * 8192, False), ((1500, 2048), 4104, False),
+    ((1500, 2048), 4099, True)])
 def test_chunk_pass_matches_the_oracle_on_affine_fields(shape, pitch, transposed, b):
     """One slice-copy rectangle over the whole tensor, ids far enough up that several chunks are in play."""
     i = np.arange(shape[0], dtype=np.int64)[:, None]
