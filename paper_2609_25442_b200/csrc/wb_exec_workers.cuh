@@ -162,9 +162,15 @@ __device__ __forceinline__ void staged_rows(const ChunkDesc& d, const char* stag
   const uint32_t smax = (n + 2 * NV - 2) / NV;     // slots a row can touch
   const uint32_t lead0 = (uint32_t)d.src & 15u, dlead = (uint32_t)d.sps & 15u;
   // the slots of all rows, numbered row by row, are dealt to the threads in order: neighbouring
-  // lanes take neighbouring slots of a row, and no lane idles at the end of a row
-  for (uint32_t idx = t; idx < d.nr * smax; idx += (uint32_t)kWorkers) {
-    const uint32_t r = idx / smax, k = idx - r * smax;
+  // lanes take neighbouring slots of a row, and no lane idles at the end of a row.  A thread's slots are
+  // kWorkers apart; (row, slot in row) advances incrementally, so there is one division per chunk, not per slot
+  const uint32_t dr = (uint32_t)kWorkers / smax, dk = (uint32_t)kWorkers - dr * smax;
+  uint32_t r = t / smax, k = t - r * smax;
+  for (; r < d.nr; r += dr, k += dk) {
+    if (k >= smax) {
+      k -= smax;
+      if (++r >= d.nr) break;
+    }
     const uint64_t D = d.dst + (uint64_t)r * d.dps;
     const uint32_t a = (uint32_t)(D & 15u) / ED;   // elements of slot 0 that precede the row
     const int32_t e0 = (int32_t)(k * NV) - (int32_t)a;
