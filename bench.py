@@ -172,9 +172,7 @@ def oracle_sample(wl, fetch_src, budget_elems=60_000_000):
         for sl in t_s:
             c = int(sl["ckpt"])
             if c not in vals:
-                rng = np.random.default_rng(wl.seed * 1000003 + c)
-                v = rng.standard_normal(wl.ckpt[c].numel, dtype=np.float32) * np.float32(0.02)
-                vals[c] = v.view(np.uint32) if wl.src_dtype == 0 else to_bits_np(torch.from_numpy(v).to(torch.bfloat16))
+                vals[c] = to_bits_np(wl.ckpt_values(c))          # the workload's own seeded generator
             i = np.arange(int(sl["nr"]), dtype=np.int64)[:, None]
             j = np.arange(int(sl["nc"]), dtype=np.int64)[None, :]
             g = (int(sl["r0"]) + i) * int(sl["ckpt_cols"]) + int(sl["c0"]) + j

@@ -482,7 +482,7 @@ wb_status wb_route_account(const wb_plan* plan, const uint32_t* trainer_node, si
 typedef struct { uint64_t row, col; int64_t value; } wb_diff2_entry;
 enum { WB_ID_I64 = 0,   /* field of int64                                              */
        WB_ID_U16 = 1,   /* raw 16-bit patterns (a 16-bit chunk held in a bf16 tensor)   */
-       WB_ID_F32 = 2,   /* fp32 holding an integer value                                 */
+       WB_ID_F32 = 2,   /* fp32 holding an integer value (below 2^24, where fp32 is exact)  */
        WB_ID_BF16 = 3   /* bf16 holding an integer value (8-bit chunks are exact)        */ };
 
 /* wb_diff2_nonzeros (device, asynchronous on cuda_stream): diff2 of the rows x cols row-major

@@ -336,26 +336,37 @@ __device__ __forceinline__ void ring_bulk_load(void* smem_dst, const void* gsrc,
                ::"r"(ring_smem(smem_dst)), "l"(gsrc), "r"(bytes), "r"(ring_smem(bar)) : "memory");
 }
 
-// The 16 bytes a thread owns, as kNE integers.
-template <int KIND> struct RingElems { static constexpr int kNE = 16 / FieldElem<KIND>::kBytes; };
-template <int KIND> __device__ __forceinline__ void ring_unpack(const uint4& w, long long (&x)[RingElems<KIND>::kNE]);
+// The 16 bytes a thread owns, as kNE integers.  Only int64 ids need 64-bit arithmetic: the values of the other
+// kinds are below 2^24, so their second differences (at most 16 times a value) fit 32 bits.
+template <int KIND> struct RingElems {
+  static constexpr int kNE = 16 / FieldElem<KIND>::kBytes;
+  using V = int;
+};
+template <> struct RingElems<WB_ID_I64> {
+  static constexpr int kNE = 2;
+  using V = long long;
+};
+template <int KIND> __device__ __forceinline__ void ring_unpack(const uint4& w, typename RingElems<KIND>::V (&x)[RingElems<KIND>::kNE]);
 template <> __device__ __forceinline__ void ring_unpack<WB_ID_I64>(const uint4& w, long long (&x)[2]) {
   x[0] = (long long)(((unsigned long long)w.y << 32) | w.x);
   x[1] = (long long)(((unsigned long long)w.w << 32) | w.z);
 }
-template <> __device__ __forceinline__ void ring_unpack<WB_ID_F32>(const uint4& w, long long (&x)[4]) {
-  x[0] = __float2ll_rn(__uint_as_float(w.x)); x[1] = __float2ll_rn(__uint_as_float(w.y));
-  x[2] = __float2ll_rn(__uint_as_float(w.z)); x[3] = __float2ll_rn(__uint_as_float(w.w));
+template <> __device__ __forceinline__ void ring_unpack<WB_ID_F32>(const uint4& w, int (&x)[4]) {
+  x[0] = __float2int_rn(__uint_as_float(w.x)); x[1] = __float2int_rn(__uint_as_float(w.y));
+  x[2] = __float2int_rn(__uint_as_float(w.z)); x[3] = __float2int_rn(__uint_as_float(w.w));
 }
-template <> __device__ __forceinline__ void ring_unpack<WB_ID_U16>(const uint4& w, long long (&x)[8]) {
+template <> __device__ __forceinline__ void ring_unpack<WB_ID_U16>(const uint4& w, int (&x)[8]) {
   const unsigned v[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-  for (int p = 0; p < 4; ++p) { x[2 * p] = v[p] & 0xFFFFu; x[2 * p + 1] = v[p] >> 16; }
+  for (int p = 0; p < 4; ++p) { x[2 * p] = (int)(v[p] & 0xFFFFu); x[2 * p + 1] = (int)(v[p] >> 16); }
 }
-template <> __device__ __forceinline__ void ring_unpack<WB_ID_BF16>(const uint4& w, long long (&x)[8]) {
+template <> __device__ __forceinline__ void ring_unpack<WB_ID_BF16>(const uint4& w, int (&x)[8]) {
   const unsigned v[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-  for (int p = 0; p < 4; ++p) { x[2 * p] = bf16_bits_to_ll(v[p] & 0xFFFFu); x[2 * p + 1] = bf16_bits_to_ll(v[p] >> 16); }
+  for (int p = 0; p < 4; ++p) {
+    x[2 * p] = __float2int_rn(__uint_as_float(v[p] << 16));
+    x[2 * p + 1] = __float2int_rn(__uint_as_float(v[p] & 0xFFFF0000u));
+  }
 }
 
 template <typename Entry>
@@ -414,7 +425,8 @@ wb_diff2_ring_kernel(const void* __restrict__ field, unsigned long long rows, un
     const unsigned g = (t >> 5) * 31 + lane;
     const bool active = g == 0 ? c0 != 0 : (unsigned long long)(g - 1) * NE < wcols;
     const unsigned long long j0 = c0 + (unsigned long long)g * NE - NE;   // this thread's first column (lane 0 of warp 0: left of the strip)
-    long long p1[NE], p2[NE];
+    using V = typename RingElems<KIND>::V;
+    V p1[NE], p2[NE];
 #pragma unroll
     for (int q = 0; q < NE; ++q) p1[q] = p2[q] = 0;
     for (unsigned long long r = i_begin >= 2 ? i_begin - 2 : 0; r < i_end; r += kRingRows, ++n) {
@@ -427,7 +439,7 @@ wb_diff2_ring_kernel(const void* __restrict__ field, unsigned long long rows, un
       const char* base = ring_smem_buf + (size_t)st * kRingStageBytes + (size_t)g * 16;
       for (unsigned k = 0; k < nrow; ++k) {
         const unsigned long long i = r + k;
-        long long cur[NE], v[NE];
+        V cur[NE], v[NE];
 #pragma unroll
         for (int q = 0; q < NE; ++q) cur[q] = 0;
         if (active) ring_unpack<KIND>(*reinterpret_cast<const uint4*>(base + (size_t)k * kRingPitch), cur);
@@ -443,13 +455,13 @@ wb_diff2_ring_kernel(const void* __restrict__ field, unsigned long long rows, un
         if (!__any_sync(0xFFFFFFFFu, nz)) continue;
         // horizontal step: the two values left of this thread's columns come from the lane below, or from
         // global memory for the first lane of the warp
-        const long long l1 = __shfl_up_sync(0xFFFFFFFFu, v[NE - 1], 1), l2 = __shfl_up_sync(0xFFFFFFFFu, v[NE - 2], 1);
+        const V l1 = __shfl_up_sync(0xFFFFFFFFu, v[NE - 1], 1), l2 = __shfl_up_sync(0xFFFFFFFFu, v[NE - 2], 1);
         if (!active || lane == 0) continue;                               // lane 0 only lends its values to lane 1
 #pragma unroll
         for (int q = 0; q < NE; ++q) {
-          const long long a1 = q >= 1 ? v[q - 1] : l1, a2 = q >= 2 ? v[q - 2] : (q == 1 ? l1 : l2);
-          const long long d = v[q] - 2 * a1 + a2;
-          if (d != 0) ring_emit(out, cap, count, i, j0 + q, d, tag);
+          const V a1 = q >= 1 ? v[q - 1] : l1, a2 = q >= 2 ? v[q - 2] : (q == 1 ? l1 : l2);
+          const V d = v[q] - 2 * a1 + a2;
+          if (d != 0) ring_emit(out, cap, count, i, j0 + q, (long long)d, tag);
         }
       }
       __syncwarp();
@@ -501,7 +513,8 @@ wb_diff2_ring_row_kernel(const void* __restrict__ field, unsigned long long cols
     if (!ok) { if (t == 0) atomicMax(count, kRingFailed); return; }
     const char* data = ring_smem_buf + (size_t)st * kRingStageBytes + 16;
     for (unsigned off = t * 16; off < bytes; off += kRingConsumers * 16) {
-      long long x[NE], p[NE];
+      using V = typename RingElems<KIND>::V;
+      V x[NE], p[NE];
       ring_unpack<KIND>(*reinterpret_cast<const uint4*>(data + off), x);
 #pragma unroll
       for (int q = 0; q < NE; ++q) p[q] = 0;
@@ -509,9 +522,9 @@ wb_diff2_ring_row_kernel(const void* __restrict__ field, unsigned long long cols
       const unsigned long long j0 = (b0 + off) / ES;
 #pragma unroll
       for (int q = 0; q < NE; ++q) {
-        const long long a1 = q >= 1 ? x[q - 1] : p[NE - 1], a2 = q >= 2 ? x[q - 2] : p[NE - 2 + q];
-        const long long d = x[q] - 2 * a1 + a2;
-        if (d != 0) ring_emit(out, cap, count, 0, j0 + q, d, tag);
+        const V a1 = q >= 1 ? x[q - 1] : p[NE - 1], a2 = q >= 2 ? x[q - 2] : p[NE - 2 + q];
+        const V d = x[q] - 2 * a1 + a2;
+        if (d != 0) ring_emit(out, cap, count, 0, j0 + q, (long long)d, tag);
       }
     }
     __syncwarp();
