@@ -1124,7 +1124,7 @@ extern "C" wb_status wb_diff2_chunk_pass(const void* field, uint32_t id_kind, ui
     if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
     ci.first = first; ci.has = has; ci.rec = sorted;
     ci.s = s_in; ci.cols = cols; ci.use_up = s_in < rows;
-    ci.s_shift = chunk_bits * pass;
+    ci.s_shift = chunk_bits * pass < 62u ? chunk_bits * pass : 62u;      // matches carry_stride
   } else if (mode == 2) {
     if (cudaMemsetAsync(carry, 0, n16, stream) != cudaSuccess) return WB_ERR_CUDA;
     const unsigned g = (unsigned)((n_carry_in + 255) / 256 < kCarryBlocks ? (n_carry_in + 255) / 256 : kCarryBlocks);
