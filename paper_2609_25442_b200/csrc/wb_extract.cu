@@ -966,7 +966,7 @@ wb_chunk_pass8_kernel(const void* __restrict__ field, unsigned long long rows, u
       for (unsigned long long x = x0; x < n; ++x) chunk_elem<KIND>(field, cols, b, mode, ci, carry, x, out, cap, count);
       continue;
     }
-    const unsigned long long i = x0 / cols, j0 = x0 - i * cols;
+    const unsigned long long i = rows == 1 ? 0ull : x0 / cols, j0 = x0 - i * cols;
     int v[8], l[2] = {0, 0};                                    // vertical second differences; l = columns j0-2, j0-1
     load8<KIND>(field, x0, v);
     if (j0) { l[0] = (int)field_at<KIND>(field, x0 - 2); l[1] = (int)field_at<KIND>(field, x0 - 1); }
@@ -1026,38 +1026,109 @@ wb_chunk_pass8_kernel(const void* __restrict__ field, unsigned long long rows, u
   }
 }
 
-// NonZeros(StridedDiff1(C)) for the carry field C (one byte per element, padded to a multiple of 16 bytes):
-// a thread takes eight adjacent elements; s and s cols are multiples of 8, so the neighbours are aligned words.
-__device__ __forceinline__ void sub8(int (&g)[8], uint2 w, int sign) {
+// One-row fields (flat shards): a thread takes sixteen adjacent elements, two 16-byte-per-eight loads in flight
+// plus the two elements before them, and stores the sixteen carries as one 16-byte word.
+template <int KIND>
+__global__ void __launch_bounds__(256)
+wb_chunk_row16_kernel(const void* __restrict__ field, unsigned long long n, unsigned b, int mode, CarryIndex ci,
+                      signed char* __restrict__ carry, wb_diff2_entry* __restrict__ out, unsigned long long cap,
+                      unsigned long long* __restrict__ count) {
+  const unsigned long long n16 = (n + 15) / 16;
+  const int half = 1 << (b - 1), mask = (1 << b) - 1;
+  for (unsigned long long q = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; q < n16;
+       q += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long x0 = q * 16;
+    if (x0 + 16 > n) {                                          // ragged end
+      for (unsigned long long x = x0; x < n; ++x) chunk_elem<KIND>(field, n, b, mode, ci, carry, x, out, cap, count);
+      continue;
+    }
+    int v[18];                                                  // v[0], v[1]: the two elements before the group
+    load8<KIND>(field, x0, reinterpret_cast<int(&)[8]>(v[2]));
+    load8<KIND>(field, x0 + 8, reinterpret_cast<int(&)[8]>(v[10]));
+    v[0] = v[1] = 0;
+    if (x0) { v[0] = (int)field_at<KIND>(field, x0 - 2); v[1] = (int)field_at<KIND>(field, x0 - 1); }
+    int d[16];
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    g[k] += sign * (signed char)((w.x >> (8 * k)) & 0xFF);
-    g[4 + k] += sign * (signed char)((w.y >> (8 * k)) & 0xFF);
+    for (int k = 0; k < 16; ++k) d[k] = v[k + 2] - 2 * v[k + 1] + v[k];
+    if (mode == 1) {
+      const unsigned bits = (unsigned)__ldg(ci.has + ((x0 >> 3) & 31u)) | ((unsigned)__ldg(ci.has + (((x0 >> 3) + 1) & 31u)) << 8);
+      if (bits) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k)
+          if (bits >> k & 1u) d[k] += gamma_at(ci, x0 + k);
+      }
+    } else if (mode == 2) {
+      const uint4 g = *reinterpret_cast<const uint4*>(carry + x0);
+      const unsigned w[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+      for (int k = 0; k < 16; ++k) d[k] += (signed char)((w[k >> 2] >> (8 * (k & 3))) & 0xFF);
+    }
+    unsigned c[4] = {0, 0, 0, 0};
+    unsigned nzmask = 0;
+    int z[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      z[k] = ((d[k] + half) & mask) - half;
+      c[k >> 2] |= ((unsigned)((d[k] - z[k]) >> b) & 0xFFu) << (8 * (k & 3));
+      nzmask |= (unsigned)(z[k] != 0) << k;
+    }
+    *reinterpret_cast<uint4*>(carry + x0) = make_uint4(c[0], c[1], c[2], c[3]);
+    if (nzmask) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+        if (nzmask >> k & 1u) {
+          const unsigned long long slot = atomicAdd(count, 1ull);
+          if (slot < cap) out[slot] = wb_diff2_entry{0, x0 + k, (long long)z[k]};
+        }
+    }
   }
+}
+
+// NonZeros(StridedDiff1(C)) for the carry field C (one byte per element, padded to a multiple of 16 bytes):
+// a thread takes sixteen adjacent elements, two such groups per step; s and s cols are multiples of 16, so the
+// neighbours are aligned 16-byte words.
+__device__ __forceinline__ void sub16(int (&g)[16], uint4 w, int sign) {
+  const unsigned v[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int p = 0; p < 4; ++p)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) g[4 * p + k] += sign * (signed char)((v[p] >> (8 * k)) & 0xFF);
 }
 __global__ void __launch_bounds__(256)
 wb_strided_diff_kernel(const signed char* __restrict__ c, unsigned long long n, unsigned long long cols,
                        unsigned long long s, unsigned long long up, int use_s, int use_up,
                        wb_diff2_entry* __restrict__ out, unsigned long long cap, unsigned long long* __restrict__ count) {
-  const unsigned long long n8 = (n + 7) / 8;
-  for (unsigned long long q = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; q < n8;
-       q += (unsigned long long)gridDim.x * blockDim.x) {
-    const unsigned long long x0 = q * 8;
-    int g[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    sub8(g, *reinterpret_cast<const uint2*>(c + x0), 1);
-    if (use_s && x0 >= s) sub8(g, *reinterpret_cast<const uint2*>(c + x0 - s), -1);
-    if (use_up && x0 >= up) sub8(g, *reinterpret_cast<const uint2*>(c + x0 - up), -1);
-    if (use_s && use_up && x0 >= s + up) sub8(g, *reinterpret_cast<const uint2*>(c + x0 - s - up), 1);
-    bool any = false;
+  const unsigned long long n16 = (n + 15) / 16, stride = (unsigned long long)gridDim.x * blockDim.x;
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  for (unsigned long long q0 = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; q0 < n16; q0 += 2 * stride) {
+    uint4 w[2][4];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) any |= g[k] != 0 && x0 + k < n;
-    if (!any) continue;
+    for (int u = 0; u < 2; ++u) {
+      const unsigned long long q = q0 + u * stride, x0 = q * 16;
+      const bool in = q < n16;
+      w[u][0] = in ? *reinterpret_cast<const uint4*>(c + x0) : zero;
+      w[u][1] = in && use_s && x0 >= s ? *reinterpret_cast<const uint4*>(c + x0 - s) : zero;
+      w[u][2] = in && use_up && x0 >= up ? *reinterpret_cast<const uint4*>(c + x0 - up) : zero;
+      w[u][3] = in && use_s && use_up && x0 >= s + up ? *reinterpret_cast<const uint4*>(c + x0 - s - up) : zero;
+    }
 #pragma unroll
-    for (int k = 0; k < 8; ++k)
-      if (g[k] != 0 && x0 + k < n) {
-        const unsigned long long slot = atomicAdd(count, 1ull);
-        if (slot < cap) out[slot] = wb_diff2_entry{(x0 + k) / cols, (x0 + k) % cols, (long long)g[k]};
-      }
+    for (int u = 0; u < 2; ++u) {
+      const unsigned long long x0 = (q0 + u * stride) * 16;
+      // all four words zero: nothing to do (almost every group)
+      const unsigned any = w[u][0].x | w[u][0].y | w[u][0].z | w[u][0].w | w[u][1].x | w[u][1].y | w[u][1].z | w[u][1].w |
+                           w[u][2].x | w[u][2].y | w[u][2].z | w[u][2].w | w[u][3].x | w[u][3].y | w[u][3].z | w[u][3].w;
+      if (!any) continue;
+      int g[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) g[k] = 0;
+      sub16(g, w[u][0], 1); sub16(g, w[u][1], -1); sub16(g, w[u][2], -1); sub16(g, w[u][3], 1);
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+        if (g[k] != 0 && x0 + k < n) {
+          const unsigned long long slot = atomicAdd(count, 1ull);
+          if (slot < cap) out[slot] = wb_diff2_entry{(x0 + k) / cols, (x0 + k) % cols, (long long)g[k]};
+        }
+    }
   }
 }
 
@@ -1134,11 +1205,12 @@ extern "C" wb_status wb_diff2_chunk_pass(const void* field, uint32_t id_kind, ui
     if (s_in < rows && strided_prefix(carry, n16, s_in * cols, part, stream) != cudaSuccess) return WB_ERR_CUDA;
   }
   const bool vec = ((uintptr_t)field % 16u) == 0 && (rows == 1 || cols % 8 == 0);
-  const unsigned long long work = vec ? (n + 7) / 8 : n;
+  const unsigned long long work = vec ? (rows == 1 ? (n + 15) / 16 : (n + 7) / 8) : n;
   const unsigned grid = (unsigned)((work + 255) / 256 < kCarryBlocks ? (work + 255) / 256 : kCarryBlocks);
 #define WB_CHUNK_LAUNCH(KIND)                                                                                        \
   do {                                                                                                               \
-    if (vec) wb_chunk_pass8_kernel<KIND><<<grid, 256, 0, stream>>>(field, rows, cols, chunk_bits, mode, ci, carry, z_out, z_cap, zc); \
+    if (vec && rows == 1) wb_chunk_row16_kernel<KIND><<<grid, 256, 0, stream>>>(field, n, chunk_bits, mode, ci, carry, z_out, z_cap, zc); \
+    else if (vec) wb_chunk_pass8_kernel<KIND><<<grid, 256, 0, stream>>>(field, rows, cols, chunk_bits, mode, ci, carry, z_out, z_cap, zc); \
     else wb_chunk_pass_kernel<KIND><<<grid, 256, 0, stream>>>(field, rows, cols, chunk_bits, mode, ci, carry, z_out, z_cap, zc);      \
   } while (0)
   switch (id_kind) {
@@ -1150,7 +1222,8 @@ extern "C" wb_status wb_diff2_chunk_pass(const void* field, uint32_t id_kind, ui
 #undef WB_CHUNK_LAUNCH
   if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
   const unsigned long long s_out = carry_stride(chunk_bits, pass);
-  const unsigned grid8 = (unsigned)(((n + 7) / 8 + 255) / 256 < kCarryBlocks ? ((n + 7) / 8 + 255) / 256 : kCarryBlocks);
+  const unsigned long long sd_blocks = ((n + 15) / 16 + 511) / 512;             // two groups of 16 per thread and step
+  const unsigned grid8 = (unsigned)(sd_blocks < kCarryBlocks ? (sd_blocks ? sd_blocks : 1) : kCarryBlocks);
   wb_strided_diff_kernel<<<grid8, 256, 0, stream>>>(carry, n, cols, s_out, s_out < rows ? s_out * cols : 0, s_out < n,
                                                    s_out < rows, carry_out, carry_cap, cc);
   return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
