@@ -256,3 +256,19 @@ def test_entries_shipped_per_pass_stay_bounded_where_plain_chunk_diffs_do_not():
             assert shipped <= 32 * n_ops, (k, shipped)
         if field.shape[0] == 1:                   # (rows 4096 ids apart repeat their wrap pattern: those cancel vertically)
             assert np.count_nonzero(diff2(id_chunk(field, 0, 8))) >= n // 256
+
+
+def test_chunk_pass_entry_point_checks_its_arguments_on_the_host():
+    """Bad arguments are refused before anything is launched (no GPU needed to see them)."""
+    nb = wb.wb_diff2_chunk_scratch_bytes(4, 4)
+    assert nb >= 16 + (1 << 18)
+    ok = dict(field_ptr=4096, id_kind=wb.WB_ID_U16, rows=4, cols=4, chunk_bits=8, pass_index=0, carry_in_ptr=0, n_carry_in=0,
+              scratch_ptr=8192, scratch_bytes=nb, z_out_ptr=4096, z_cap=1, z_count_ptr=4096, carry_out_ptr=4096, carry_cap=1,
+              carry_count_ptr=4096)
+    for bad in (dict(field_ptr=0), dict(id_kind=9), dict(chunk_bits=12), dict(pass_index=8), dict(scratch_ptr=8200),
+                dict(scratch_bytes=nb - 1), dict(n_carry_in=3), dict(pass_index=1, n_carry_in=3), dict(z_count_ptr=0),
+                dict(rows=1 << 31, cols=2)):
+        with pytest.raises(wb.WbError) as e:
+            wb.wb_diff2_chunk_pass(**{**ok, **bad})
+        assert e.value.name == "WB_ERR_INVALID_ARG", bad
+    wb.wb_diff2_chunk_pass(**{**ok, "rows": 0})          # an empty field: nothing to do

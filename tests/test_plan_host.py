@@ -292,6 +292,25 @@ def test_error_bucket_too_small_and_unbound_execution():
     _expect("WB_ERR_NOT_BOUND", lambda: plan.transfer_rounds_fp8(256, 512, 1024, 2048, 4096))
     _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds_fp8(256, 256, 1024, 2048, 4096))
     _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds_fp8(256, 512, 1024, 2050, 4096))
+    # the fused forms and the rank subsets likewise
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.pack_fp8(0, 256, 1024))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.pack_fp8(0, 258, 1024))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.unpack_fp8(99, 256, 1024))
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.transfer_rounds_fp8_fused(256, 512, 1024))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.transfer_rounds_fp8_fused(256, 256, 1024))
+    _expect("WB_ERR_NOT_BOUND", lambda: plan.pack_ranks(0, [0], 256))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.pack_ranks(0, [0], 258))
+    _expect("WB_ERR_INVALID_ARG", lambda: plan.unpack_ranks(99, [0], 256))
+    nt, nr = plan.num_ranks()
+    assert (nt, nr) == (4, 1)                                  # TP2 x FSDP2 trainer ranks, one rollout rank
+    regions = plan.bucket_regions(0)
+    assert sorted((int(g["receiver"]), int(g["sender"])) for g in regions) == [(0, s) for s in range(4)]
+    assert all(int(g["off"]) % 256 == 0 for g in regions) and int(regions["bytes"].sum()) <= plan.bucket_bytes(0)
+    entries = plan.bucket_entries(0)
+    for e in entries:                                          # every payload lies in the region of its pair
+        g = regions[(regions["receiver"] == e["receiver"]) & (regions["sender"] == e["sender"])][0]
+        size = int(e["nr"]) * int(e["nc"]) * 2
+        assert int(g["off"]) <= int(e["bucket_off"]) and int(e["bucket_off"]) + size <= int(g["off"]) + int(g["bytes"])
     _expect("WB_ERR_INVALID_ARG", lambda: plan.bind([0] * plan.n_src, [0] * plan.n_dst))
     lib = wb.load()
     assert lib.wb_remap(None, None) == 1
