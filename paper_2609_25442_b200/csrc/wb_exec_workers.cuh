@@ -376,17 +376,17 @@ __device__ __forceinline__ void warp_transpose(const TileFields& f, char* patch,
 }
 
 // Workers: ROWS tile with short rows (dst[i*dsr + j] = cast(src[i*ssr + j]), nc small).  The tile is
-// a flat sequence of nr*nc elements; every warp takes batches of 256 consecutive elements on its
+// a flat sequence of nr*nc elements; every warp takes batches of 384 consecutive elements on its
 // own.  Lane l loads elements l, l+32, ... of the batch (coalesced inside each row; row and column
-// advance incrementally, no division per element), eight loads in flight, one batch ahead.  If the
-// destination rows are contiguous (dsr == nc) the cast values go through a 512-byte private patch
+// advance incrementally, no division per element), twelve loads in flight, one batch ahead.  If the
+// destination rows are contiguous (dsr == nc) the cast values go through a private patch of a batch
 // and leave as 16-byte vectors; otherwise each value is stored to its own row.
 template <int ES, int ED>
 __device__ __forceinline__ void warp_small_rows(const TileFields& f, char* patch_mem, uint32_t warp, uint32_t nw,
                                                 uint32_t lane) {
   using E = Elem<ES, ED>;
   constexpr uint32_t NV = 16 / ED;
-  constexpr int U = 8;
+  constexpr int U = 12;          // loads in flight per lane (16 spills registers; 8 leaves rows of 520 B 10 % slower)
   constexpr uint32_t B = 32 * U;
   const uint32_t nc = f.nc, cnt = f.nr * f.nc;
   const bool packed = f.dsr == nc;
