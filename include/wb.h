@@ -107,6 +107,10 @@ typedef struct {
 #define WB_PLAN_STATIC_SCHEDULE 2u  /* every thread block walks the fixed, byte-balanced tile
                                        range the planner gave it, instead of drawing batches
                                        of tiles from a shared counter at run time          */
+#define WB_PLAN_NO_TENSOR_MAPS 4u   /* wb_plan_bind builds no tensor maps: wb_remap stages the
+                                       source rows of transposing tiles with per-lane copies
+                                       (as wb_unpack and wb_remap_static always do) instead
+                                       of tensor-map (TMA) loads                           */
 
 typedef struct {
   uint64_t n_ckpt_tensors;      /* checkpoint tensors the destination consumes              */

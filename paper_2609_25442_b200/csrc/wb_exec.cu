@@ -29,6 +29,7 @@
 // Files: wb_exec_prims.cuh (access, cast, mbarrier and copy primitives), wb_exec_workers.cuh (rings,
 // slot descriptors, worker routines), wb_exec_kernel.cuh (the kernel), this file (launch, binding
 // and the extern "C" entry points).
+#include <cuda.h>            // CUtensorMap and its enums only: the encoder is looked up at run time
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -67,7 +68,7 @@ cudaError_t launch_one(const wb_plan* plan, const TileTable& T, uint64_t src_add
   }
   wb_exec_kernel<ES, ED><<<dim3(plan->grid), dim3(kThreads), Rings<ES, ED>::kDyn, stream>>>(
       T.d_tiles + tile_off, T.d_cta_begin, T.d_extras, src_add, dst_add, plan->d_err, tile_count,
-      (whole && (plan->opts.flags & WB_PLAN_STATIC_SCHEDULE)) ? nullptr : T.d_sched);
+      (whole && (plan->opts.flags & WB_PLAN_STATIC_SCHEDULE)) ? nullptr : T.d_sched, T.d_maps);
   return cudaGetLastError();
 }
 
@@ -90,6 +91,60 @@ wb_status launch_table(const wb_plan* plan, const TileTable& T, uint64_t src_add
 
 inline uint32_t esize(uint32_t dt) { return dt == WB_F32 ? 4u : 2u; }
 inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+// ---------------------------------------------------------------------------------------------
+// tensor maps of the staged transposition (see kTmaClasses)
+// ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+// The driver's encoder, through the runtime (the library does not link the driver); null if this
+// driver has none, and the tables then keep the per-lane copies.
+EncodeTiledFn tensor_map_encoder() {
+  static std::atomic<EncodeTiledFn> cached{nullptr};
+  static std::atomic<bool> looked{false};
+  if (!looked.load(std::memory_order_acquire)) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult res = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess ||
+        res != cudaDriverEntryPointSuccess)
+      fn = nullptr;
+    (void)cudaGetLastError();
+    cached.store(reinterpret_cast<EncodeTiledFn>(fn), std::memory_order_release);
+    looked.store(true, std::memory_order_release);
+  }
+  return cached.load(std::memory_order_acquire);
+}
+
+// limits of a tensor map: pitches below 2^40 bytes, extents up to 2^32 elements (any tile meets the second)
+bool pitch_ok(const HTile& h, uint32_t es) { return (uint64_t)h.ssr * es * kTmaClasses < (1ull << 40); }
+
+// Does tile h of a table whose source elements have `es` bytes (destination `ed`) get tensor maps?
+bool tile_wants_maps(const HTile& h, uint32_t es) {
+  if (h.src_tensor < 0) return false;       // the bucket's address is only known at launch
+  return es == 4 ? staged_trans_ok<4>(h.kind, h.n_extra, h.nr, h.nc) : staged_trans_ok<2>(h.kind, h.n_extra, h.nr, h.nc);
+}
+
+// The kTmaClasses maps of one tile: class q covers tile rows q, q + 8, ...; its base is the 16-byte
+// boundary at or before the first element of row q, its rows are 8 tile pitches apart, and its width is
+// the 16-byte aligned superset of a tile row, so a load never touches memory outside the supersets
+// of the tile's rows (coordinates beyond read as zero).
+template <int ES, int ED>
+bool encode_tile_maps(EncodeTiledFn encode, uint64_t tile_src, const HTile& h, CUtensorMap* out) {
+  const uint64_t pitch = (uint64_t)h.ssr * ES;
+  for (uint32_t q = 0; q < kTmaClasses; ++q) {
+    const uint64_t a = tile_src + q * pitch, lead = a & 15u;
+    cuuint64_t dims[2] = {(lead + (uint64_t)h.nc * ES + 15) / 16 * 16 / ES, (h.nr - q + kTmaClasses - 1) / kTmaClasses};
+    cuuint64_t strides[1] = {pitch * kTmaClasses};
+    cuuint32_t box[2] = {kTmaInner / ES, TransGeom<ES, ED>::kBoxRows};
+    cuuint32_t estr[2] = {1, 1};
+    if (encode(&out[q], ES == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 2,
+               reinterpret_cast<void*>(a - lead), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  return true;
+}
 
 }  // namespace
 
@@ -131,10 +186,18 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
     // lay every table out in one arena
     std::vector<TileTable*> tabs{&plan->remap};
     for (Round& R : plan->rounds) { tabs.push_back(&R.pack); tabs.push_back(&R.unpack); }
+    // tensor maps: the transposing tiles of the fused remap table whose rows get staged (the source
+    // of an unpack table is the bucket, whose address arrives with the launch)
+    EncodeTiledFn encode = (plan->opts.flags & WB_PLAN_NO_TENSOR_MAPS) ? nullptr : tensor_map_encoder();
+    size_t n_map_tiles = 0;
+    if (encode)
+      for (const HTile& h : plan->remap.tiles) n_map_tiles += tile_wants_maps(h, es) && pitch_ok(h, es);
     size_t bytes = 0;
     for (TileTable* T : tabs)
       bytes += up256(T->tiles.size() * sizeof(DTile)) + up256(T->extras.size() * sizeof(DDst)) +
                up256(T->cta_begin.size() * sizeof(uint32_t)) + 256;
+    const size_t maps_off = up256(bytes);
+    bytes = maps_off + n_map_tiles * kTmaClasses * sizeof(CUtensorMap);
     const size_t err_off = up256(bytes);
     const size_t cmp_off = err_off + 256;
     bytes = up256(cmp_off + plan->replica_pairs.size() * sizeof(DCompare) + 256);
@@ -175,7 +238,9 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
                       : (uint64_t)(uintptr_t)plan->dst_base[tensor] + elem_off * ed;
       };
       T->d_tiles = reinterpret_cast<DTile*>(dbase + off);
+      T->d_maps = nullptr;
       DTile* ht = reinterpret_cast<DTile*>(host.data() + off);
+      size_t n_maps = 0;       // maps of this table written so far
       for (size_t k = 0; k < T->tiles.size(); ++k) {
         const HTile& h = T->tiles[k];
         DTile dt{};
@@ -184,8 +249,19 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
         dt.nr = h.nr; dt.nc = h.nc; dt.ssr = h.ssr; dt.ssc = h.ssc; dt.dsr = h.dsr; dt.dsc = h.dsc;
         dt.kind_extra = h.kind | (h.n_extra << 8);
         dt.extra = h.extra;
+        if (ti == 0 && encode && tile_wants_maps(h, es) && pitch_ok(h, es)) {
+          CUtensorMap* hm = reinterpret_cast<CUtensorMap*>(host.data() + maps_off) + n_maps;
+          const bool ok = es == 4 ? (ed == 4 ? encode_tile_maps<4, 4>(encode, dt.src, h, hm) : encode_tile_maps<4, 2>(encode, dt.src, h, hm))
+                                  : (ed == 4 ? encode_tile_maps<2, 4>(encode, dt.src, h, hm) : encode_tile_maps<2, 2>(encode, dt.src, h, hm));
+          if (ok) {                           // a refused map leaves the tile on the per-lane copies
+            dt.kind_extra |= kTileHasMaps;
+            dt.extra = (uint32_t)n_maps;
+            n_maps += kTmaClasses;
+          }
+        }
         ht[k] = dt;
       }
+      if (ti == 0 && n_maps) T->d_maps = dbase + maps_off;
       off += up256(T->tiles.size() * sizeof(DTile));
       T->d_extras = reinterpret_cast<DDst*>(dbase + off);
       DDst* hx = reinterpret_cast<DDst*>(host.data() + off);
@@ -632,10 +708,10 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
   uint32_t* d_sched = (plan->opts.flags & WB_PLAN_STATIC_SCHEDULE) ? nullptr : reinterpret_cast<uint32_t*>(dbase + 64);
   const uint32_t n_tiles = (uint32_t)T.tiles.size();
   const dim3 grid(plan->grid), block(kThreads);
-  if (es == 2 && ed == 2) wb_exec_kernel<2, 2><<<grid, block, Rings<2, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
-  else if (es == 4 && ed == 4) wb_exec_kernel<4, 4><<<grid, block, Rings<4, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
-  else if (es == 4 && ed == 2) wb_exec_kernel<4, 2><<<grid, block, Rings<4, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
-  else wb_exec_kernel<2, 4><<<grid, block, Rings<2, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched);
+  if (es == 2 && ed == 2) wb_exec_kernel<2, 2><<<grid, block, Rings<2, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched, nullptr);
+  else if (es == 4 && ed == 4) wb_exec_kernel<4, 4><<<grid, block, Rings<4, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched, nullptr);
+  else if (es == 4 && ed == 2) wb_exec_kernel<4, 2><<<grid, block, Rings<4, 2>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched, nullptr);
+  else wb_exec_kernel<2, 4><<<grid, block, Rings<2, 4>::kDyn, stream>>>(d_tiles, d_begin, d_extras, 0, 0, d_err, n_tiles, d_sched, nullptr);
   if (cudaGetLastError() != cudaSuccess) return WB_ERR_CUDA;
   if (flags & WB_STATIC_SYNC_CHECK) {
     uint32_t err = 0;
@@ -645,3 +721,4 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
   }
   return WB_OK;
 }
+

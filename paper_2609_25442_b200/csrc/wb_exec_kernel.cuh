@@ -7,7 +7,9 @@ namespace {
 //   warp 0   "producer".  Lane 0 moves direct tiles by itself through a ring of bulk (TMA) copies
 //            global -> shared -> global.  For every other tile the warp feeds the worker ring:
 //            either the tile's rows are staged into a ring slot with bulk loads (one per row, the
-//            16-byte aligned superset of the row), or the tile index is queued as is.
+//            16-byte aligned superset of the row; transposing tiles: eight tensor-map loads per chunk,
+//            or per-lane asynchronous copies where the table has no tensor maps), or the tile index
+//            is queued as is.
 //   warps 1.. "workers".  Take ring slots in order: convert staged rows (cast in registers,
 //            realignment by funnel shifts, 16-byte vector stores), transpose staged blocks, or
 //            run a queued tile cooperatively (element-wise fan-out and other rare shapes).
@@ -15,8 +17,9 @@ template <int ES, int ED>
 __global__ void __launch_bounds__(kThreads, 1)
 wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta_begin,
                const DDst* __restrict__ extras, uint64_t src_add, uint64_t dst_add, uint32_t* __restrict__ err,
-               uint32_t n_tiles, uint32_t* __restrict__ sched) {
+               uint32_t n_tiles, uint32_t* __restrict__ sched, const char* __restrict__ tmaps) {
   using E = Elem<ES, ED>;
+  using TG = TransGeom<ES, ED>;
   extern __shared__ __align__(128) char dyn_smem[];
   constexpr int kSlots = Rings<ES, ED>::kSlots;
   constexpr int kSlotBytes = Rings<ES, ED>::kSlotBytes;
@@ -25,6 +28,7 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
   __shared__ __align__(8) uint64_t direct_full[kDirectStages];
   __shared__ __align__(8) uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots];
   __shared__ __align__(16) ChunkDesc desc[kMaxSlots];
+  __shared__ __align__(16) uint32_t trans_tab[kMaxSlots][kTmaClasses * (16 / ED)];   // see staged_trans (tensor-map chunks)
   __shared__ char* q_dst[kDirectStages];        // direct ring: where each loaded stage goes
   __shared__ uint32_t q_bytes[kDirectStages];
 
@@ -59,6 +63,8 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
         staged_rows<ES, ED>(d, stage, tr);
       } else if (d.mode == MODE_TRANS) {
         staged_trans<ES, ED>(d, stage, tr);
+      } else if (d.mode == MODE_TRANS_TMA) {
+        staged_trans_tma<ES, ED>(d, stage, tr, smem_u32(trans_tab[slot]));
       } else {
         // queued tiles: one big tile shared by all worker warps, or a run of small tiles with one
         // warp per tile
@@ -175,6 +181,43 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     if (lane == 0) mbar_arrive(&slot_full[slot]);   // after every lane's pending arrival is counted
     ++n_w;
   };
+  // the same chunk by tensor-map loads: lane q fetches the box of row class q (rows q, q + 8, ... of the
+  // chunk; `tile_src` is the tile's first element, (i0, j0) the chunk's position in the tile)
+  auto push_trans_tma = [&](uint32_t map0, const char* tile_src, uint32_t i0, uint32_t j0, char* dst, uint32_t R,
+                            uint32_t n, uint64_t sps, uint64_t dps, uint32_t own, uint32_t first) {
+    if (!acquire_slot()) return;
+    const uint32_t slot = n_w % kSlots;
+    char* stage = wring + (size_t)slot * kSlotBytes;
+    {
+      // where the rows of a destination window are in the slot: entry (h, k) is the offset of row
+      // e0 + k relative to the box row of e0, for a window whose first row e0 has class h
+      constexpr uint32_t NV = 16 / ED;
+      const uint32_t lead0 = (uint32_t)(((uintptr_t)tile_src + (uint64_t)j0 * ES) & 15u), dlead = (uint32_t)sps & 15u;
+      for (uint32_t e = lane; e < kTmaClasses * NV; e += 32) {
+        const uint32_t hk = e / NV + e % NV, cls = hk % kTmaClasses;
+        trans_tab[slot][e] = cls * TG::kClassStride + ((lead0 + cls * dlead) & 15u) + (hk / kTmaClasses) * kTmaInner;
+      }
+      __syncwarp();
+    }
+    if (lane == 0) {
+      ChunkDesc c;
+      c.mode = MODE_TRANS_TMA; c.tile = own; c.nr = R; c.nc = n; c.pitch = kTmaInner; c.pad = first;
+      c.src = (uint64_t)(uintptr_t)tile_src + (uint64_t)i0 * sps + (uint64_t)j0 * ES;
+      c.dst = (uint64_t)(uintptr_t)dst; c.sps = sps; c.dps = dps;
+      desc[slot] = c;
+      // every box counts in full, whatever part of it lies outside the tile
+      mbar_expect_tx(&slot_full[slot], kTmaClasses * TG::kBoxRows * kTmaInner);
+    }
+    __syncwarp();
+    if (lane < kTmaClasses) {
+      // the class's map starts at the 16-byte boundary at or before the first element of tile row `lane`
+      const uint32_t lead = (uint32_t)(((uintptr_t)tile_src + (uint64_t)lane * sps) & 15u);
+      const uint32_t x = ((lead + j0 * ES) >> 4) * (16 / ES);
+      tensor_load_2d(stage + lane * TG::kClassStride, tmaps + (size_t)(map0 + lane) * 128, x, i0 / kTmaClasses,
+                     &slot_full[slot]);
+    }
+    ++n_w;
+  };
   // direct ring (lane 0): store the oldest loaded chunk; one store behind, its stage is free again
   auto store_oldest = [&]() {
     const uint32_t st = n_store % kDirectStages;
@@ -270,20 +313,31 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
             push_staged(MODE_ROWS, f.s + ((size_t)r * f.ssr + c) * ES, f.d + ((size_t)r * f.dsr + c) * ED, 1,
                         min(piece, f.nc - c), 0, 0, (uint32_t)kSlotBytes);
       }
-    } else if (f.kind == KIND_TRANS && f.n_extra == 0 && (size_t)f.nc * ES >= kTransMinPiece && f.nr >= kTransMinRows) {
+    } else if (staged_trans_ok<ES>(f.kind, f.n_extra, f.nr, f.nc)) {
       // staged transposition: chunks of kTransPiece bytes of columns x kOwn rows (+ halo), rows fastest
-      constexpr uint32_t kOwn = (((uint32_t)kSlotBytes / kTransPitch) - kTransHalo) & ~7u;
-      constexpr uint32_t kCols = kTransChunkBytes / ES;
+      const uint32_t kOwn = f.tmaps ? TG::kOwnTma : TG::kOwn;
+      const uint32_t kCols = f.tmaps ? TG::kColsTma : TG::kCols;
       // no halo when every destination run starts on a 16-byte boundary: windows never straddle chunks
       const uint32_t halo = ((((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0 && kOwn % (16 / ED) == 0) ? 0u : kTransHalo;
       // equal column shares per chunk (no thin last chunk), a multiple of four columns
       const uint32_t n_col = (f.nc + kCols - 1) / kCols;
       const uint32_t cols = min(kCols, (((f.nc + n_col - 1) / n_col) + 3u) & ~3u);
-      for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cols)
-        for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += kOwn)
-          push_trans(f.s + ((size_t)i0 * f.ssr + j0) * ES, f.d + ((size_t)j0 * f.dsc + i0) * ED,
-                     min(kOwn + halo, f.nr - i0), min(cols, f.nc - j0), (uint64_t)f.ssr * ES,
-                     (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0), i0 == 0 ? 1u : 0u);
+      if (f.tmaps) {
+        // the descriptors of the next tile's maps are on their way while this tile is loaded
+        if (k + 1 < bend && lane < kTmaClasses && (nxt.c.z & kTileHasMaps))
+          tensor_map_prefetch(tmaps + (size_t)(nxt.c.w + lane) * 128);
+        for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cols)
+          for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += kOwn)
+            push_trans_tma(f.extra, f.s, i0, j0, f.d + ((size_t)j0 * f.dsc + i0) * ED, min(kOwn + halo, f.nr - i0),
+                           min(cols, f.nc - j0), (uint64_t)f.ssr * ES, (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0),
+                           i0 == 0 ? 1u : 0u);
+      } else {
+        for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cols)
+          for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += kOwn)
+            push_trans(f.s + ((size_t)i0 * f.ssr + j0) * ES, f.d + ((size_t)j0 * f.dsc + i0) * ED,
+                       min(kOwn + halo, f.nr - i0), min(cols, f.nc - j0), (uint64_t)f.ssr * ES,
+                       (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0), i0 == 0 ? 1u : 0u);
+      }
     } else {
       push_simple(MODE_COOP, k, 1, &cur);   // narrow transposes, short rows, fan-out: the workers share the tile
     }

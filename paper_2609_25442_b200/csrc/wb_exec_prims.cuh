@@ -223,6 +223,18 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
                ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Tiled 2-D tensor-map (TMA) load: the box at element coordinates (x, y) of the tensor that `map`
+// describes (a 128-byte CUtensorMap in global memory) lands densely at smem_dst (128-byte aligned)
+// and completes on the mbarrier with the box's full byte count.  x * element size must be a
+// multiple of 16 bytes.  Coordinates outside the tensor read as zero without touching memory.
+__device__ __forceinline__ void tensor_load_2d(void* smem_dst, const void* map, uint32_t x, uint32_t y, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tensor_map_prefetch(const void* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
 // Per-thread asynchronous 16-byte copy global -> shared (both 16-byte aligned), and the arrival that
 // signals an mbarrier once all earlier copies of the calling thread have landed (the pending count
 // is raised by the instruction itself, so the barrier's initial count is not involved).

@@ -42,7 +42,7 @@ constexpr int kWorkerWarps = kWorkers / 32;
 #endif
 constexpr size_t kStagedMinRowBytes = WB_STAGED_MIN_ROW_BYTES;   // shorter rows take the warp-level path
 
-enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3, MODE_TRANS = 4 };
+enum : uint32_t { MODE_END = 0, MODE_COOP = 1, MODE_ROWS = 2, MODE_BATCH = 3, MODE_TRANS = 4, MODE_TRANS_TMA = 5 };
 // Staged transposition: a chunk is kTransChunkBytes of consecutive source columns (the
 // 16-byte aligned superset of a row piece is one 16-byte asynchronous copy per lane of the producer
 // warp - bulk copies this small are limited by their issue rate) by as many source rows as fit a slot.  Row r of the chunk lands at r * kTransPitch + 16 * ((r / NV) & 7) in the slot
@@ -64,6 +64,22 @@ constexpr uint32_t kTransHalo = 8;
 #endif
 constexpr uint32_t kTransMinPiece = WB_TRANS_MIN_PIECE;   // narrower tiles stay with the warp-level transposition
 constexpr uint32_t kTransMinRows = 16;
+// Staged transposition fed by tensor-map (TMA) loads.  A tensor map wants a 16-byte aligned base and
+// row pitches that are multiples of 16 bytes, which arbitrary tiles do not have.  But eight times any
+// pitch of 2- or 4-byte elements is such a multiple: the rows of a tile are dealt to kTmaClasses = 8
+// classes by row index mod 8, and class q gets a map of its own - base = the 16-byte boundary at or
+// before the first element of row q, pitch = 8 x the tile's pitch.  A chunk is then eight loads (one box
+// of kTmaInner bytes x (rows / 8) per class) instead of a per-lane copy for every 16 bytes.  Class q's box
+// sits at q * (class stride) in the slot, its rows kTmaInner bytes apart: lanes that read one column
+// eight rows apart (neighbouring windows of a 2-byte destination run) are 124 words apart, on different
+// banks.
+constexpr uint32_t kTmaClasses = 8;
+#ifndef WB_TMA_CHUNK_BYTES
+#define WB_TMA_CHUNK_BYTES 480
+#endif
+constexpr uint32_t kTmaChunkBytes = WB_TMA_CHUNK_BYTES;   // source bytes of a chunk's row pieces
+constexpr uint32_t kTmaInner = kTmaChunkBytes + 16;       // box width in bytes: the aligned superset of a row piece
+static_assert(kTmaInner % 32 == 16, "box rows must be an odd multiple of 16 bytes apart (bank spread)");
 #ifndef WB_BATCH_TILE_BYTES
 #define WB_BATCH_TILE_BYTES 8192
 #endif
@@ -90,6 +106,7 @@ struct TileFields {
   const char* s;
   char* d;
   uint32_t nr, nc, ssr, ssc, dsr, dsc, kind, n_extra, extra;
+  bool tmaps;          // `extra` is the index of the tile's first tensor map (staged transposition by TMA)
 };
 __device__ __forceinline__ TileFields decode(const TileRegs& r, uint64_t src_add, uint64_t dst_add) {
   TileFields f;
@@ -98,6 +115,7 @@ __device__ __forceinline__ TileFields decode(const TileRegs& r, uint64_t src_add
   f.nr = r.b.x; f.nc = r.b.y; f.ssr = r.b.z; f.ssc = r.b.w;
   f.dsr = r.c.x; f.dsc = r.c.y;
   f.kind = r.c.z & 0xFF; f.n_extra = (r.c.z >> 8) & 0xFF; f.extra = r.c.w;
+  f.tmaps = (r.c.z & kTileHasMaps) != 0;
   return f;
 }
 
@@ -488,6 +506,25 @@ __device__ __forceinline__ void coop_tile(const TileFields& f, const DDst* __res
   }
 }
 
+// Which tiles take the staged transposition, and how such a tile is cut into chunks: a chunk's columns
+// x its own rows (+ halo), emitted columns outer, rows inner.
+template <int ES> __device__ __host__ __forceinline__ bool staged_trans_ok(uint32_t kind, uint32_t n_extra, uint32_t nr, uint32_t nc) {
+  return kind == KIND_TRANS && n_extra == 0 && (size_t)nc * ES >= kTransMinPiece && nr >= kTransMinRows;
+}
+template <int ES, int ED> struct TransGeom {
+  // chunks staged by per-lane copies
+  static constexpr uint32_t kOwn = (((uint32_t)Rings<ES, ED>::kSlotBytes / kTransPitch) - kTransHalo) & ~7u;
+  static constexpr uint32_t kCols = kTransChunkBytes / ES;
+  // chunks staged by tensor-map loads: the classes' boxes are kClassStride apart in a slot and hold as
+  // many rows as fit
+  static constexpr uint32_t kClassStride = ((uint32_t)Rings<ES, ED>::kSlotBytes / kTmaClasses) & ~127u;
+  static constexpr uint32_t kBoxRows = kClassStride / kTmaInner;
+  static constexpr uint32_t kOwnTma = kBoxRows * kTmaClasses - kTransHalo;
+  static constexpr uint32_t kColsTma = kTmaChunkBytes / ES;
+  static_assert(kTransHalo % kTmaClasses == 0 && kOwnTma % kTmaClasses == 0, "chunks start on a class-0 row");
+  static_assert(kTmaInner / ES <= 256 && kBoxRows <= 256, "box dimensions are limited to 256 elements");
+};
+
 // Workers: a staged transposition chunk (rows of the source in shared memory, see kTransPitch)
 // -> destination runs, dst[j*dps + i] = cast(chunk[i][j]).  A run may start at any 2-/4-byte
 // alignment in global memory; it is written in 16-byte aligned windows.  The chunk owns the windows
@@ -526,6 +563,69 @@ __device__ __forceinline__ void staged_trans(const ChunkDesc& d, const char* sta
       uint32_t v[NV];
 #pragma unroll
       for (uint32_t k = 0; k < NV; ++k) v[k] = elem(e0 + k, j);
+      uint4 x;
+      if constexpr (ED == 2)
+        x = make_uint4(pack_pair16<ES>(v[0], v[1]), pack_pair16<ES>(v[2], v[3]), pack_pair16<ES>(v[4], v[5]),
+                       pack_pair16<ES>(v[6], v[7]));
+      else
+        x = make_uint4((uint32_t)cast_raw<ES, ED>(v[0]), (uint32_t)cast_raw<ES, ED>(v[1]),
+                       (uint32_t)cast_raw<ES, ED>(v[2]), (uint32_t)cast_raw<ES, ED>(v[3]));
+      st16(out, x);
+    } else {
+      // the run ends inside this window
+      for (uint32_t e = e0; e < nl; ++e)
+        E::store(out + (size_t)(e - e0) * ED, cast_raw<ES, ED>(elem(e, j)));
+    }
+  }
+}
+
+// Workers: the same for a chunk that tensor-map loads brought in (eight per-class boxes, see
+// kTmaClasses).  Row i of the chunk has class i mod 8 and is row i / 8 of its class's box.  `tab` is the
+// shared-memory address of the producer's table for this chunk: entry (h, k), k < NV, is the offset of
+// row e0 + k from (box row of e0) * kTmaInner for a window whose first row e0 has class h - it folds the
+// class's box, the box row carry and the alignment remainder of the class's rows, so an element costs
+// one add and one shared-memory load.  Windows are numbered run by run and dealt to the threads in
+// order, as above; (run, window) of a thread advance incrementally.
+template <int ES, int ED>
+__device__ __forceinline__ void staged_trans_tma(const ChunkDesc& d, const char* stage, uint32_t t, uint32_t tab) {
+  using E = Elem<ES, ED>;
+  using TG = TransGeom<ES, ED>;
+  constexpr uint32_t NV = 16 / ED;
+  const uint32_t own = d.tile, nl = d.nr;
+  const uint32_t wins = (own + NV - 1) / NV;                   // windows per run, at most
+  const uint32_t sbase = smem_u32(stage);
+  const uint32_t lead0 = (uint32_t)d.src & 15u, dlead = (uint32_t)d.sps & 15u;
+  auto elem = [&](uint32_t i, uint32_t j) -> uint32_t {         // raw source element (i, j) of the chunk (ragged ends only)
+    return lds_raw<ES>(sbase + (i % kTmaClasses) * TG::kClassStride + (i / kTmaClasses) * kTmaInner +
+                       ((lead0 + i * dlead) & 15u) + j * ES);
+  };
+  const uint32_t dj = (uint32_t)kWorkers / wins, dw = (uint32_t)kWorkers - dj * wins;
+  uint32_t j = t / wins, w = t - j * wins;
+  for (; j < d.nc; j += dj, w += dw) {
+    if (w >= wins) {
+      w -= wins;
+      if (++j >= d.nc) break;
+    }
+    const uint64_t run = d.dst + (uint64_t)j * d.dps;           // destination element (j, first own row)
+    const uint32_t a = (uint32_t)(run / ED) & (NV - 1);
+    const uint32_t lead = a ? NV - a : 0;                       // rows before the first window that starts here
+    // those rows belong to the previous chunk's last window, except at the very start of the run
+    if (w == 0 && d.pad)
+      for (uint32_t e = 0; e < min(lead, own); ++e)
+        E::store(reinterpret_cast<char*>(run) + (size_t)e * ED, cast_raw<ES, ED>(elem(e, j)));
+    const uint32_t e0 = lead + w * NV;
+    if (e0 >= own) continue;
+    char* out = reinterpret_cast<char*>(run) + (size_t)e0 * ED;   // 16-byte aligned
+    if (e0 + NV <= nl) {
+      const uint32_t base = sbase + (e0 / kTmaClasses) * kTmaInner + j * ES;
+      const uint32_t trow = tab + (e0 % kTmaClasses) * (NV * 4);
+      uint32_t off[NV], v[NV];
+#pragma unroll
+      for (uint32_t q = 0; q < NV; q += 4)
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(off[q]), "=r"(off[q + 1]), "=r"(off[q + 2]), "=r"(off[q + 3]) : "r"(trow + q * 4));
+#pragma unroll
+      for (uint32_t k = 0; k < NV; ++k) v[k] = lds_raw<ES>(base + off[k]);
       uint4 x;
       if constexpr (ED == 2)
         x = make_uint4(pack_pair16<ES>(v[0], v[1]), pack_pair16<ES>(v[2], v[3]), pack_pair16<ES>(v[4], v[5]),

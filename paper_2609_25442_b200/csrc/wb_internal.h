@@ -97,9 +97,10 @@ struct alignas(16) DTile {
   uint32_t nr, nc;
   uint32_t ssr, ssc;
   uint32_t dsr, dsc;
-  uint32_t kind_extra;   // kind | n_extra << 8
-  uint32_t extra;
+  uint32_t kind_extra;   // kind | n_extra << 8 | kTileHasMaps
+  uint32_t extra;        // first fan-out record, or (kTileHasMaps) the tile's first tensor map
 };
+constexpr uint32_t kTileHasMaps = 1u << 16;
 static_assert(sizeof(DTile) == 48, "tile descriptor is three 16-byte words");
 
 struct alignas(16) DDst {
@@ -118,6 +119,7 @@ struct TileTable {
   DDst* d_extras = nullptr;
   uint32_t* d_cta_begin = nullptr;
   uint32_t* d_sched = nullptr;        // {next tile, blocks done} for dynamic scheduling
+  char* d_maps = nullptr;             // tensor maps (128 bytes each) of the tiles flagged kTileHasMaps
 };
 
 struct Slab {

@@ -267,14 +267,17 @@ def test_unaligned_runs(device, src_off, dst_off, dts):
 
 
 TRANS_SHAPES = [(16, 64), (17, 65), (15, 300), (40, 124), (41, 125), (63, 123), (64, 124), (65, 125), (71, 247),
-                (72, 248), (73, 249), (64, 496), (129, 497), (200, 1000), (333, 130), (1, 700), (700, 1), (8, 2048)]
+                (72, 248), (73, 249), (64, 496), (129, 497), (200, 1000), (333, 130), (1, 700), (700, 1), (8, 2048),
+                (55, 121), (56, 120), (57, 241), (87, 119), (88, 120), (89, 121), (96, 240), (176, 122), (177, 481)]
 
 
 @pytest.mark.parametrize("dts", [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)])
 @pytest.mark.parametrize("skew", [(0, 0, 0), (1, 3, 0), (2, 5, 7), (4, 8, 4)])
-def test_transposition_shapes(device, dts, skew):
+@pytest.mark.parametrize("flags", [0, wb.WB_PLAN_NO_TENSOR_MAPS])
+def test_transposition_shapes(device, dts, skew, flags):
     """dst[j, i] = cast(src[i, j]) for shapes on both sides of every block and chunk size of the
-    transposing paths, with the source starting `so` elements into its tensor, the destination `do`,
+    transposing paths (chunks staged by tensor-map loads, and - WB_PLAN_NO_TENSOR_MAPS - by per-lane
+    copies), with the source starting `so` elements into its tensor, the destination `do`,
     and the source rows `extra` elements longer than the part that is moved (so row starts fall on
     every alignment).  The oracle is numpy's transpose of the seeded bits; the element before and
     after every destination must keep the canary."""
@@ -288,7 +291,7 @@ def test_transposition_shapes(device, dts, skew):
         rl.add_tensor("R", 0, dts[1], do + R * C + 3)
         rl.add_slice(0, do, 1, R, 0, R, pitch, 0, 0, R, C)        # checkpoint (i, j) -> local do + j*R + i
         tl.freeze(); rl.freeze()
-        plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices))
+        plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices), flags=flags)
         src = RankArenas(tl.tensors, device, fill_byte=0)
         dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
         bind(plan, src, dst)
@@ -304,6 +307,30 @@ def test_transposition_shapes(device, dts, skew):
         assert np.array_equal(got[do:do + R * C], want), (R, C)
         canary = 0xCDCD if dts[1] == WB_BF16 else 0xCDCDCDCD
         assert (got[:do] == canary).all() and (got[do + R * C:] == canary).all(), (R, C)
+
+
+def test_rebinding_rebuilds_the_tensor_maps(device):
+    """The tensor maps of transposing tiles hold device addresses: binding the plan to other trainer
+    tensors (here at another alignment) must re-encode them, and the old tensors may then be freed."""
+    wl = make_workload("cfg5", "medium")
+    case = DeviceCase(wl, device)
+    want = oracle_for(case)
+    case.plan.remap()
+    torch.cuda.synchronize()
+    assert_dst_equals(case, want)
+    # a second set of trainer tensors, every one 4 bytes further from a 16-byte boundary, same contents
+    flat = [torch.zeros(t.numel() + 8, dtype=t.dtype, device=device) for t in case.src.tensors]
+    shifted = [f[4 // f.element_size():4 // f.element_size() + t.numel()] for f, t in zip(flat, case.src.tensors)]
+    for a, b in zip(shifted, case.src.tensors):
+        a.copy_(b)
+    case.plan.bind([t.data_ptr() for t in shifted], [t.data_ptr() for t in case.dst.tensors])
+    for t in case.src.tensors:
+        t.zero_()                        # reading the old tensors would now give zeros
+    case.reset_dst()
+    case.plan.remap()
+    torch.cuda.synchronize()
+    case.plan.check()
+    assert_dst_equals(case, want)
 
 
 def test_inverse_remap_restores_the_trainer(device):
