@@ -164,6 +164,13 @@ typedef struct {
 } wb_tile_view;
 
 #define WB_TILE_FANOUT_CONT 1u
+/* A transposing slab cut into tiles along its rows: the tile holding the rows just before / after
+ * this one continues the same destination runs.  The executor then writes a 16-byte destination
+ * vector that straddles the seam from the tile that holds its first row (reading the up to 7 source
+ * rows it needs from the tile after), and the tile after leaves those rows to it; the table as a
+ * whole still writes every element once.  Both tiles of a seam belong to one (sender, receiver) pair. */
+#define WB_TILE_ROWS_BEFORE 2u
+#define WB_TILE_ROWS_AFTER 4u
 
 enum { WB_TABLE_REMAP = 0, WB_TABLE_PACK = 1, WB_TABLE_UNPACK = 2 };
 

@@ -21,6 +21,7 @@ WB_TILE_FANOUT_CONT = 1
 WB_PLAN_NO_REPLICA_SPLIT = 1
 WB_PLAN_STATIC_SCHEDULE = 2
 WB_PLAN_NO_TENSOR_MAPS = 4
+WB_TILE_ROWS_BEFORE, WB_TILE_ROWS_AFTER = 2, 4
 
 STATUS_NAMES = {
     0: "WB_OK", 1: "WB_ERR_INVALID_ARG", 2: "WB_ERR_DTYPE", 3: "WB_ERR_SHAPE_MISMATCH",

@@ -134,7 +134,9 @@ bool encode_tile_maps(EncodeTiledFn encode, uint64_t tile_src, const HTile& h, C
   const uint64_t pitch = (uint64_t)h.ssr * ES;
   for (uint32_t q = 0; q < kTmaClasses; ++q) {
     const uint64_t a = tile_src + q * pitch, lead = a & 15u;
-    cuuint64_t dims[2] = {(lead + (uint64_t)h.nc * ES + 15) / 16 * 16 / ES, (h.nr - q + kTmaClasses - 1) / kTmaClasses};
+    // rows the tile may read: its own and, across a seam, the first of the tile below (see kTileRowsAfter)
+    const uint64_t rows = h.nr + ((h.seam & kTileRowsAfter) ? 16 / ED - 1 : 0);
+    cuuint64_t dims[2] = {(lead + (uint64_t)h.nc * ES + 15) / 16 * 16 / ES, (rows - q + kTmaClasses - 1) / kTmaClasses};
     cuuint64_t strides[1] = {pitch * kTmaClasses};
     cuuint32_t box[2] = {kTmaInner / ES, TransGeom<ES, ED>::kBoxRows};
     cuuint32_t estr[2] = {1, 1};
@@ -247,7 +249,7 @@ extern "C" wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, si
         dt.src = addr(h.src_tensor, h.src_off, true);
         dt.dst = addr(h.dst_tensor, h.dst_off, false);
         dt.nr = h.nr; dt.nc = h.nc; dt.ssr = h.ssr; dt.ssc = h.ssc; dt.dsr = h.dsr; dt.dsc = h.dsc;
-        dt.kind_extra = h.kind | (h.n_extra << 8);
+        dt.kind_extra = h.kind | (h.n_extra << 8) | h.seam;
         dt.extra = h.extra;
         if (ti == 0 && encode && tile_wants_maps(h, es) && pitch_ok(h, es)) {
           CUtensorMap* hm = reinterpret_cast<CUtensorMap*>(host.data() + maps_off) + n_maps;
@@ -687,7 +689,7 @@ extern "C" wb_status wb_remap_static(const wb_plan* plan, const void* const* src
     dt.src = (uint64_t)(uintptr_t)src_base[h.src_tensor] + h.src_off * es;
     dt.dst = (uint64_t)(uintptr_t)dst_base[h.dst_tensor] + h.dst_off * ed;
     dt.nr = h.nr; dt.nc = h.nc; dt.ssr = h.ssr; dt.ssc = h.ssc; dt.dsr = h.dsr; dt.dsc = h.dsc;
-    dt.kind_extra = h.kind | (h.n_extra << 8);
+    dt.kind_extra = h.kind | (h.n_extra << 8) | h.seam;
     dt.extra = h.extra;
     ht[k] = dt;
   }

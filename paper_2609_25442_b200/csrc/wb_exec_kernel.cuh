@@ -317,8 +317,15 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
       // staged transposition: chunks of kTransPiece bytes of columns x kOwn rows (+ halo), rows fastest
       const uint32_t kOwn = f.tmaps ? TG::kOwnTma : TG::kOwn;
       const uint32_t kCols = f.tmaps ? TG::kColsTma : TG::kCols;
+      constexpr uint32_t NV = 16 / ED;
       // no halo when every destination run starts on a 16-byte boundary: windows never straddle chunks
-      const uint32_t halo = ((((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0 && kOwn % (16 / ED) == 0) ? 0u : kTransHalo;
+      // (nor the seam to the tile below, if this tile's rows are whole windows)
+      const uint32_t halo = ((((uintptr_t)f.d | ((size_t)f.dsc * ED)) & 15u) == 0 && kOwn % NV == 0 &&
+                             (!f.rows_after || f.nr % NV == 0)) ? 0u : kTransHalo;
+      // source rows this tile may read: its own, and - to complete the window that straddles the seam -
+      // the first rows of the tile below
+      const uint32_t avail = f.nr + (f.rows_after ? NV - 1 : 0u);
+      // the rows before a run's first window are written here only at the top of a slab's column
       // equal column shares per chunk (no thin last chunk), a multiple of four columns
       const uint32_t n_col = (f.nc + kCols - 1) / kCols;
       const uint32_t cols = min(kCols, (((f.nc + n_col - 1) / n_col) + 3u) & ~3u);
@@ -328,15 +335,15 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
           tensor_map_prefetch(tmaps + (size_t)(nxt.c.w + lane) * 128);
         for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cols)
           for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += kOwn)
-            push_trans_tma(f.extra, f.s, i0, j0, f.d + ((size_t)j0 * f.dsc + i0) * ED, min(kOwn + halo, f.nr - i0),
+            push_trans_tma(f.extra, f.s, i0, j0, f.d + ((size_t)j0 * f.dsc + i0) * ED, min(kOwn + halo, avail - i0),
                            min(cols, f.nc - j0), (uint64_t)f.ssr * ES, (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0),
-                           i0 == 0 ? 1u : 0u);
+                           (i0 == 0 && !f.rows_before) ? 1u : 0u);
       } else {
         for (uint32_t j0 = 0; j0 < f.nc && !failed; j0 += cols)
           for (uint32_t i0 = 0; i0 < f.nr && !failed; i0 += kOwn)
             push_trans(f.s + ((size_t)i0 * f.ssr + j0) * ES, f.d + ((size_t)j0 * f.dsc + i0) * ED,
-                       min(kOwn + halo, f.nr - i0), min(cols, f.nc - j0), (uint64_t)f.ssr * ES,
-                       (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0), i0 == 0 ? 1u : 0u);
+                       min(kOwn + halo, avail - i0), min(cols, f.nc - j0), (uint64_t)f.ssr * ES,
+                       (uint64_t)f.dsc * ED, min(kOwn, f.nr - i0), (i0 == 0 && !f.rows_before) ? 1u : 0u);
       }
     } else {
       push_simple(MODE_COOP, k, 1, &cur);   // narrow transposes, short rows, fan-out: the workers share the tile

@@ -59,11 +59,7 @@ constexpr uint32_t kTransPitch = kTransPiece + 128;
 constexpr uint32_t kTransChunkBytes = 480;
 static_assert(kTransChunkBytes + 16 <= kTransPiece, "the aligned superset of a row piece must fit the copy");
 constexpr uint32_t kTransHalo = 8;
-#ifndef WB_TRANS_MIN_PIECE
-#define WB_TRANS_MIN_PIECE 128
-#endif
-constexpr uint32_t kTransMinPiece = WB_TRANS_MIN_PIECE;   // narrower tiles stay with the warp-level transposition
-constexpr uint32_t kTransMinRows = 16;
+constexpr uint32_t kTransMinPiece = kTransMinPieceBytes;   // narrower tiles stay with the warp-level transposition
 // Staged transposition fed by tensor-map (TMA) loads.  A tensor map wants a 16-byte aligned base and
 // row pitches that are multiples of 16 bytes, which arbitrary tiles do not have.  But eight times any
 // pitch of 2- or 4-byte elements is such a multiple: the rows of a tile are dealt to kTmaClasses = 8
@@ -80,10 +76,6 @@ constexpr uint32_t kTmaClasses = 8;
 constexpr uint32_t kTmaChunkBytes = WB_TMA_CHUNK_BYTES;   // source bytes of a chunk's row pieces
 constexpr uint32_t kTmaInner = kTmaChunkBytes + 16;       // box width in bytes: the aligned superset of a row piece
 static_assert(kTmaInner % 32 == 16, "box rows must be an odd multiple of 16 bytes apart (bank spread)");
-#ifndef WB_BATCH_TILE_BYTES
-#define WB_BATCH_TILE_BYTES 8192
-#endif
-constexpr uint32_t kBatchTileBytes = WB_BATCH_TILE_BYTES;   // tiles moving less than this are batched, one warp per tile
 constexpr uint32_t kBatchMaxTiles = 120;
 
 // What the producer tells the workers about one ring slot.
@@ -107,6 +99,7 @@ struct TileFields {
   char* d;
   uint32_t nr, nc, ssr, ssc, dsr, dsc, kind, n_extra, extra;
   bool tmaps;          // `extra` is the index of the tile's first tensor map (staged transposition by TMA)
+  bool rows_before, rows_after;   // see kTileRowsBefore
 };
 __device__ __forceinline__ TileFields decode(const TileRegs& r, uint64_t src_add, uint64_t dst_add) {
   TileFields f;
@@ -116,6 +109,8 @@ __device__ __forceinline__ TileFields decode(const TileRegs& r, uint64_t src_add
   f.dsr = r.c.x; f.dsc = r.c.y;
   f.kind = r.c.z & 0xFF; f.n_extra = (r.c.z >> 8) & 0xFF; f.extra = r.c.w;
   f.tmaps = (r.c.z & kTileHasMaps) != 0;
+  f.rows_before = (r.c.z & kTileRowsBefore) != 0;
+  f.rows_after = (r.c.z & kTileRowsAfter) != 0;
   return f;
 }
 

@@ -65,6 +65,24 @@ namespace wbi {
 
 enum : uint32_t { KIND_ROWS = 0, KIND_TRANS = 1, KIND_ELEM = 2 };
 
+// Which transposing tiles the executor stages through shared memory in chunks (the others are
+// transposed by single warps): tiles that move at least kBatchTileBytes, with source rows of at least
+// kTransMinPieceBytes and at least kTransMinRows of them, and one destination.  The planner needs
+// the same rule: only between two staged tiles may a 16-byte destination window cross a seam.
+#ifndef WB_TRANS_MIN_PIECE
+#define WB_TRANS_MIN_PIECE 128
+#endif
+#ifndef WB_BATCH_TILE_BYTES
+#define WB_BATCH_TILE_BYTES 8192
+#endif
+constexpr uint32_t kTransMinPieceBytes = WB_TRANS_MIN_PIECE;
+constexpr uint32_t kTransMinRows = 16;
+constexpr uint32_t kBatchTileBytes = WB_BATCH_TILE_BYTES;   // tiles moving less than this are batched, one warp per tile
+inline bool staged_transposition(uint32_t kind, uint32_t n_extra, uint64_t nr, uint64_t nc, uint32_t es, uint32_t ed) {
+  return kind == KIND_TRANS && n_extra == 0 && nc * es >= kTransMinPieceBytes && nr >= kTransMinRows &&
+         nr * nc * (es + ed) >= kBatchTileBytes;
+}
+
 // Resident thread blocks per SM the executor kernel is compiled for; the planner's default
 // grid is kNumSMs * kCtasPerSM so that one launch is exactly one wave on a B200.
 constexpr uint32_t kNumSMs = 148;
@@ -78,6 +96,7 @@ struct HTile {
   uint32_t ssr, ssc, dsr, dsc;        // element strides over (i, j)
   uint32_t kind;
   uint32_t n_extra, extra;            // fan-out destinations beyond the first
+  uint32_t seam;                      // kTileRowsBefore | kTileRowsAfter (staged transposing tiles)
   uint32_t cta;
   uint64_t bytes;                     // bytes moved (read + all writes)
 };
@@ -97,10 +116,16 @@ struct alignas(16) DTile {
   uint32_t nr, nc;
   uint32_t ssr, ssc;
   uint32_t dsr, dsc;
-  uint32_t kind_extra;   // kind | n_extra << 8 | kTileHasMaps
+  uint32_t kind_extra;   // kind | n_extra << 8 | kTileHasMaps | kTileRowsBefore | kTileRowsAfter
   uint32_t extra;        // first fan-out record, or (kTileHasMaps) the tile's first tensor map
 };
 constexpr uint32_t kTileHasMaps = 1u << 16;
+// A transposing slab cut into tiles along its rows: the tile above / below continues the same
+// destination runs and is staged too.  A 16-byte destination window that straddles such a seam is
+// written whole by the tile that holds its first row (which reads the few source rows it needs from
+// the tile below); the tile below leaves those rows alone.  Without the flags either tile writes its
+// part of the window with element stores.
+constexpr uint32_t kTileRowsBefore = 1u << 17, kTileRowsAfter = 1u << 18;
 static_assert(sizeof(DTile) == 48, "tile descriptor is three 16-byte words");
 
 struct alignas(16) DDst {

@@ -128,8 +128,9 @@ struct TileBuilder {
   bool ok = true;
 
   void emit(const Ref& src, const Ref* dsts, uint32_t n_dst, uint64_t i0, uint64_t j0,
-            uint64_t ni, uint64_t nj, uint32_t kind) {
+            uint64_t ni, uint64_t nj, uint32_t kind, uint32_t seam = 0) {
     HTile t{};
+    t.seam = seam;
     auto fits = [&](uint64_t v) { if (v >= (1ull << 32)) ok = false; return (uint32_t)v; };
     t.src_tensor = src.tensor;
     t.src_off = src.off + i0 * src.sr + j0 * src.sc;
@@ -231,10 +232,22 @@ struct TileBuilder {
       tr = std::min<uint64_t>(tr, roundup((nr + n_row - 1) / n_row, 64));
     }
     if (trans) {
-      // rows fastest: consecutive tiles continue the same destination runs
-      for (uint64_t j = 0; j < nc; j += tc)
-        for (uint64_t i = 0; i < nr; i += tr)
-          emit(src, dsts.data(), n_dst, i, j, std::min(tr, nr - i), std::min(tc, nc - j), kind);
+      // rows fastest: consecutive tiles continue the same destination runs; where two neighbours in
+      // a column are both staged by the executor, destination windows may cross their seam
+      for (uint64_t j = 0; j < nc; j += tc) {
+        const uint64_t w = std::min(tc, nc - j);
+        auto staged = [&](uint64_t i) {
+          return i < nr && staged_transposition(kind, n_dst - 1, std::min(tr, nr - i), w, es, ed);
+        };
+        for (uint64_t i = 0; i < nr; i += tr) {
+          uint32_t seam = 0;
+          if (staged(i)) {
+            if (i > 0 && staged(i - tr)) seam |= kTileRowsBefore;
+            if (staged(i + tr)) seam |= kTileRowsAfter;
+          }
+          emit(src, dsts.data(), n_dst, i, j, std::min(tr, nr - i), w, kind, seam);
+        }
+      }
       return;
     }
     for (uint64_t i = 0; i < nr; i += tr)
@@ -762,12 +775,14 @@ extern "C" wb_status wb_plan_tiles(const wb_plan* plan, int which, size_t round,
       v.src_tensor = t.src_tensor; v.src_off = t.src_off;
       v.nr = t.nr; v.nc = t.nc; v.src_sr = t.ssr; v.src_sc = t.ssc;
       v.kind = t.kind; v.cta = t.cta;
+      if (t.seam & kTileRowsBefore) v.flags |= WB_TILE_ROWS_BEFORE;
+      if (t.seam & kTileRowsAfter) v.flags |= WB_TILE_ROWS_AFTER;
       if (d == 0) {
         v.dst_tensor = t.dst_tensor; v.dst_off = t.dst_off; v.dst_sr = t.dsr; v.dst_sc = t.dsc;
       } else {
         const HDst& x = T->extras[t.extra + d - 1];
         v.dst_tensor = x.tensor; v.dst_off = x.off; v.dst_sr = x.sr; v.dst_sc = x.sc;
-        v.flags = WB_TILE_FANOUT_CONT;
+        v.flags |= WB_TILE_FANOUT_CONT;
       }
       out[count] = v;
     }

@@ -309,6 +309,46 @@ def test_transposition_shapes(device, dts, skew, flags):
         assert (got[:do] == canary).all() and (got[do + R * C:] == canary).all(), (R, C)
 
 
+ROW_SHAPES = [(16, 64), (17, 65), (40, 100), (64, 127), (100, 128), (176, 129), (177, 200), (300, 249), (301, 250),
+              (90, 252), (91, 253), (92, 254), (700, 131), (15, 200), (2000, 67)]
+
+
+@pytest.mark.parametrize("dts", [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)])
+@pytest.mark.parametrize("skew", [(0, 0, 3, 0), (1, 3, 0, 5), (2, 5, 7, 0), (4, 8, 4, 8)])
+def test_short_row_shapes(device, dts, skew):
+    """dst[i, j] = cast(src[i, j]) for rows below 1 KiB (the warp-level short-row path and the runs of
+    small tiles): the source starts `so` elements into its tensor and its rows are `sx` elements longer
+    than the part that is moved, the destination likewise with `do` and `dx`, so that row starts fall
+    on every alignment and the destination is packed or strided.  The element before and after every
+    destination row must keep the canary."""
+    so, do, sx, dx = skew
+    for (R, C) in ROW_SHAPES:
+        sp, dp = C + sx, C + dx
+        tl, rl = Layout("t"), Layout("r")
+        tl.add_tensor("T", 0, dts[0], so + R * sp)
+        rl.add_tensor("R", 0, dts[1], do + R * dp + 3)
+        # checkpoint tensor 0 is the wider [R, sp] source matrix; the rollout keeps its left C columns
+        tl.add_slice(0, so, sp, 1, 0, R, sp, 0, 0, R, sp)
+        rl.add_slice(0, do, dp, 1, 0, R, sp, 0, 0, R, C)
+        tl.freeze(); rl.freeze()
+        plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices))
+        src = RankArenas(tl.tensors, device, fill_byte=0)
+        dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+        bind(plan, src, dst)
+        rng = np.random.default_rng(R * 1000 + C)
+        bits = random_bits(rng, so + R * sp, dts[0])
+        src.tensors[0].copy_(from_bits(bits).to(device))
+        plan.remap()
+        torch.cuda.synchronize()
+        plan.check()
+        got = to_bits(dst.tensors[0])
+        want = cast_bits(np.ascontiguousarray(bits[so:].reshape(R, sp)[:, :C]).reshape(-1), dts[0], dts[1]).reshape(R, C)
+        canary = 0xCDCD if dts[1] == WB_BF16 else 0xCDCDCDCD
+        body = got[do:do + R * dp].reshape(R, dp)
+        assert np.array_equal(body[:, :C], want), (R, C)
+        assert (body[:, C:] == canary).all() and (got[:do] == canary).all() and (got[do + R * dp:] == canary).all(), (R, C)
+
+
 def test_rebinding_rebuilds_the_tensor_maps(device):
     """The tensor maps of transposing tiles hold device addresses: binding the plan to other trainer
     tensors (here at another alignment) must re-encode them, and the old tensors may then be freed."""

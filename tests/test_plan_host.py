@@ -336,6 +336,50 @@ def test_interleaved_column_blocks_are_not_an_overlap():
     assert np.array_equal(dst[0], src[0])
 
 
+@pytest.mark.parametrize("dts", [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_BF16, WB_F32)])
+def test_seam_flags_pair_up_between_staged_transposing_tiles(dts):
+    """A transposing slab is cut into tiles along its rows.  WB_TILE_ROWS_AFTER on a tile and
+    WB_TILE_ROWS_BEFORE on the tile that holds the next rows of the same columns come in pairs, only
+    between tiles the executor stages in chunks (rows of at least 128 source bytes, at least 16 of them,
+    at least 8 KiB moved), and never on other kinds of tile - in the fused table and in the unpack
+    tables alike."""
+    es = 4 if dts[0] == WB_F32 else 2
+    ed = 4 if dts[1] == WB_F32 else 2
+    found = 0
+    for (R, C, tile_bytes) in [(1000, 300, 65536), (130, 500, 4096), (2000, 40, 32768), (70, 4000, 0), (4096, 130, 0)]:
+        tl, rl = Layout("t"), Layout("r")
+        tl.add_tensor("T", 0, dts[0], R * C)
+        tl.add_slice(0, 0, C, 1, 0, R, C, 0, 0, R, C)
+        rl.add_tensor("R", 0, dts[1], R * C)
+        rl.add_slice(0, 0, 1, R, 0, R, C, 0, 0, R, C)            # checkpoint (i, j) -> local j*R + i
+        tl.freeze(); rl.freeze()
+        plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices), tile_bytes=tile_bytes,
+                       bucket_budget_bytes=1 << 20)
+        plan.verify()
+        tables = [plan.tiles(wb.WB_TABLE_REMAP)]
+        for r in range(plan.num_rounds()):
+            tables.append(plan.tiles(wb.WB_TABLE_PACK, r))
+            tables.append(plan.tiles(wb.WB_TABLE_UNPACK, r))
+        for k, t in enumerate(tables):
+            src_es = ed if (k and k % 2 == 0) else es           # an unpack table reads the bucket (rollout dtype)
+            before = (t["flags"] & wb.WB_TILE_ROWS_BEFORE) != 0
+            after = (t["flags"] & wb.WB_TILE_ROWS_AFTER) != 0
+            staged = ((t["kind"] == 1) & (t["nc"].astype(np.int64) * src_es >= 128) & (t["nr"] >= 16) &
+                      (t["nr"].astype(np.int64) * t["nc"] * (src_es + ed) >= 8192))
+            assert not (before & ~staged).any() and not (after & ~staged).any()
+            # the tile below continues the destination runs: its first element follows this tile's last row
+            below = {(int(x["dst_tensor"]), int(x["dst_off"])): i for i, x in enumerate(t)}
+            for i in np.nonzero(after)[0]:
+                x = t[i]
+                assert int(x["dst_sr"]) == 1
+                j = below.get((int(x["dst_tensor"]), int(x["dst_off"]) + int(x["nr"])))
+                assert j is not None and before[j] and int(t[j]["nc"]) == int(x["nc"])
+                assert int(t[j]["src_off"]) == int(x["src_off"]) + int(x["nr"]) * int(x["src_sr"])
+                found += 1
+            assert before.sum() == after.sum()
+    assert found > 20
+
+
 def test_flat_range_helper_gives_the_rectangles_of_a_flat_shard():
     """wb_layout_add_flat_range against brute force on ids (every element of the flat range is described
     exactly once, at the local offset it has in the shard) and against the generator's own statement."""
