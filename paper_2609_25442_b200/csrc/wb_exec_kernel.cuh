@@ -101,6 +101,8 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
   // --------------------------------- producer warp -----------------------------------------------
   const uint32_t lane = threadIdx.x;
   uint32_t n_w = 0;                     // worker-ring slots handed out so far (warp-uniform)
+  uint64_t tab_keys = 0;                // 8 bits per slot: what trans_tab[slot] was computed for (0: nothing yet)
+  static_assert(kMaxSlots <= 8, "one 8-bit key per slot");
   uint32_t n_load = 0, n_store = 0;     // direct ring positions (lane 0)
   bool failed = false;                  // warp-uniform
 
@@ -188,11 +190,14 @@ wb_exec_kernel(const DTile* __restrict__ tiles, const uint32_t* __restrict__ cta
     if (!acquire_slot()) return;
     const uint32_t slot = n_w % kSlots;
     char* stage = wring + (size_t)slot * kSlotBytes;
-    {
-      // where the rows of a destination window are in the slot: entry (h, k) is the offset of row
-      // e0 + k relative to the box row of e0, for a window whose first row e0 has class h
+    // where the rows of a destination window are in the slot: entry (h, k) is the offset of row
+    // e0 + k relative to the box row of e0, for a window whose first row e0 has class h.  It depends
+    // on the alignment of the rows only, so the chunks of a column of tiles find it in place
+    const uint32_t lead0 = (uint32_t)(((uintptr_t)tile_src + (uint64_t)j0 * ES) & 15u), dlead = (uint32_t)sps & 15u;
+    const uint32_t key = 0x80u | (lead0 >> 1 << 3) | (dlead >> 1);       // both are even and below 16
+    if (((tab_keys >> (8 * slot)) & 0xFFu) != key) {
+      tab_keys = (tab_keys & ~(0xFFull << (8 * slot))) | ((uint64_t)key << (8 * slot));
       constexpr uint32_t NV = 16 / ED;
-      const uint32_t lead0 = (uint32_t)(((uintptr_t)tile_src + (uint64_t)j0 * ES) & 15u), dlead = (uint32_t)sps & 15u;
       for (uint32_t e = lane; e < kTmaClasses * NV; e += 32) {
         const uint32_t hk = e / NV + e % NV, cls = hk % kTmaClasses;
         trans_tab[slot][e] = cls * TG::kClassStride + ((lead0 + cls * dlead) & 15u) + (hk / kTmaClasses) * kTmaInner;

@@ -8,7 +8,9 @@ namespace {
 constexpr int kWorkers = kThreads - 32;       // warps 1.. convert staged chunks and run queued tiles
 // Shared-memory rings (tuned on B200; the direct ring is very sensitive: 3 x 32 KiB moves 5 % more
 // than 4 x 16 KiB).  Kernels whose element sizes differ never use the direct ring and give all of
-// it to the worker ring.
+// it to the worker ring: five slots of 44 KiB, 220 of the 227 KiB a block can have - a slot is busy
+// for a load's latency plus the workers' time on it, so the ring's depth sets the rate of the staged
+// classes that are not DRAM-bound (transposition chunks: 4 x 48 KiB -> 5 x 44 KiB, + 4 %).
 #ifndef WB_DIRECT_STAGES
 #define WB_DIRECT_STAGES 3
 #endif
@@ -16,16 +18,16 @@ constexpr int kWorkers = kThreads - 32;       // warps 1.. convert staged chunks
 #define WB_DIRECT_BYTES 32768
 #endif
 #ifndef WB_SLOTS_SAME
-#define WB_SLOTS_SAME 3
+#define WB_SLOTS_SAME 4
 #endif
 #ifndef WB_SLOT_BYTES_SAME
 #define WB_SLOT_BYTES_SAME 32768
 #endif
 #ifndef WB_SLOTS_CAST
-#define WB_SLOTS_CAST 4
+#define WB_SLOTS_CAST 5
 #endif
 #ifndef WB_SLOT_BYTES_CAST
-#define WB_SLOT_BYTES_CAST 49152
+#define WB_SLOT_BYTES_CAST 45056
 #endif
 constexpr int kDirectStages = WB_DIRECT_STAGES;   // bulk ring of the direct (load -> store) path
 constexpr int kDirectBytes = WB_DIRECT_BYTES;
