@@ -256,6 +256,10 @@ wb_status wb_plan_tiles(const wb_plan* plan, int which, size_t round, wb_tile_vi
  * must not alias each other.  The kernels fetch whole 16-byte units: they may READ (never write)
  * the up to 15 bytes between a run's first / last element and the enclosing 16-byte boundaries,
  * which always lie inside the same device allocation (allocations are at least 256-byte granular).
+ * For the transposing tiles of the fused table whose rows are staged through shared memory the call
+ * also encodes tensor maps of the bound source addresses (8 x 128 bytes per tile, in the same device
+ * allocation; the driver's cuTensorMapEncodeTiled is looked up at run time, and without it - or under
+ * WB_PLAN_NO_TENSOR_MAPS - the kernels copy those rows lane by lane instead).
  * Errors: INVALID_ARG, OOM, CUDA. */
 wb_status wb_plan_bind(wb_plan* plan, const void* const* src_base, size_t n_src,
                        void* const* dst_base, size_t n_dst);

@@ -11,9 +11,10 @@
 //            global through a small ring; the data never touches registers.
 //   staged   other ROWS tiles with rows of at least kStagedMinRowBytes: the producer warp bulk-
 //            loads the rows into a ring slot, the workers realign, cast and store 16 bytes at a time.
-//   staged   transposing tiles: the producer warp copies chunks of source rows into a ring slot
-//   transp.  (per-lane asynchronous copies, bank-swizzled rows), the workers write 16-byte windows
-//            of the destination runs, neighbouring lanes on neighbouring windows of one run.
+//   staged   transposing tiles: the producer warp brings chunks of source rows into a ring slot - eight
+//   transp.  2-D tensor-map (TMA) loads per chunk where wb_plan_bind could encode maps (the fused table),
+//            per-lane asynchronous copies into bank-swizzled rows otherwise; the workers write 16-byte
+//            windows of the destination runs, neighbouring lanes on neighbouring windows of one run.
 //   queued   everything else is handed to the workers by tile index, either one tile shared by all
 //            worker warps or a run of small tiles, one warp per tile.
 //
