@@ -99,7 +99,8 @@ typedef struct {
   uint32_t tile_bytes;          /* target bytes moved (read + written) per tile; 0 = auto   */
   uint32_t grid_ctas;           /* thread blocks per launch; 0 = auto (multiple of 148 SMs) */
   uint32_t flags;               /* WB_PLAN_* bits                                           */
-  uint32_t reserved;
+  uint32_t host_group_kib;      /* wb_remap_host: KiB moved (read + written) per pipeline stage;
+                                   0 = auto (1/24 of the transfer, at least 256 MiB)        */
 } wb_plan_opts;
 
 #define WB_PLAN_NO_REPLICA_SPLIT 1u /* read replicated source regions from the lowest rank

@@ -52,7 +52,7 @@ class wb_slice(C.Structure):
 
 class wb_plan_opts(C.Structure):
     _fields_ = [("bucket_budget_bytes", C.c_uint64), ("tile_bytes", C.c_uint32),
-                ("grid_ctas", C.c_uint32), ("flags", C.c_uint32), ("reserved", C.c_uint32)]
+                ("grid_ctas", C.c_uint32), ("flags", C.c_uint32), ("host_group_kib", C.c_uint32)]
 
 
 class wb_plan_stats_t(C.Structure):
@@ -211,9 +211,9 @@ class Plan:
     """Owns a wb_plan*."""
 
     def __init__(self, trainer: Layout, rollout: Layout, bucket_budget_bytes: int = 0,
-                 tile_bytes: int = 0, grid_ctas: int = 0, flags: int = 0):
+                 tile_bytes: int = 0, grid_ctas: int = 0, flags: int = 0, host_group_kib: int = 0):
         lib = load()
-        opts = wb_plan_opts(bucket_budget_bytes, tile_bytes, grid_ctas, flags, 0)
+        opts = wb_plan_opts(bucket_budget_bytes, tile_bytes, grid_ctas, flags, host_group_kib)
         self.handle = C.c_void_p()
         self.n_src, self.n_dst = trainer.n_tensors, rollout.n_tensors
         _check(lib.wb_plan_build(trainer.handle, rollout.handle, C.byref(opts), C.byref(self.handle)),

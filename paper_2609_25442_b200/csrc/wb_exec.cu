@@ -510,7 +510,8 @@ static wb_status build_host_groups(wb_plan* plan) {
   const uint32_t es = esize(plan->src.dtype), ed = esize(plan->dst.dtype);
   uint64_t total = 0;
   for (const HTile& t : T.tiles) total += t.bytes;
-  const uint64_t target = std::max<uint64_t>(256ull << 20, total / 24);
+  const uint64_t target = plan->opts.host_group_kib ? (uint64_t)plan->opts.host_group_kib << 10
+                                                    : std::max<uint64_t>(256ull << 20, total / 24);
   plan->host_groups.clear();
   HostGroup g{};
   uint64_t acc = 0;
@@ -543,7 +544,9 @@ static wb_status build_host_groups(wb_plan* plan) {
   };
   for (uint32_t k = 0; k < T.tiles.size(); ++k) {
     const HTile& t = T.tiles[k];
-    touch(smin, stouched, t.src_tensor, t.src_off, t.nr, t.nc, t.ssr, t.ssc);
+    // a transposing tile flagged kTileRowsAfter also reads the first rows of the tile below (the window
+    // that straddles the seam), which may belong to a later group
+    touch(smin, stouched, t.src_tensor, t.src_off, t.nr + ((t.seam & kTileRowsAfter) ? 16 / ed - 1 : 0), t.nc, t.ssr, t.ssc);
     touch(dmin, dtouched, t.dst_tensor, t.dst_off, t.nr, t.nc, t.dsr, t.dsc);
     for (uint32_t x = 0; x < t.n_extra; ++x) {
       const HDst& o = T.extras[t.extra + x];

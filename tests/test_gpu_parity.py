@@ -401,6 +401,26 @@ def test_remap_from_host_buffers(device):
         assert np.array_equal(to_bits(t), want.dst[k])
 
 
+@pytest.mark.parametrize("name,scale,kib", [("cfg5", "medium", 512), ("cfg3", "medium", 2048), ("cfg2", "medium", 4096)])
+def test_remap_from_host_buffers_in_many_stages(device, name, scale, kib):
+    """wb_remap_host with small pipeline stages: a stage's kernel may only read what its own uploads
+    brought (the trainer tensors on the device hold zeros beforehand), including the source rows a
+    transposing tile reads across the seam to the tile below, which may belong to the next stage."""
+    wl = make_workload(name, scale)
+    case = DeviceCase(wl, device, host_group_kib=kib)
+    want = oracle_for(case)
+    host_src = [t.cpu().pin_memory() for t in case.src.tensors]
+    host_dst = [torch.full(t.shape, -1, dtype=torch.int16 if t.element_size() == 2 else torch.int32).view(t.dtype).pin_memory()
+                for t in case.dst.tensors]
+    for a in case.src.arenas.values():
+        a.zero_()
+    case.plan.remap_host([t.data_ptr() for t in host_src], [t.data_ptr() for t in host_dst])
+    torch.cuda.synchronize()
+    case.plan.check()
+    for k, t in enumerate(host_dst):
+        assert np.array_equal(to_bits(t), want.dst[k]), k
+
+
 def test_empty_layouts_launch_nothing(device):
     tl, rl = Layout("t"), Layout("r")
     tl.add_tensor("T", 0, WB_F32, 16)
