@@ -87,22 +87,56 @@ template <int ES> __device__ __forceinline__ uint32_t abs_word(uint32_t w) {
   return max((w << 16) & 0x7FFFFFFFu, w & 0x7FFF0000u);
 }
 
+// One work item (tile) at a time for the whole block, drawn from a counter in device memory.
+__device__ __forceinline__ uint32_t next_tile(uint32_t* counter, uint32_t* slot) {
+  __syncthreads();                                   // everyone is done with the previous value
+  if (threadIdx.x == 0) *slot = atomicAdd(counter, 1u);
+  __syncthreads();
+  return *slot;
+}
+
 // amax: magnitudes are compared as unsigned integers of the sign-cleared fp32 patterns (a NaN wins).
 // A warp takes a run; the part between 16-byte boundaries is read with 16-byte loads, four in
-// flight per lane, the ends element by element.
+// flight per lane, the ends element by element.  Items whose runs are short (a column piece of a
+// wider matrix) are read as one flat sequence of n0 * n1 elements instead, a lane taking every 32nd
+// element (coalesced inside each run; run and column advance incrementally) with eight loads in
+// flight: one run per warp and round trip would leave the memory idle.  Eight blocks per SM.
 template <int ES, int ED>
-__global__ void __launch_bounds__(256)
-wb_absmax_kernel(const AmaxItem* __restrict__ items, uint32_t n_items, uint32_t* __restrict__ amax) {
+__global__ void __launch_bounds__(256, 8)
+wb_absmax_kernel(const AmaxItem* __restrict__ items, uint32_t n_items, uint32_t* __restrict__ amax,
+                 uint32_t* __restrict__ counter) {
   __shared__ uint32_t warp_max[8];
+  __shared__ uint32_t slot;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr uint32_t PER = 16 / ES;
-  for (uint32_t k = blockIdx.x; k < n_items; k += gridDim.x) {
+  for (uint32_t k = next_tile(counter, &slot); k < n_items; k = next_tile(counter, &slot)) {
     const AmaxItem it = items[k];
     uint32_t m = 0;
+    constexpr uint32_t kShortRunBytes = 1024;
+    const bool short_runs = it.n0 > 1 && it.n1 * ES < kShortRunBytes;
+    if (short_runs) {
+      constexpr int U = 8;
+      const uint32_t n1 = it.n1, total = it.n0 * n1;       // an item has about kItemElems elements
+      const uint32_t q32 = 32 / n1, r32 = 32 % n1;
+      for (uint32_t e0 = warp * (32 * U); e0 < total; e0 += 8 * 32 * U) {
+        uint32_t i = (e0 + lane) / n1, j = (e0 + lane) - i * n1;
+        uint32_t x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          x[u] = 0;
+          if (e0 + lane + 32u * u < total)
+            x[u] = abs_elem<ES>(reinterpret_cast<const char*>(it.a) + ((size_t)i * it.s0 + j) * ES);
+          i += q32; j += r32;
+          if (j >= n1) { j -= n1; ++i; }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) m = max(m, x[u]);
+      }
+    }
     // the warps share the item's runs in segments of kSeg elements (a flat shard is one long run)
     constexpr uint32_t kSeg = 8192;
     const uint32_t segs = (it.n1 + kSeg - 1) / kSeg;
-    for (uint32_t t = warp; t < it.n0 * segs; t += 8) {
+    for (uint32_t t = warp; t < it.n0 * segs && !short_runs; t += 8) {
       const uint32_t i = t / segs, sg = t - i * segs;
       const char* row = reinterpret_cast<const char*>(it.a) + ((size_t)i * it.s0 + (size_t)sg * kSeg) * ES;
       const uint32_t n1 = min(kSeg, it.n1 - sg * kSeg);
@@ -133,7 +167,6 @@ wb_absmax_kernel(const AmaxItem* __restrict__ items, uint32_t n_items, uint32_t*
       if (ES == 4 && ED == 2) m = f32_to_bf16_bits(m) << 16;
       if (m) atomicMax(amax + it.ckpt, m);
     }
-    __syncthreads();
   }
 }
 
@@ -287,14 +320,6 @@ template <int EDP> __device__ __forceinline__ void dequant_store(char* d, uint32
   const float f = __fmul_rn(e4m3x2_to_f32x2(code).x, s);
   if (EDP == 2) *reinterpret_cast<uint16_t*>(d) = (uint16_t)(f32x2_to_bf16x2(f, 0.f) & 0xFFFFu);
   else *reinterpret_cast<float*>(d) = f;
-}
-
-// One tile at a time for the whole block.
-__device__ __forceinline__ uint32_t next_tile(uint32_t* counter, uint32_t* slot) {
-  __syncthreads();                                   // everyone is done with the previous value
-  if (threadIdx.x == 0) *slot = atomicAdd(counter, 1u);
-  __syncthreads();
-  return *slot;
 }
 
 template <int ES, int EDP>
@@ -617,7 +642,7 @@ struct QuantTables {
   std::vector<uint32_t> n_round;
   // fused quantising pack / dequantising unpack: checkpoint index of every tile, one tile counter per launch
   std::vector<uint32_t*> d_pack_ckpt, d_unpack_ckpt;
-  uint32_t* d_counters = nullptr;         // 2 per round: [2r] pack, [2r + 1] unpack
+  uint32_t* d_counters = nullptr;         // 2 per round: [2r] pack, [2r + 1] unpack; then one for the amax pass
 };
 
 wb_status build_tables(wb_plan* plan) {
@@ -654,7 +679,7 @@ wb_status build_tables(wb_plan* plan) {
   size_t bytes = amax.size() * sizeof(AmaxItem) + 256;
   for (auto& v : rounds) bytes += v.size() * sizeof(QuantItem) + 256;
   for (const Round& R : plan->rounds) bytes += up256(R.pack_ckpt.size() * 4) + up256(R.unpack_ckpt.size() * 4);
-  bytes += up256(plan->rounds.size() * 8) + 256;
+  bytes += up256(plan->rounds.size() * 8 + 8) + 256;
   auto* T = new (std::nothrow) QuantTables;
   if (!T) return WB_ERR_OOM;
   if (cudaMalloc(&T->d_mem, bytes) != cudaSuccess) { delete T; return WB_ERR_OOM; }
@@ -679,7 +704,7 @@ wb_status build_tables(wb_plan* plan) {
     off += up256(R.unpack_ckpt.size() * 4);
   }
   T->d_counters = reinterpret_cast<uint32_t*>(static_cast<char*>(T->d_mem) + off);
-  off += up256(plan->rounds.size() * 8);
+  off += up256(plan->rounds.size() * 8 + 8);
   if (cudaMemcpy(T->d_mem, host.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
     cudaFree(T->d_mem);
     delete T;
@@ -730,9 +755,11 @@ extern "C" wb_status wb_absmax(const wb_plan* plan_c, float* amax, void* cuda_st
   if (T->n_amax == 0) return WB_OK;
   const uint32_t es = esize(plan->src.dtype), ed = esize(plan->dst.dtype), grid = grid_for(T->n_amax);
   uint32_t* out = reinterpret_cast<uint32_t*>(amax);
-  if (es == 4 && ed == 2) wb_absmax_kernel<4, 2><<<grid, 256, 0, stream>>>(T->d_amax, T->n_amax, out);
-  else if (es == 4) wb_absmax_kernel<4, 4><<<grid, 256, 0, stream>>>(T->d_amax, T->n_amax, out);
-  else wb_absmax_kernel<2, 2><<<grid, 256, 0, stream>>>(T->d_amax, T->n_amax, out);   // bf16 widens exactly
+  uint32_t* counter = T->d_counters + 2 * plan->rounds.size();      // the slot after the rounds' counters
+  if (cudaMemsetAsync(counter, 0, sizeof(uint32_t), stream) != cudaSuccess) return WB_ERR_CUDA;
+  if (es == 4 && ed == 2) wb_absmax_kernel<4, 2><<<grid, 256, 0, stream>>>(T->d_amax, T->n_amax, out, counter);
+  else if (es == 4) wb_absmax_kernel<4, 4><<<grid, 256, 0, stream>>>(T->d_amax, T->n_amax, out, counter);
+  else wb_absmax_kernel<2, 2><<<grid, 256, 0, stream>>>(T->d_amax, T->n_amax, out, counter);   // bf16 widens exactly
   return cudaGetLastError() == cudaSuccess ? WB_OK : WB_ERR_CUDA;
 }
 
