@@ -309,6 +309,65 @@ def test_transposition_shapes(device, dts, skew, flags):
         assert (got[:do] == canary).all() and (got[do + R * C:] == canary).all(), (R, C)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_fuzz_transposing_slabs(device, seed):
+    """Random transposed slabs - rows 8..3000, columns 8..1200, every offset and pitch remainder on
+    both sides, one to three destination tensors, tile sizes from 4 KiB up, all four dtype pairs, with
+    and without tensor maps - through the fused call, the two-pass rounds and the staged host call.
+    The oracle is numpy's transpose of the seeded bits; gaps and padding must keep the canary."""
+    rng = np.random.default_rng(4000 + seed)
+    for case in range(40):
+        dts = [(WB_F32, WB_BF16), (WB_BF16, WB_BF16), (WB_F32, WB_F32), (WB_BF16, WB_F32)][case % 4]
+        R, C = int(rng.integers(8, 3000)), int(rng.integers(8, 1200))
+        so, do, sx, dx = (int(rng.integers(0, 9)) for _ in range(4))
+        sp, dp = C + sx, R + dx
+        k = int(rng.integers(1, 4))
+        tl, rl = Layout("t"), Layout("r")
+        tl.add_tensor("T", 0, dts[0], so + R * sp)
+        tl.add_slice(0, so, sp, 1, 0, R, sp, 0, 0, R, sp)
+        bounds = [int(b) for b in np.linspace(0, C, k + 1)]
+        parts = [(bounds[g], bounds[g + 1]) for g in range(k) if bounds[g + 1] > bounds[g]]
+        for g, (c0, c1) in enumerate(parts):
+            t = rl.add_tensor(f"R{g}", g % 2, dts[1], do + (c1 - c0) * dp + 3)
+            rl.add_slice(t, do, 1, dp, 0, R, sp, 0, c0, R, c1 - c0)      # checkpoint (i, j) -> do + (j - c0) * dp + i
+        tl.freeze(); rl.freeze()
+        plan = wb.Plan(wb.Layout(tl.tensors, tl.slices), wb.Layout(rl.tensors, rl.slices),
+                       tile_bytes=int(rng.choice([0, 4096, 16384, 65536])),
+                       flags=int(rng.choice([0, 0, wb.WB_PLAN_NO_TENSOR_MAPS])),
+                       bucket_budget_bytes=int(rng.choice([0, 1 << 18])), host_group_kib=int(rng.choice([64, 512])))
+        src = RankArenas(tl.tensors, device, fill_byte=0)
+        dst = RankArenas(rl.tensors, device, fill_byte=CANARY)
+        bind(plan, src, dst)
+        bits = random_bits(rng, so + R * sp, dts[0])
+        src.tensors[0].copy_(from_bits(bits).to(device))
+        if case % 3 == 0:
+            plan.remap()
+        elif case % 3 == 1:
+            for r in range(plan.num_rounds()):
+                bucket = torch.empty(plan.bucket_bytes(r) + 16, dtype=torch.uint8, device=device)
+                plan.pack(r, bucket.data_ptr())
+                plan.unpack(r, bucket.data_ptr())
+        else:
+            hs = [t.cpu().pin_memory() for t in src.tensors]
+            hd = [t.cpu().pin_memory() for t in dst.tensors]
+            for a in src.arenas.values():
+                a.zero_()
+            plan.remap_host([t.data_ptr() for t in hs], [t.data_ptr() for t in hd])
+            torch.cuda.synchronize()
+            for t, h in zip(dst.tensors, hd):
+                t.copy_(h)
+        torch.cuda.synchronize()
+        plan.check()
+        m = bits[so:].reshape(R, sp)
+        canary = 0xCDCD if dts[1] == WB_BF16 else 0xCDCDCDCD
+        for g, (c0, c1) in enumerate(parts):
+            got = to_bits(dst.tensors[g])
+            want = cast_bits(np.ascontiguousarray(m[:, c0:c1].T).reshape(-1), dts[0], dts[1]).reshape(c1 - c0, R)
+            body = got[do:do + (c1 - c0) * dp].reshape(c1 - c0, dp)
+            assert np.array_equal(body[:, :R], want), (seed, case, R, C, g)
+            assert (body[:, R:] == canary).all() and (got[:do] == canary).all() and (got[do + (c1 - c0) * dp:] == canary).all(), (seed, case)
+
+
 ROW_SHAPES = [(16, 64), (17, 65), (40, 100), (64, 127), (100, 128), (176, 129), (177, 200), (300, 249), (301, 250),
               (90, 252), (91, 253), (92, 254), (700, 131), (15, 200), (2000, 67)]
 
